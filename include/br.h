@@ -1,0 +1,195 @@
+/*
+ * br.h -- C-ABI of the basis-rotation optimizer step for NVIDIA B200 (sm_100a).
+ *
+ * One handle owns the optimizer state of a set of independent weight matrices
+ * ("layers").  Each call of br_step() submits one gradient per layer and applies
+ * the update that is due under a delay of tau calls:
+ *
+ *   Algorithm 1 ("Adam with Basis Rotation") of the paper, per W in R^{m x n}:
+ *     M  <- beta1 M + (1-beta1) G
+ *     if t mod freq == 0:  U, V <- Eigenbasis-Estimation (Algorithm 2)
+ *     G~ <- U^T G V ;  M~ <- U^T M V
+ *     V~ <- beta2 V~ + (1-beta2) G~ .* G~
+ *     W  <- W - eta U ( M~ / sqrt(V~ + eps) ) V^T
+ *   Algorithm 2, source S in {1st, 2nd} x geometry in {unilateral, bilateral}:
+ *     S=2nd: L <- beta L + (1-beta) G G^T, U <- Power(L, U); bilateral: same with R = G^T G, V
+ *     S=1st: U <- Power(M M^T, U); bilateral: V <- Power(M^T M, V)
+ *     unilateral: only the smaller dimension is rotated (Sec. 3.2)
+ *   Power(A, Q) = Q-factor of the QR decomposition of A Q (Sec. 3.2), made unique
+ *   by a positive diagonal of R.
+ *   Geometry NONE is plain Adam as Eq. (adam) writes it: eps inside the square
+ *   root, no bias correction.
+ *   Delay (App. B, Eq. delayed_grad): the gradient applied at a call is the one
+ *   submitted tau calls earlier; the first tau calls apply no update.
+ *
+ * All pointers named DEVICE are CUDA device pointers on the handle's device; all
+ * others are host pointers.  Matrices are row-major and contiguous.  Every entry
+ * point returns a br_status: 0 = ok, > 0 informational (state is valid), < 0
+ * error.  An error detected on the host leaves the handle unchanged.  Work is
+ * enqueued on the handle's stream; only the calls documented as synchronising
+ * wait for it.  There is no CPU fallback: every step of the path runs in CUDA
+ * kernels, and the calls fail with BR_ERR_CUDA when no device is usable.
+ */
+#ifndef BR_H_
+#define BR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define BR_API __attribute__((visibility("default")))
+#else
+#define BR_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct br_handle br_handle; /* opaque; owned by the library */
+
+typedef enum {
+  BR_OK = 0,
+  BR_WARMUP = 1,              /* no layer applied an update (call index <= tau)            */
+  BR_WARN_RANK_DEFICIENT = 2, /* a refresh met a numerically rank-deficient factor         */
+  BR_ERR_INVALID = -1,        /* NULL pointer, bad enum, bad hyper-parameter               */
+  BR_ERR_SHAPE = -2,
+  BR_ERR_DTYPE = -3,
+  BR_ERR_TAU = -4,            /* tau outside [0, tau_max]                                  */
+  BR_ERR_OOM = -5,            /* allocator returned NULL; br_last_error has the byte count */
+  BR_ERR_CUDA = -6,
+  BR_ERR_STATE = -7,          /* e.g. forced refresh before the first update               */
+  BR_ERR_TIMEOUT = -8         /* a bounded device-side wait gave up (status word)          */
+} br_status;
+
+typedef enum { BR_GEOM_NONE = 0, BR_GEOM_UNILATERAL = 1, BR_GEOM_BILATERAL = 2 } br_geometry;
+typedef enum { BR_SRC_FIRST = 1, BR_SRC_SECOND = 2 } br_source;
+typedef enum { BR_F32 = 0, BR_BF16 = 1 } br_dtype;
+/* Arithmetic of the rotation / factor contractions.
+ *   BR_GEMM_FP32: fp32 FFMA kernels (relative error ~1e-7 per product).
+ *   BR_GEMM_BF16: tcgen05 tensor-core tiles on bf16 operands with fp32 accumulation in
+ *   tensor memory; fp32 operands of the forward rotations are carried as a bf16 hi/lo pair.
+ *   Layers whose dimensions are not multiples of 8 always use the fp32 kernels. */
+typedef enum { BR_GEMM_FP32 = 0, BR_GEMM_BF16 = 2 } br_gemm_prec;
+/* When L and R are accumulated: at every update (default), or only inside the refresh as
+ * Algorithm 2 literally places the line. */
+typedef enum { BR_ACCUM_EVERY_STEP = 0, BR_ACCUM_ON_REFRESH = 1 } br_accum_mode;
+
+typedef struct {
+  int64_t m, n;        /* W is m x n, row-major, leading dimension n                        */
+  int32_t geom;        /* br_geometry                                                      */
+  int32_t src;         /* br_source (ignored for BR_GEOM_NONE)                             */
+  int32_t grad_dtype;  /* br_dtype of the gradients passed to br_step                      */
+  int32_t tau_max;     /* ring capacity in calls for this layer, >= 0                      */
+  int32_t freq;        /* refresh period in updates; <= 0 -> br_hparams.freq               */
+  int32_t reserved;
+  float* weight;       /* DEVICE fp32 m*n, owned by the caller, updated in place           */
+} br_layer_desc;
+
+typedef struct {
+  float lr, beta1, beta2, eps, weight_decay; /* weight decay is decoupled; paper default 0 here */
+  float beta_factor;   /* EMA rate of L and R; < 0 -> beta2 (Algorithm 2 reuses beta2)       */
+  int32_t freq;        /* default refresh period, >= 1 (the paper uses 10)                  */
+  int32_t power_iters; /* Power() applications per refresh, >= 1 (the paper uses 1)         */
+  int32_t accum;       /* br_accum_mode                                                    */
+  int32_t gemm_prec;   /* br_gemm_prec                                                     */
+  uint32_t flags;      /* reserved, 0                                                      */
+  int32_t reserved;
+  uint64_t scratch_limit_bytes; /* cap on per-step transient scratch; 0 -> library default */
+} br_hparams;
+
+/* Device-memory allocator.  NULL (or NULL members) -> cudaMalloc / cudaFree.  alloc returns a
+ * DEVICE pointer aligned to at least 256 bytes, or NULL. */
+typedef struct {
+  void* (*alloc)(size_t bytes, void* ctx);
+  void (*free)(void* ptr, void* ctx);
+  void* ctx;
+} br_allocator;
+
+typedef struct {
+  int64_t calls;          /* br_step calls so far (handle-wide)                              */
+  int64_t t;              /* updates applied to this layer (Algorithm 1's t)                 */
+  int64_t ring_slot;      /* ring slot the next call writes: calls mod tau_max (0 if no ring) */
+  int64_t refresh_count;  /* refreshes done for this layer, scheduled and forced             */
+  int64_t next_refresh_t; /* next t with t mod freq == 0                                     */
+} br_counters;
+
+typedef enum {
+  BR_BUF_W = 0,   /* m*n fp32                                         */
+  BR_BUF_M = 1,   /* m*n fp32, original space                         */
+  BR_BUF_V2 = 2,  /* m*n fp32, V~ in the rotated space                */
+  BR_BUF_U = 3,   /* m*m fp32 (absent when the left side is unrotated) */
+  BR_BUF_V = 4,   /* n*n fp32 (absent when the right side is unrotated) */
+  BR_BUF_L = 5,   /* m*m fp32 (S=2nd, left side rotated)              */
+  BR_BUF_R = 6,   /* n*n fp32 (S=2nd, right side rotated)             */
+  BR_BUF_RING = 7 /* tau_max * m*n gradients in grad_dtype, slot-major */
+} br_buf;
+
+/* Bytes of device memory br_create would request for these layers (state, ring, operand
+ * shadows and scratch).  Host only.  App. H's table is overhead_bytes: rotation matrices
+ * plus factor buffers in fp32, summed over layers (either out pointer may be NULL). */
+BR_API br_status br_state_bytes(const br_layer_desc* layers, int n_layers, const br_hparams* hp,
+                         size_t* total_bytes, size_t* overhead_bytes);
+
+/* Create a handle on `device`, enqueueing on `cuda_stream` (a cudaStream_t cast to void*;
+ * NULL = the legacy default stream).  State starts as M = V~ = L = R = 0, U = V = I, t = 0.
+ * Layer descriptors and hyper-parameters are copied.  Synchronises the stream once. */
+BR_API br_status br_create(br_handle** out, const br_layer_desc* layers, int n_layers,
+                    const br_hparams* hp, int device, void* cuda_stream,
+                    const br_allocator* alloc);
+
+/* One call of the delayed step.  grads: host array of n_layers DEVICE pointers, each m*n
+ * elements of the layer's grad_dtype, owned by the caller and read only by the work this call
+ * enqueues (the caller may overwrite them once the stream has passed that work).
+ * tau in [0, tau_max] applies to every layer; tau = -1 uses each layer's own tau_max.
+ * Returns BR_WARMUP when no layer applied an update.  Does not synchronise. */
+BR_API br_status br_step(br_handle* h, const void* const* grads, int tau);
+
+/* Learning rate eta_t used by the following steps. */
+BR_API br_status br_set_lr(br_handle* h, float lr);
+
+/* Run the Power() part of Algorithm 2 now, from the current L, R (S=2nd) or M (S=1st);
+ * layer = -1 refreshes every rotated layer.  Does not change t.  BR_ERR_STATE if a target
+ * layer has t == 0 (its factor is all zero). */
+BR_API br_status br_refresh_basis(br_handle* h, int layer);
+
+/* Wait for the stream and return the device status word (BR_OK, BR_WARN_RANK_DEFICIENT,
+ * BR_ERR_TIMEOUT ...); the word is cleared when it held a warning. */
+BR_API br_status br_sync_status(br_handle* h);
+
+BR_API br_status br_get_counters(br_handle* h, int layer, br_counters* out);
+BR_API br_status br_set_counters(br_handle* h, int layer, const br_counters* in);
+
+/* Copy a state buffer to / from HOST memory; `bytes` must equal the buffer's size.
+ * Both synchronise the stream.  Setting U or V also refreshes the operand shadows. */
+BR_API br_status br_get_state(br_handle* h, int layer, int which, void* host_dst, size_t bytes);
+BR_API br_status br_set_state(br_handle* h, int layer, int which, const void* host_src, size_t bytes);
+
+/* Counts of the library's own kernel launches and of floating-point operations issued by its
+ * contraction kernels since creation (for benchmarks). */
+BR_API br_status br_get_launch_stats(br_handle* h, int64_t* kernel_launches, double* gemm_flops);
+
+/* Free everything the handle allocated.  NULL is accepted.  Synchronises the stream. */
+BR_API br_status br_destroy(br_handle* h);
+
+BR_API const char* br_strerror(int status);
+/* Message of the last error on this handle (or of the last failed br_create when h is NULL). */
+BR_API const char* br_last_error(const br_handle* h);
+
+/*
+ * Stand-alone contraction entry point (used by tests and profiling of the tensor-core tile
+ * kernel): D = sum_p A_p * B_p^T with bf16 operands and fp32 accumulation, where A_p is
+ * Md x K and B_p is Nd x K.  a_mn / b_mn != 0 means the operand is stored with its M (or N)
+ * index contiguous, i.e. as a K x Md (K x Nd) row-major array; otherwise K is contiguous.
+ * lda / ldb are leading dimensions in elements.  D (fp32, ld = ldd) receives
+ * alpha * acc + beta * D.  All pointers DEVICE; dims and leading dimensions multiples of 8.
+ * Enqueues on `cuda_stream`, does not synchronise.  n_pairs in [1, 3].
+ */
+BR_API br_status br_gemm_bf16(void* cuda_stream, int64_t Md, int64_t Nd, int64_t K, int n_pairs,
+                       const void* const* A, const void* const* B, int a_mn, int b_mn,
+                       int64_t lda, int64_t ldb, float* D, int64_t ldd, float alpha, float beta);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BR_H_ */

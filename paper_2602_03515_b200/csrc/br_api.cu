@@ -1,0 +1,636 @@
+// Host side of libbr: handle, validation, integer state (calls, t, ring slots, refresh schedule),
+// memory layout and the launch plan of one delayed rotated-Adam step.  See include/br.h for the
+// contract of every entry point.
+#include <algorithm>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <string>
+#include <vector>
+
+#include "br_internal.h"
+#include "step_tc.h"
+
+using namespace br;
+
+namespace {
+
+thread_local std::string g_create_error;
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+}  // namespace
+
+namespace br {
+
+std::string format(const char* fmt, ...) {
+  char buf[512];
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(buf, sizeof buf, fmt, ap);
+  va_end(ap);
+  return std::string(buf);
+}
+
+size_t dtype_size(int dt) { return dt == BR_BF16 ? 2 : 4; }
+
+// Which sides carry a rotation: unilateral rotates the smaller dimension (Sec. 3.2), ties left.
+void rotated_sides(int64_t m, int64_t n, int geom, bool* left, bool* right) {
+  *left = *right = false;
+  if (geom == BR_GEOM_BILATERAL) { *left = *right = true; }
+  else if (geom == BR_GEOM_UNILATERAL) { *left = (m <= n); *right = (m > n); }
+}
+
+}  // namespace br
+
+// ---------------------------------------------------------------------------------------------
+// Validation and memory layout (host only)
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+br_status validate(const br_layer_desc* layers, int n_layers, const br_hparams* hp, std::string* err) {
+  if (!layers || !hp || n_layers <= 0) { *err = "NULL layers/hparams or n_layers <= 0"; return BR_ERR_INVALID; }
+  if (!(hp->beta1 >= 0.f && hp->beta1 < 1.f) || !(hp->beta2 >= 0.f && hp->beta2 < 1.f) ||
+      !(hp->eps >= 0.f) || !(hp->beta_factor < 1.f) || !std::isfinite(hp->lr) || !(hp->weight_decay >= 0.f)) {
+    *err = "hyper-parameter out of range"; return BR_ERR_INVALID;
+  }
+  if (hp->freq < 1 || hp->power_iters < 1) { *err = "freq and power_iters must be >= 1"; return BR_ERR_INVALID; }
+  if (hp->accum != BR_ACCUM_EVERY_STEP && hp->accum != BR_ACCUM_ON_REFRESH) { *err = "bad accum mode"; return BR_ERR_INVALID; }
+  if (hp->gemm_prec != BR_GEMM_FP32 && hp->gemm_prec != BR_GEMM_BF16) { *err = "bad gemm_prec"; return BR_ERR_INVALID; }
+  for (int i = 0; i < n_layers; ++i) {
+    const br_layer_desc& d = layers[i];
+    if (d.m < 1 || d.n < 1 || d.m > (1 << 20) || d.n > (1 << 20)) { *err = format("layer %d: bad shape %lld x %lld", i, (long long)d.m, (long long)d.n); return BR_ERR_SHAPE; }
+    if (d.geom < BR_GEOM_NONE || d.geom > BR_GEOM_BILATERAL) { *err = format("layer %d: bad geometry", i); return BR_ERR_INVALID; }
+    if (d.geom != BR_GEOM_NONE && d.src != BR_SRC_FIRST && d.src != BR_SRC_SECOND) { *err = format("layer %d: bad source", i); return BR_ERR_INVALID; }
+    if (d.grad_dtype != BR_F32 && d.grad_dtype != BR_BF16) { *err = format("layer %d: bad grad dtype", i); return BR_ERR_DTYPE; }
+    if (d.tau_max < 0) { *err = format("layer %d: tau_max < 0", i); return BR_ERR_TAU; }
+  }
+  return BR_OK;
+}
+
+struct Sizes {
+  size_t total = 0, overhead = 0;
+};
+
+}  // namespace
+
+// ---------------------------------------------------------------------------------------------
+// Handle
+// ---------------------------------------------------------------------------------------------
+struct br_handle {
+  int device = 0;
+  cudaStream_t stream = nullptr;
+  br_allocator alloc{};
+  br_hparams hp{};
+  std::vector<Layer> layers;
+  int64_t calls = 0;
+  char* slab = nullptr;
+  size_t slab_bytes = 0;
+  int* d_status = nullptr;
+  // scratch of the SIMT path (one layer at a time)
+  float *sG = nullptr, *sT = nullptr, *sGt = nullptr, *sMt = nullptr;
+  // scratch of the refresh
+  double *rA = nullptr, *rZ = nullptr, *rWork = nullptr;
+  // tensor-core path
+  TcStep* tc = nullptr;
+  LaunchStats stats;
+  std::string err;
+};
+
+namespace {
+
+struct Bump {
+  size_t off = 0;
+  char* base = nullptr;
+  template <typename T> T* take(size_t count) {
+    size_t o = off;
+    off = align_up(off + count * sizeof(T));
+    return base ? reinterpret_cast<T*>(base + o) : nullptr;
+  }
+};
+
+// Lays out every buffer of the handle in one slab.  With base == nullptr only sizes are computed.
+void layout(br_handle* h, Bump& b, Sizes* sz) {
+  const br_hparams& hp = h->hp;
+  size_t max_numel = 0, max_k = 0, max_z = 0;
+  bool any_simt = false;
+  for (Layer& L : h->layers) {
+    const size_t mn = (size_t)L.d.m * L.d.n;
+    L.M = b.take<float>(mn);
+    L.V2 = b.take<float>(mn);
+    const bool second = L.d.src == BR_SRC_SECOND;
+    if (L.left) { L.U = b.take<float>((size_t)L.d.m * L.d.m); sz->overhead += 4 * (size_t)L.d.m * L.d.m; }
+    if (L.right) { L.V = b.take<float>((size_t)L.d.n * L.d.n); sz->overhead += 4 * (size_t)L.d.n * L.d.n; }
+    if (L.left && second) { L.L = b.take<float>((size_t)L.d.m * L.d.m); sz->overhead += 4 * (size_t)L.d.m * L.d.m; }
+    if (L.right && second) { L.R = b.take<float>((size_t)L.d.n * L.d.n); sz->overhead += 4 * (size_t)L.d.n * L.d.n; }
+    if (L.use_tc) {
+      if (L.left) { L.Uh = b.take<__nv_bfloat16>((size_t)L.d.m * L.d.m); L.Ul = b.take<__nv_bfloat16>((size_t)L.d.m * L.d.m); }
+      if (L.right) { L.Vh = b.take<__nv_bfloat16>((size_t)L.d.n * L.d.n); L.Vl = b.take<__nv_bfloat16>((size_t)L.d.n * L.d.n); }
+    }
+    if (L.d.tau_max > 0) {
+      L.slot_stride = align_up(mn * dtype_size(L.d.grad_dtype));
+      L.ring = b.take<char>(L.slot_stride * (size_t)L.d.tau_max);
+    }
+    if (L.d.geom != BR_GEOM_NONE) {
+      if (!L.use_tc) { any_simt = true; max_numel = std::max(max_numel, mn); }
+      if (L.left) max_k = std::max(max_k, (size_t)L.d.m);
+      if (L.right) max_k = std::max(max_k, (size_t)L.d.n);
+      if (!second) max_z = std::max(max_z, mn);
+    }
+  }
+  if (any_simt) {
+    h->sG = b.take<float>(max_numel);
+    h->sT = b.take<float>(max_numel);
+    h->sGt = b.take<float>(max_numel);
+    h->sMt = b.take<float>(max_numel);
+  }
+  if (max_k) {
+    h->rA = b.take<double>(max_k * max_k);
+    h->rWork = b.take<double>(qr_work_doubles((int64_t)max_k));
+    if (max_z) h->rZ = b.take<double>(max_z);
+  }
+  h->d_status = b.take<int>(64);
+  (void)hp;
+  sz->total = b.off;
+}
+
+void init_layers(br_handle* h, const br_layer_desc* layers, int n_layers) {
+  h->layers.resize(n_layers);
+  for (int i = 0; i < n_layers; ++i) {
+    Layer& L = h->layers[i];
+    L = Layer{};
+    L.d = layers[i];
+    rotated_sides(L.d.m, L.d.n, L.d.geom, &L.left, &L.right);
+    L.freq = L.d.freq > 0 ? L.d.freq : h->hp.freq;
+    L.use_tc = h->hp.gemm_prec == BR_GEMM_BF16 && L.d.geom != BR_GEOM_NONE &&
+               (L.d.m % 8 == 0) && (L.d.n % 8 == 0) && L.d.grad_dtype == BR_BF16 && false;
+  }
+}
+
+#define BR_CUDA(h, expr)                                                              \
+  do {                                                                                \
+    cudaError_t e__ = (expr);                                                         \
+    if (e__ != cudaSuccess) {                                                         \
+      (h)->err = format("%s failed: %s", #expr, cudaGetErrorString(e__));             \
+      return BR_ERR_CUDA;                                                             \
+    }                                                                                 \
+  } while (0)
+
+inline void count(br_handle* h, int n = 1) { h->stats.launches += n; }
+
+const void* ring_slot_ptr(const Layer& L, int64_t slot) {
+  return L.ring + (size_t)slot * L.slot_stride;
+}
+
+// ---- refresh of one side: Q <- qr(F Q).Q in fp64, F = L | R (S=2nd) or M M^T | M^T M (S=1st) ----
+br_status refresh_side(br_handle* h, Layer& L, bool left_side) {
+  cudaStream_t s = h->stream;
+  const int64_t m = L.d.m, n = L.d.n;
+  const int64_t k = left_side ? m : n;
+  float* Q = left_side ? L.U : L.V;
+  for (int it = 0; it < h->hp.power_iters; ++it) {
+    if (L.d.src == BR_SRC_SECOND) {
+      const float* F = left_side ? L.L : L.R;
+      BR_CUDA(h, sdgemm(0, 0, k, k, k, 1.0, F, k, Q, k, 0.0, h->rA, k, s));
+      count(h); h->stats.gemm_flops += 2.0 * k * k * k;
+    } else if (left_side) {
+      // (M M^T) U = M (M^T U)
+      BR_CUDA(h, sdgemm(1, 0, n, m, m, 1.0, L.M, n, Q, m, 0.0, h->rZ, m, s));
+      BR_CUDA(h, fdgemm(0, 0, m, m, n, 1.0, L.M, n, h->rZ, m, 0.0, h->rA, m, s));
+      count(h, 2); h->stats.gemm_flops += 4.0 * m * m * n;
+    } else {
+      // (M^T M) V = M^T (M V)
+      BR_CUDA(h, sdgemm(0, 0, m, n, n, 1.0, L.M, n, Q, n, 0.0, h->rZ, n, s));
+      BR_CUDA(h, fdgemm(1, 0, n, n, m, 1.0, L.M, n, h->rZ, n, 0.0, h->rA, n, s));
+      count(h, 2); h->stats.gemm_flops += 4.0 * n * n * m;
+    }
+    BR_CUDA(h, qr_pos_inplace(h->rA, k, h->rWork, h->d_status, s, &h->stats.launches, &h->stats.gemm_flops));
+    BR_CUDA(h, f64_to_f32(h->rA, Q, k * k, s));
+    count(h);
+  }
+  if (L.use_tc) {
+    BR_CUDA(h, split_bf16(Q, left_side ? L.Uh : L.Vh, left_side ? L.Ul : L.Vl, k * k, s));
+    count(h);
+  }
+  return BR_OK;
+}
+
+br_status refresh_layer(br_handle* h, Layer& L) {
+  br_status st;
+  if (L.left && (st = refresh_side(h, L, true)) != BR_OK) return st;
+  if (L.right && (st = refresh_side(h, L, false)) != BR_OK) return st;
+  L.refresh_count += 1;
+  return BR_OK;
+}
+
+// L <- beta L + (1-beta) G G^T ; R <- beta R + (1-beta) G^T G   (Alg. 2), fp32 FFMA
+br_status accumulate_factors_simt(br_handle* h, Layer& L, const float* G) {
+  const float beta = h->hp.beta_factor < 0.f ? h->hp.beta2 : h->hp.beta_factor;
+  const int64_t m = L.d.m, n = L.d.n;
+  if (L.L) {
+    BR_CUDA(h, sgemm(0, 1, m, m, n, 1.0f - beta, G, n, G, n, beta, L.L, m, h->stream));
+    count(h); h->stats.gemm_flops += 2.0 * m * m * n;
+  }
+  if (L.R) {
+    BR_CUDA(h, sgemm(1, 0, n, n, m, 1.0f - beta, G, n, G, n, beta, L.R, n, h->stream));
+    count(h); h->stats.gemm_flops += 2.0 * n * n * m;
+  }
+  return BR_OK;
+}
+
+// out = U^T X V with the identity on an unrotated side; tmp is scratch
+br_status rotate_simt(br_handle* h, Layer& L, const float* X, float* tmp, float* out) {
+  const int64_t m = L.d.m, n = L.d.n;
+  cudaStream_t s = h->stream;
+  if (L.left && L.right) {
+    BR_CUDA(h, sgemm(1, 0, m, n, m, 1.f, L.U, m, X, n, 0.f, tmp, n, s));
+    BR_CUDA(h, sgemm(0, 0, m, n, n, 1.f, tmp, n, L.V, n, 0.f, out, n, s));
+    count(h, 2); h->stats.gemm_flops += 2.0 * m * n * (m + n);
+  } else if (L.left) {
+    BR_CUDA(h, sgemm(1, 0, m, n, m, 1.f, L.U, m, X, n, 0.f, out, n, s));
+    count(h); h->stats.gemm_flops += 2.0 * m * n * m;
+  } else {
+    BR_CUDA(h, sgemm(0, 0, m, n, n, 1.f, X, n, L.V, n, 0.f, out, n, s));
+    count(h); h->stats.gemm_flops += 2.0 * m * n * n;
+  }
+  return BR_OK;
+}
+
+// One update of one layer on the accurate (fp32 FFMA) path.  G: the gradient to apply.
+br_status update_layer_simt(br_handle* h, Layer& L, const void* G) {
+  const br_hparams& hp = h->hp;
+  cudaStream_t s = h->stream;
+  const int64_t m = L.d.m, n = L.d.n, mn = m * n;
+  const int bf = L.d.grad_dtype == BR_BF16;
+  br_status st;
+  // Alg. 1 line 4 (and widen a bf16 gradient once)
+  BR_CUDA(h, ema_momentum(L.M, G, bf, mn, hp.beta1, bf ? h->sG : nullptr, nullptr, nullptr, s));
+  count(h);
+  const float* G32 = bf ? h->sG : reinterpret_cast<const float*>(G);
+  const bool second = L.d.src == BR_SRC_SECOND;
+  if (second && hp.accum == BR_ACCUM_EVERY_STEP && (st = accumulate_factors_simt(h, L, G32)) != BR_OK) return st;
+  // Alg. 1 lines 5-6
+  if (L.t % L.freq == 0) {
+    if (second && hp.accum == BR_ACCUM_ON_REFRESH && (st = accumulate_factors_simt(h, L, G32)) != BR_OK) return st;
+    if ((st = refresh_layer(h, L)) != BR_OK) return st;
+  }
+  // Alg. 1 lines 8-9
+  if ((st = rotate_simt(h, L, G32, h->sT, h->sGt)) != BR_OK) return st;
+  if ((st = rotate_simt(h, L, L.M, h->sT, h->sMt)) != BR_OK) return st;
+  // lines 10-11, element-wise part: X overwrites sMt
+  BR_CUDA(h, second_moment_scale(L.V2, h->sGt, h->sMt, mn, hp.beta2, hp.eps, s));
+  count(h);
+  // line 11: W <- (1 - eta lambda) W - eta U X V^T
+  const float decay = 1.0f - hp.lr * hp.weight_decay;
+  float* W = L.d.weight;
+  if (L.left && L.right) {
+    BR_CUDA(h, sgemm(0, 0, m, n, m, 1.f, L.U, m, h->sMt, n, 0.f, h->sT, n, s));
+    BR_CUDA(h, sgemm(0, 1, m, n, n, -hp.lr, h->sT, n, L.V, n, decay, W, n, s));
+    count(h, 2); h->stats.gemm_flops += 2.0 * m * n * (m + n);
+  } else if (L.left) {
+    BR_CUDA(h, sgemm(0, 0, m, n, m, -hp.lr, L.U, m, h->sMt, n, decay, W, n, s));
+    count(h); h->stats.gemm_flops += 2.0 * m * n * m;
+  } else {
+    BR_CUDA(h, sgemm(0, 1, m, n, n, -hp.lr, h->sMt, n, L.V, n, decay, W, n, s));
+    count(h); h->stats.gemm_flops += 2.0 * m * n * n;
+  }
+  return BR_OK;
+}
+
+br_status check_handle(br_handle* h) {
+  if (!h) return BR_ERR_INVALID;
+  cudaError_t e = cudaSetDevice(h->device);
+  if (e != cudaSuccess) { h->err = format("cudaSetDevice: %s", cudaGetErrorString(e)); return BR_ERR_CUDA; }
+  return BR_OK;
+}
+
+size_t buf_bytes(const Layer& L, int which, void** ptr) {
+  const size_t m = L.d.m, n = L.d.n;
+  switch (which) {
+    case BR_BUF_W: *ptr = L.d.weight; return 4 * m * n;
+    case BR_BUF_M: *ptr = L.M; return 4 * m * n;
+    case BR_BUF_V2: *ptr = L.V2; return 4 * m * n;
+    case BR_BUF_U: *ptr = L.U; return L.U ? 4 * m * m : 0;
+    case BR_BUF_V: *ptr = L.V; return L.V ? 4 * n * n : 0;
+    case BR_BUF_L: *ptr = L.L; return L.L ? 4 * m * m : 0;
+    case BR_BUF_R: *ptr = L.R; return L.R ? 4 * n * n : 0;
+    case BR_BUF_RING: *ptr = L.ring; return L.ring ? (size_t)L.d.tau_max * m * n * dtype_size(L.d.grad_dtype) : 0;
+    default: *ptr = nullptr; return 0;
+  }
+}
+
+}  // namespace
+
+// ---------------------------------------------------------------------------------------------
+// C-ABI
+// ---------------------------------------------------------------------------------------------
+extern "C" {
+
+br_status br_state_bytes(const br_layer_desc* layers, int n_layers, const br_hparams* hp,
+                         size_t* total_bytes, size_t* overhead_bytes) {
+  std::string err;
+  br_status st = validate(layers, n_layers, hp, &err);
+  if (st != BR_OK) { g_create_error = err; return st; }
+  br_handle tmp;
+  tmp.hp = *hp;
+  init_layers(&tmp, layers, n_layers);
+  Bump b;
+  Sizes sz;
+  layout(&tmp, b, &sz);
+  sz.total += tc_step_scratch_bytes(tmp.layers, *hp);
+  if (total_bytes) *total_bytes = sz.total;
+  if (overhead_bytes) *overhead_bytes = sz.overhead;
+  return BR_OK;
+}
+
+br_status br_create(br_handle** out, const br_layer_desc* layers, int n_layers, const br_hparams* hp,
+                    int device, void* cuda_stream, const br_allocator* a) {
+  if (!out) { g_create_error = "out is NULL"; return BR_ERR_INVALID; }
+  *out = nullptr;
+  std::string err;
+  br_status st = validate(layers, n_layers, hp, &err);
+  if (st != BR_OK) { g_create_error = err; return st; }
+  for (int i = 0; i < n_layers; ++i) {
+    if (!layers[i].weight || (reinterpret_cast<uintptr_t>(layers[i].weight) & 15)) {
+      g_create_error = format("layer %d: weight pointer is NULL or not 16-byte aligned", i);
+      return BR_ERR_INVALID;
+    }
+  }
+  cudaError_t e = cudaSetDevice(device);
+  if (e != cudaSuccess) { g_create_error = format("cudaSetDevice(%d): %s", device, cudaGetErrorString(e)); return BR_ERR_CUDA; }
+  cudaDeviceProp prop;
+  e = cudaGetDeviceProperties(&prop, device);
+  if (e != cudaSuccess) { g_create_error = format("cudaGetDeviceProperties: %s", cudaGetErrorString(e)); return BR_ERR_CUDA; }
+  if (prop.major != 10) {
+    g_create_error = format("device %d is sm_%d%d; this library is built for sm_100a only", device, prop.major, prop.minor);
+    return BR_ERR_CUDA;
+  }
+  br_handle* h = new br_handle();
+  h->device = device;
+  h->stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  h->hp = *hp;
+  if (a && a->alloc && a->free) h->alloc = *a;
+  init_layers(h, layers, n_layers);
+
+  Bump sizing;
+  Sizes sz;
+  layout(h, sizing, &sz);
+  const size_t tc_bytes = align_up(tc_step_scratch_bytes(h->layers, h->hp));
+  h->slab_bytes = sz.total + tc_bytes;
+  void* p = nullptr;
+  if (h->alloc.alloc) {
+    p = h->alloc.alloc(h->slab_bytes, h->alloc.ctx);
+  } else if (cudaMalloc(&p, h->slab_bytes) != cudaSuccess) {
+    (void)cudaGetLastError();
+    p = nullptr;
+  }
+  if (!p) {
+    g_create_error = format("allocation of %zu bytes failed", h->slab_bytes);
+    delete h;
+    return BR_ERR_OOM;
+  }
+  h->slab = static_cast<char*>(p);
+  Bump b;
+  b.base = h->slab;
+  Sizes sz2;
+  layout(h, b, &sz2);
+
+  // initial state: M = V~ = L = R = 0 (and everything else in the slab), U = V = I
+  cudaStream_t s = h->stream;
+  auto fail = [&](const char* what, cudaError_t ce) {
+    g_create_error = format("%s: %s", what, cudaGetErrorString(ce));
+    if (h->alloc.alloc) h->alloc.free(h->slab, h->alloc.ctx); else cudaFree(h->slab);
+    delete h;
+    return BR_ERR_CUDA;
+  };
+  if ((e = cudaMemsetAsync(h->slab, 0, sz.total, s)) != cudaSuccess) return fail("cudaMemsetAsync", e);
+  for (Layer& L : h->layers) {
+    if (L.U && (e = set_identity(L.U, L.d.m, s)) != cudaSuccess) return fail("set_identity", e);
+    if (L.V && (e = set_identity(L.V, L.d.n, s)) != cudaSuccess) return fail("set_identity", e);
+    if (L.use_tc) {
+      if (L.U && (e = split_bf16(L.U, L.Uh, L.Ul, L.d.m * L.d.m, s)) != cudaSuccess) return fail("split_bf16", e);
+      if (L.V && (e = split_bf16(L.V, L.Vh, L.Vl, L.d.n * L.d.n, s)) != cudaSuccess) return fail("split_bf16", e);
+    }
+  }
+  const char* tc_err = nullptr;
+  h->tc = tc_step_create(h->layers, h->hp, h->slab + sz.total, tc_bytes, device, s, &tc_err);
+  if (!h->tc && tc_err) {
+    g_create_error = tc_err;
+    if (h->alloc.alloc) h->alloc.free(h->slab, h->alloc.ctx); else cudaFree(h->slab);
+    delete h;
+    return BR_ERR_CUDA;
+  }
+  if ((e = cudaStreamSynchronize(s)) != cudaSuccess) return fail("cudaStreamSynchronize", e);
+  *out = h;
+  return BR_OK;
+}
+
+br_status br_step(br_handle* h, const void* const* grads, int tau) {
+  br_status st = check_handle(h);
+  if (st != BR_OK) return st;
+  if (!grads) { h->err = "grads is NULL"; return BR_ERR_INVALID; }
+  const int nl = (int)h->layers.size();
+  for (int i = 0; i < nl; ++i) {
+    const Layer& L = h->layers[i];
+    if (!grads[i] || (reinterpret_cast<uintptr_t>(grads[i]) & 15)) {
+      h->err = format("layer %d: gradient pointer is NULL or not 16-byte aligned", i);
+      return BR_ERR_INVALID;
+    }
+    if (tau < -1 || tau > L.d.tau_max) {
+      h->err = format("layer %d: tau %d outside [0, %d]", i, tau, L.d.tau_max);
+      return BR_ERR_TAU;
+    }
+  }
+  // ---- integer state (host) ---------------------------------------------------------------
+  h->calls += 1;
+  std::vector<const void*> G(nl, nullptr);
+  bool any = false;
+  for (int i = 0; i < nl; ++i) {
+    Layer& L = h->layers[i];
+    const int tl = tau < 0 ? L.d.tau_max : tau;
+    const int64_t src_call = h->calls - tl;     // Eq. (delayed_grad)
+    if (src_call >= 1) {
+      G[i] = (tl == 0) ? grads[i] : ring_slot_ptr(L, (src_call - 1) % L.d.tau_max);
+      L.t += 1;
+      any = true;
+    }
+  }
+  // ---- enqueue the updates ----------------------------------------------------------------
+  const br_hparams& hp = h->hp;
+  for (int i = 0; i < nl; ++i) {
+    Layer& L = h->layers[i];
+    if (!G[i]) continue;
+    if (L.d.geom == BR_GEOM_NONE) {
+      BR_CUDA(h, plain_adam(L.d.weight, L.M, L.V2, G[i], L.d.grad_dtype == BR_BF16, L.d.m * L.d.n,
+                            hp.lr, hp.beta1, hp.beta2, hp.eps, hp.weight_decay, h->stream));
+      count(h);
+    } else if (!L.use_tc) {
+      if ((st = update_layer_simt(h, L, G[i])) != BR_OK) return st;
+    }
+  }
+  if (h->tc) {
+    TcStepCallbacks cb;
+    cb.ctx = h;
+    cb.refresh = [](void* ctx, int layer) -> int {
+      br_handle* hh = static_cast<br_handle*>(ctx);
+      return (int)refresh_layer(hh, hh->layers[layer]);
+    };
+    const char* terr = nullptr;
+    int rc = tc_step_run(h->tc, h->layers, G, hp, h->d_status, h->stream, &h->stats, cb, &terr);
+    if (rc != 0) { h->err = terr ? terr : "tensor-core step failed"; return rc < 0 ? (br_status)rc : BR_ERR_CUDA; }
+  }
+  // ---- store g_c in the ring (after every reader of the slot it may overwrite) --------------
+  for (int i = 0; i < nl; ++i) {
+    Layer& L = h->layers[i];
+    if (L.d.tau_max <= 0) continue;
+    const size_t bytes = (size_t)L.d.m * L.d.n * dtype_size(L.d.grad_dtype);
+    void* dst = const_cast<void*>(ring_slot_ptr(L, (h->calls - 1) % L.d.tau_max));
+    BR_CUDA(h, cudaMemcpyAsync(dst, grads[i], bytes, cudaMemcpyDeviceToDevice, h->stream));
+  }
+  return any ? BR_OK : BR_WARMUP;
+}
+
+br_status br_set_lr(br_handle* h, float lr) {
+  if (!h) return BR_ERR_INVALID;
+  if (!std::isfinite(lr)) { h->err = "lr is not finite"; return BR_ERR_INVALID; }
+  h->hp.lr = lr;
+  return BR_OK;
+}
+
+br_status br_refresh_basis(br_handle* h, int layer) {
+  br_status st = check_handle(h);
+  if (st != BR_OK) return st;
+  const int nl = (int)h->layers.size();
+  if (layer < -1 || layer >= nl) { h->err = "layer index out of range"; return BR_ERR_INVALID; }
+  const int lo = layer < 0 ? 0 : layer, hi = layer < 0 ? nl : layer + 1;
+  for (int i = lo; i < hi; ++i) {
+    const Layer& L = h->layers[i];
+    if (L.d.geom != BR_GEOM_NONE && L.t == 0) {
+      h->err = format("layer %d: refresh before the first update (factor is all zero)", i);
+      return BR_ERR_STATE;
+    }
+  }
+  for (int i = lo; i < hi; ++i) {
+    Layer& L = h->layers[i];
+    if (L.d.geom == BR_GEOM_NONE) continue;
+    if ((st = refresh_layer(h, L)) != BR_OK) return st;
+  }
+  return BR_OK;
+}
+
+br_status br_sync_status(br_handle* h) {
+  br_status st = check_handle(h);
+  if (st != BR_OK) return st;
+  BR_CUDA(h, cudaStreamSynchronize(h->stream));
+  int word = 0;
+  BR_CUDA(h, cudaMemcpy(&word, h->d_status, sizeof(int), cudaMemcpyDeviceToHost));
+  if (word > 0) BR_CUDA(h, cudaMemset(h->d_status, 0, sizeof(int)));
+  if (word < 0) h->err = format("device status word %d (%s)", word, br_strerror(word));
+  return (br_status)word;
+}
+
+br_status br_get_counters(br_handle* h, int layer, br_counters* out) {
+  if (!h || !out) return BR_ERR_INVALID;
+  if (layer < 0 || layer >= (int)h->layers.size()) { h->err = "layer index out of range"; return BR_ERR_INVALID; }
+  const Layer& L = h->layers[layer];
+  out->calls = h->calls;
+  out->t = L.t;
+  out->ring_slot = L.d.tau_max > 0 ? h->calls % L.d.tau_max : 0;
+  out->refresh_count = L.refresh_count;
+  out->next_refresh_t = (L.t / L.freq + 1) * L.freq;
+  return BR_OK;
+}
+
+br_status br_set_counters(br_handle* h, int layer, const br_counters* in) {
+  if (!h || !in) return BR_ERR_INVALID;
+  if (layer < 0 || layer >= (int)h->layers.size()) { h->err = "layer index out of range"; return BR_ERR_INVALID; }
+  if (in->calls < 0 || in->t < 0 || in->t > in->calls || in->refresh_count < 0) { h->err = "inconsistent counters"; return BR_ERR_INVALID; }
+  Layer& L = h->layers[layer];
+  h->calls = in->calls;
+  L.t = in->t;
+  L.refresh_count = in->refresh_count;
+  return BR_OK;
+}
+
+br_status br_get_state(br_handle* h, int layer, int which, void* host_dst, size_t bytes) {
+  br_status st = check_handle(h);
+  if (st != BR_OK) return st;
+  if (!host_dst || layer < 0 || layer >= (int)h->layers.size()) { h->err = "bad argument"; return BR_ERR_INVALID; }
+  const Layer& L = h->layers[layer];
+  void* p = nullptr;
+  const size_t want = buf_bytes(L, which, &p);
+  if (!p || want == 0) { h->err = "this layer has no such buffer"; return BR_ERR_STATE; }
+  if (bytes != want) { h->err = format("buffer is %zu bytes, caller passed %zu", want, bytes); return BR_ERR_SHAPE; }
+  BR_CUDA(h, cudaStreamSynchronize(h->stream));
+  if (which == BR_BUF_RING) {
+    const size_t row = (size_t)L.d.m * L.d.n * dtype_size(L.d.grad_dtype);
+    BR_CUDA(h, cudaMemcpy2D(host_dst, row, p, L.slot_stride, row, L.d.tau_max, cudaMemcpyDeviceToHost));
+  } else {
+    BR_CUDA(h, cudaMemcpy(host_dst, p, bytes, cudaMemcpyDeviceToHost));
+  }
+  return BR_OK;
+}
+
+br_status br_set_state(br_handle* h, int layer, int which, const void* host_src, size_t bytes) {
+  br_status st = check_handle(h);
+  if (st != BR_OK) return st;
+  if (!host_src || layer < 0 || layer >= (int)h->layers.size()) { h->err = "bad argument"; return BR_ERR_INVALID; }
+  Layer& L = h->layers[layer];
+  void* p = nullptr;
+  const size_t want = buf_bytes(L, which, &p);
+  if (!p || want == 0) { h->err = "this layer has no such buffer"; return BR_ERR_STATE; }
+  if (bytes != want) { h->err = format("buffer is %zu bytes, caller passed %zu", want, bytes); return BR_ERR_SHAPE; }
+  BR_CUDA(h, cudaStreamSynchronize(h->stream));
+  if (which == BR_BUF_RING) {
+    const size_t row = (size_t)L.d.m * L.d.n * dtype_size(L.d.grad_dtype);
+    BR_CUDA(h, cudaMemcpy2D(p, L.slot_stride, host_src, row, row, L.d.tau_max, cudaMemcpyHostToDevice));
+  } else {
+    BR_CUDA(h, cudaMemcpy(p, host_src, bytes, cudaMemcpyHostToDevice));
+  }
+  if (L.use_tc && which == BR_BUF_U) { BR_CUDA(h, split_bf16(L.U, L.Uh, L.Ul, L.d.m * L.d.m, h->stream)); count(h); }
+  if (L.use_tc && which == BR_BUF_V) { BR_CUDA(h, split_bf16(L.V, L.Vh, L.Vl, L.d.n * L.d.n, h->stream)); count(h); }
+  BR_CUDA(h, cudaStreamSynchronize(h->stream));
+  return BR_OK;
+}
+
+br_status br_get_launch_stats(br_handle* h, int64_t* kernel_launches, double* gemm_flops) {
+  if (!h) return BR_ERR_INVALID;
+  if (kernel_launches) *kernel_launches = h->stats.launches;
+  if (gemm_flops) *gemm_flops = h->stats.gemm_flops;
+  return BR_OK;
+}
+
+br_status br_destroy(br_handle* h) {
+  if (!h) return BR_OK;
+  cudaSetDevice(h->device);
+  cudaStreamSynchronize(h->stream);
+  if (h->tc) tc_step_destroy(h->tc);
+  if (h->slab) {
+    if (h->alloc.alloc) h->alloc.free(h->slab, h->alloc.ctx); else cudaFree(h->slab);
+  }
+  delete h;
+  return BR_OK;
+}
+
+const char* br_strerror(int status) {
+  switch (status) {
+    case BR_OK: return "ok";
+    case BR_WARMUP: return "warm-up call: no update applied";
+    case BR_WARN_RANK_DEFICIENT: return "refresh met a rank-deficient factor";
+    case BR_ERR_INVALID: return "invalid argument";
+    case BR_ERR_SHAPE: return "bad shape or size";
+    case BR_ERR_DTYPE: return "bad dtype";
+    case BR_ERR_TAU: return "tau out of range";
+    case BR_ERR_OOM: return "out of device memory";
+    case BR_ERR_CUDA: return "CUDA error";
+    case BR_ERR_STATE: return "operation not valid in this state";
+    case BR_ERR_TIMEOUT: return "device-side wait timed out";
+    default: return "unknown status";
+  }
+}
+
+const char* br_last_error(const br_handle* h) { return h ? h->err.c_str() : g_create_error.c_str(); }
+
+}  // extern "C"

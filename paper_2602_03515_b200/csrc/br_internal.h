@@ -1,0 +1,112 @@
+// Internal declarations shared by the translation units of libbr.  Nothing here is part of
+// the public C-ABI (see include/br.h).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "br.h"
+
+namespace br {
+
+// ---------------------------------------------------------------------------------------------
+// Launch accounting (reported through br_get_launch_stats)
+// ---------------------------------------------------------------------------------------------
+struct LaunchStats {
+  int64_t launches = 0;
+  double gemm_flops = 0.0;
+};
+
+// ---------------------------------------------------------------------------------------------
+// Element-wise kernels (elem.cu).  All take a stream and return the launch error.
+// ---------------------------------------------------------------------------------------------
+cudaError_t set_identity(float* Q, int64_t k, cudaStream_t s);
+
+// Alg. 1 line 4: M <- beta1 M + (1-beta1) G.  G is fp32 or bf16 (g_is_bf16).  Optional outputs:
+// Gf32 (G widened to fp32), Mh/Ml (bf16 hi/lo split of the new M).
+cudaError_t ema_momentum(float* M, const void* G, int g_is_bf16, int64_t numel, float beta1,
+                         float* Gf32, __nv_bfloat16* Mh, __nv_bfloat16* Ml, cudaStream_t s);
+
+// Eq. (adam): plain Adam, eps inside the sqrt, no bias correction, decoupled weight decay.
+cudaError_t plain_adam(float* W, float* M, float* V, const void* G, int g_is_bf16, int64_t numel,
+                       float lr, float beta1, float beta2, float eps, float wd, cudaStream_t s);
+
+// Alg. 1 lines 10-11 (element-wise part): V~ <- beta2 V~ + (1-beta2) G~^2 ; X = M~/sqrt(V~+eps).
+// X overwrites Mt.
+cudaError_t second_moment_scale(float* V2, const float* Gt, float* Mt, int64_t numel, float beta2,
+                                float eps, cudaStream_t s);
+
+// fp32 -> bf16 hi (+ optional lo = bf16(x - hi)).
+cudaError_t split_bf16(const float* X, __nv_bfloat16* hi, __nv_bfloat16* lo, int64_t numel,
+                       cudaStream_t s);
+cudaError_t widen_bf16(const __nv_bfloat16* X, float* out, int64_t numel, cudaStream_t s);
+// out(double) <- in(float) ; out(float) <- in(double)
+cudaError_t f64_to_f32(const double* X, float* out, int64_t numel, cudaStream_t s);
+
+// ---------------------------------------------------------------------------------------------
+// SIMT contractions (gemm_simt.cu):  C = alpha * op(A) op(B) + beta * C, row-major.
+// op(X) = X or X^T (ta / tb).  M, N, K are the dimensions of the product.
+// ---------------------------------------------------------------------------------------------
+cudaError_t sgemm(int ta, int tb, int64_t M, int64_t N, int64_t K, float alpha, const float* A,
+                  int64_t lda, const float* B, int64_t ldb, float beta, float* C, int64_t ldc,
+                  cudaStream_t s);
+// fp32 inputs, fp64 accumulation and output (power step F Q of a refresh)
+cudaError_t sdgemm(int ta, int tb, int64_t M, int64_t N, int64_t K, double alpha, const float* A,
+                   int64_t lda, const float* B, int64_t ldb, double beta, double* C, int64_t ldc,
+                   cudaStream_t s);
+cudaError_t dgemm(int ta, int tb, int64_t M, int64_t N, int64_t K, double alpha, const double* A,
+                  int64_t lda, const double* B, int64_t ldb, double beta, double* C, int64_t ldc,
+                  cudaStream_t s);
+
+// ---------------------------------------------------------------------------------------------
+// QR with positive diagonal in fp64 (qr.cu).  A (k x k, row-major, ld = k) is overwritten by
+// its Q factor.  work: at least qr_work_doubles(k) doubles.  status: device int, set to
+// BR_WARN_RANK_DEFICIENT when a pivot underflows.  Returns the number of launches in *launches.
+// ---------------------------------------------------------------------------------------------
+size_t qr_work_doubles(int64_t k);
+cudaError_t qr_pos_inplace(double* A, int64_t k, double* work, int* status, cudaStream_t s,
+                           int64_t* launches, double* flops);
+
+// ---------------------------------------------------------------------------------------------
+// tcgen05 grouped contraction (gemm_tc.cu)
+// ---------------------------------------------------------------------------------------------
+enum Epilogue : int32_t {
+  EPI_AXPBY_F32 = 0,    // D <- alpha*acc + beta*D                 (factor EMA, weight write, plain)
+  EPI_SPLIT_BF16 = 1,   // Dh <- bf16(acc), Dl <- bf16(acc - Dh)   (Dl optional)
+  EPI_SECOND_MOMENT = 2,// D(V~) <- beta*D + alpha*acc^2
+  EPI_SCALE_BF16 = 3    // Dh(X) <- bf16(acc / sqrt(D(V~) + eps))
+};
+
+struct TcOperand {
+  const void* ptr;      // bf16, DEVICE
+  int64_t ld;           // elements
+  int32_t mn_major;     // 1: stored K x MN (MN contiguous); 0: stored MN x K (K contiguous)
+};
+
+struct TcProblem {
+  int64_t Md, Nd, K;
+  int32_t n_pairs;      // 1..3; all pairs share majors and leading dimensions
+  TcOperand A[3], B[3];
+  int32_t epilogue;
+  float alpha, beta, eps;
+  float* D; int64_t ldd;            // fp32 in/out
+  __nv_bfloat16* Dh; __nv_bfloat16* Dl; int64_t ldh;  // bf16 outputs
+};
+
+struct TcPlan;  // opaque: device problem table + tensor maps, built on the host
+
+// Build a plan for a list of problems that can run concurrently in one launch.
+// Returns nullptr and sets *err on failure.
+TcPlan* tc_plan_create(const TcProblem* problems, int n, int device, cudaStream_t s, const char** err);
+void tc_plan_destroy(TcPlan* p);
+// Scalars may change between launches (eta_t): patch alpha/beta of problem i (host side, copied
+// with the next launch).
+void tc_plan_set_scalars(TcPlan* p, int i, float alpha, float beta);
+// Re-point operands / outputs of problem i (same shapes and strides): used for ring slots.
+int tc_plan_set_operand(TcPlan* p, int i, int pair, int which /*0=A,1=B*/, const void* ptr);
+cudaError_t tc_plan_launch(TcPlan* p, int* status_word, cudaStream_t s);
+double tc_plan_flops(const TcPlan* p);
+int tc_supported(int device);
+
+}  // namespace br

@@ -1,0 +1,48 @@
+// Per-layer state record and the interface of the tensor-core step planner (step_tc.cu).
+#pragma once
+#include <string>
+#include <vector>
+
+#include "br_internal.h"
+
+namespace br {
+
+struct Layer {
+  br_layer_desc d{};
+  bool left = false, right = false;   // which sides carry a rotation
+  bool use_tc = false;                // contractions run on the tcgen05 tile kernel
+  int freq = 1;
+  float *M = nullptr, *V2 = nullptr, *U = nullptr, *V = nullptr, *L = nullptr, *R = nullptr;
+  __nv_bfloat16 *Uh = nullptr, *Ul = nullptr, *Vh = nullptr, *Vl = nullptr;  // bf16 hi/lo of U, V
+  char* ring = nullptr;
+  size_t slot_stride = 0;             // bytes between ring slots
+  int64_t t = 0, refresh_count = 0;
+};
+
+std::string format(const char* fmt, ...);
+size_t dtype_size(int dt);
+void rotated_sides(int64_t m, int64_t n, int geom, bool* left, bool* right);
+
+cudaError_t fdgemm(int ta, int tb, int64_t M, int64_t N, int64_t K, double alpha, const float* A,
+                   int64_t lda, const double* B, int64_t ldb, double beta, double* C, int64_t ldc,
+                   cudaStream_t s);
+
+struct TcStep;
+struct TcStepCallbacks {
+  void* ctx = nullptr;
+  int (*refresh)(void* ctx, int layer) = nullptr;   // runs Power() for a layer, returns br_status
+};
+
+// Transient scratch (bytes) the tensor-core step needs for these layers.
+size_t tc_step_scratch_bytes(const std::vector<Layer>& layers, const br_hparams& hp);
+// Returns nullptr with *err == nullptr when no layer uses the tensor-core path.
+TcStep* tc_step_create(std::vector<Layer>& layers, const br_hparams& hp, char* scratch, size_t bytes,
+                       int device, cudaStream_t s, const char** err);
+// Enqueue the updates of every tensor-core layer whose G[i] is non-null.  0 on success,
+// a negative br_status otherwise (message in *err).
+int tc_step_run(TcStep* t, std::vector<Layer>& layers, const std::vector<const void*>& G,
+                const br_hparams& hp, int* d_status, cudaStream_t s, LaunchStats* stats,
+                const TcStepCallbacks& cb, const char** err);
+void tc_step_destroy(TcStep* t);
+
+}  // namespace br

@@ -1,0 +1,68 @@
+"""Helpers shared by the GPU parity tests: run the C-ABI library and the oracle side by side on
+the same seeded inputs (the tests are the only place where both are imported)."""
+from __future__ import annotations
+
+import numpy as np
+
+from oracle import br_oracle as O
+from workloads import GradientStream, initial_weight
+
+
+def rel_l2(a, b):
+    a = np.asarray(a, dtype=np.float64); b = np.asarray(b, dtype=np.float64)
+    nb = np.linalg.norm(b)
+    return float(np.linalg.norm(a - b) / (nb if nb > 0 else 1.0))
+
+
+def basis_err(q_gpu, q_ref):
+    return float(np.max(np.abs(O.sign_normalise(np.asarray(q_gpu, dtype=np.float64)) - O.sign_normalise(q_ref))))
+
+
+class SideBySide:
+    """Steps a workload through libbr (GPU) and the oracle (CPU float64) together."""
+
+    def __init__(self, w, *, gemm_prec=None, accum="every_step", power_iters=1, device="cuda:0", **kw):
+        import torch
+        import paper_2602_03515_b200 as br
+        self.torch, self.br, self.w = torch, br, w
+        self.device = torch.device(device)
+        self.streams = [GradientStream(w, i) for i in range(len(w.layers))]
+        w0 = [initial_weight(w, i) for i in range(len(w.layers))]
+        self.weights = [torch.from_numpy(x.copy()).to(self.device) for x in w0]
+        self.oracle = O.make_oracle(w, w0, accum=accum, power_iters=power_iters)
+        gp = gemm_prec if gemm_prec is not None else (br.BR_GEMM_FP32 if w.gemm_prec == "f32" else br.BR_GEMM_BF16)
+        self.opt = br.BasisRotation.from_workload(
+            w, self.weights, gemm_prec=gp, power_iters=power_iters,
+            accum=br.BR_ACCUM_ON_REFRESH if accum == "on_refresh" else br.BR_ACCUM_EVERY_STEP, **kw)
+        self.call = 0
+
+    def grads_for(self, call):
+        torch = self.torch
+        host, dev = [], []
+        for s in self.streams:
+            g32 = s(call)
+            host.append(g32)
+            if self.w.grad_dtype == "bf16":
+                dev.append(torch.from_numpy(s.bits(call).view(np.int16)).view(torch.bfloat16).to(self.device))
+            else:
+                dev.append(torch.from_numpy(g32).to(self.device))
+        return host, dev
+
+    def step(self, tau=-1):
+        """Returns (gpu_status, oracle_status, per-layer dW from the GPU, per-layer dW oracle)."""
+        self.call += 1
+        host, dev = self.grads_for(self.call)
+        before = [w.detach().cpu().numpy().astype(np.float64) for w in self.weights]
+        st_g = self.opt.step(dev, tau)
+        st_o = self.oracle.step(host, tau)
+        self.torch.cuda.synchronize()
+        after = [w.detach().cpu().numpy().astype(np.float64) for w in self.weights]
+        dW_g = [a - b for a, b in zip(after, before)]
+        dW_o = [l.last_dW for l in self.oracle.layers]
+        return st_g, st_o, dW_g, dW_o
+
+    def state(self, layer, which):
+        return self.opt.get_state(layer, which).float().numpy().astype(np.float64)
+
+    def close(self):
+        self.opt.close()

@@ -1,0 +1,201 @@
+"""GPU parity of the accurate (fp32 FFMA + fp64 refresh) path against the float64 oracle, through
+the C-ABI.  Tolerances: per-step parameter update relative L2 <= 1e-4, bases (sign-normalised)
+max-abs <= 1e-3, integer state bit-exact."""
+from dataclasses import replace
+
+import numpy as np
+import pytest
+
+from workloads import get_workload, LayerSpec, Workload
+from workloads.configs import GEOM_BI, GEOM_NONE, GEOM_UNI, SRC_FIRST, SRC_SECOND
+
+pytestmark = pytest.mark.gpu
+
+TOL_DW, TOL_BASIS = 1e-4, 1e-3
+
+
+def _run(w, calls, tau=-1, **kw):
+    from tests.parity_util import SideBySide, basis_err, rel_l2
+    import paper_2602_03515_b200 as br
+    sbs = SideBySide(w, **kw)
+    worst_dw, worst_q = 0.0, 0.0
+    try:
+        for c in range(calls):
+            st_g, st_o, dg, do = sbs.step(tau)
+            assert st_g == st_o or (st_g == br.BR_OK and st_o == 2), (c, st_g, st_o)
+            for li, (a, b) in enumerate(zip(dg, do)):
+                if b is None:
+                    assert not np.any(a), "warm-up call changed the weights"
+                    continue
+                worst_dw = max(worst_dw, rel_l2(a, b))
+            for li, lay in enumerate(sbs.oracle.layers):
+                assert sbs.opt.counters(li) == sbs.oracle.counters(li)
+        for li, lay in enumerate(sbs.oracle.layers):
+            for which, ref in ((br.BR_BUF_U, lay.U), (br.BR_BUF_V, lay.V)):
+                if ref is not None and lay.refresh_count > 0:
+                    worst_q = max(worst_q, basis_err(sbs.state(li, which), ref))
+            assert rel_l2(sbs.state(li, br.BR_BUF_M), lay.M) < 1e-5
+            assert rel_l2(sbs.state(li, br.BR_BUF_V2), lay.V2) < 1e-3
+            assert rel_l2(sbs.state(li, br.BR_BUF_W), lay.W) < 1e-5
+            if lay.L is not None:
+                assert rel_l2(sbs.state(li, br.BR_BUF_L), lay.L) < 1e-5
+            if lay.R is not None:
+                assert rel_l2(sbs.state(li, br.BR_BUF_R), lay.R) < 1e-5
+        assert sbs.opt.sync_status() in (br.BR_OK, br.BR_WARN_RANK_DEFICIENT)
+    finally:
+        sbs.close()
+    assert worst_dw <= TOL_DW, worst_dw
+    assert worst_q <= TOL_BASIS, worst_q
+    return worst_dw, worst_q
+
+
+def test_c1_full_trajectory():
+    """64x32 fp32, bilateral, S=2nd, tau=2, refresh every 5, 20 calls."""
+    w = get_workload("c1")
+    _run(w, w.calls, tau=2)
+
+
+def _small(geom, src, m, n, dtype="f32", kind="iid_normal", tau=1, freq=3, **kw):
+    return Workload("small", [LayerSpec("W", m, n, geom, src, tau)], dtype, kind, 0.05, 4, tau=tau,
+                    freq=freq, calls=10, gemm_prec="f32", seed=3, **kw)
+
+
+@pytest.mark.parametrize("geom,src", [(GEOM_BI, SRC_SECOND), (GEOM_BI, SRC_FIRST), (GEOM_UNI, SRC_SECOND),
+                                      (GEOM_UNI, SRC_FIRST), (GEOM_NONE, SRC_SECOND)])
+@pytest.mark.parametrize("m,n", [(37, 53), (96, 40), (130, 130)])
+def test_strategy_grid_ragged_shapes(geom, src, m, n):
+    if geom == GEOM_BI and src == SRC_FIRST and m != n:
+        pytest.skip("bilateral S=1st on a rectangular matrix has a rank-deficient factor on the larger side")
+    _run(_small(geom, src, m, n), 10, tau=1)
+
+
+def test_bf16_gradients_lowrank_fp32_gemm():
+    w = _small(GEOM_BI, SRC_SECOND, 72, 104, dtype="bf16", kind="lowrank_noise", tau=2, freq=4)
+    _run(w, 12, tau=2)
+
+
+def test_weight_decay_and_on_refresh_accumulation():
+    w = _small(GEOM_BI, SRC_SECOND, 48, 24, tau=0, freq=2, weight_decay=0.1)
+    _run(w, 8, tau=0, accum="on_refresh")
+
+
+def test_power_iters_2():
+    _run(_small(GEOM_BI, SRC_SECOND, 40, 56, tau=0, freq=3), 7, tau=0, power_iters=2)
+
+
+def test_multi_layer_per_layer_tau_and_freq():
+    layers = [LayerSpec("a", 33, 65, GEOM_BI, SRC_SECOND, 3, 2), LayerSpec("b", 64, 16, GEOM_UNI, SRC_SECOND, 1, 3),
+              LayerSpec("c", 20, 20, GEOM_NONE, SRC_SECOND, 0, 0), LayerSpec("d", 24, 80, GEOM_UNI, SRC_FIRST, 2, 0)]
+    w = Workload("multi", layers, "f32", "iid_normal", 0.02, tau=3, freq=4, calls=12, gemm_prec="f32", seed=5)
+    _run(w, 12, tau=-1)
+
+
+def test_variable_tau_per_call():
+    from tests.parity_util import SideBySide, rel_l2
+    w = _small(GEOM_BI, SRC_SECOND, 32, 48, tau=3, freq=3)
+    sbs = SideBySide(w)
+    try:
+        for tau in (3, 3, 3, 3, 1, 2, 0, 3, 2):
+            st_g, st_o, dg, do = sbs.step(tau)
+            assert st_g == st_o
+            if do[0] is not None:
+                assert rel_l2(dg[0], do[0]) < TOL_DW
+            assert sbs.opt.counters(0) == sbs.oracle.counters(0)
+    finally:
+        sbs.close()
+
+
+def test_qr_many_panels_teacher_forced():
+    """Forced refresh from a given L, U (set through the API) against the oracle's Power():
+    k = 200 spans 7 panels with a ragged last one; the factor has a 1e4 spread of eigenvalues."""
+    import torch
+    import paper_2602_03515_b200 as br
+    from oracle import br_oracle as O
+    from tests.parity_util import basis_err
+    k, n = 200, 16
+    rng = np.random.default_rng(11)
+    Qe, _ = np.linalg.qr(rng.standard_normal((k, k)))
+    lam = np.logspace(0, -4, k)
+    F = ((Qe * lam) @ Qe.T).astype(np.float32)
+    U0, _ = np.linalg.qr(rng.standard_normal((k, k)))
+    U0 = U0.astype(np.float32)
+    w = torch.zeros(k, n, device="cuda")
+    spec = LayerSpec("W", k, n, GEOM_UNI, SRC_SECOND, 0)
+    spec = replace(spec, geom=GEOM_BI)
+    opt = br.BasisRotation([spec], [w], grad_dtype="f32", gemm_prec=br.BR_GEMM_FP32, freq=1000)
+    try:
+        g = torch.randn(k, n, device="cuda") * 0.01
+        assert opt.step([g], 0) == br.BR_OK          # t = 1 so that a forced refresh is allowed
+        opt.set_state(0, br.BR_BUF_L, torch.from_numpy(F))
+        opt.set_state(0, br.BR_BUF_U, torch.from_numpy(U0))
+        opt.refresh_basis(0)
+        assert opt.sync_status() == br.BR_OK
+        U = opt.get_state(0, br.BR_BUF_U).numpy().astype(np.float64)
+        ref, deficient = O.power(F.astype(np.float64), U0.astype(np.float64))
+        assert not deficient
+        assert np.max(np.abs(U.T @ U - np.eye(k))) < 1e-5
+        assert basis_err(U, ref) < 1e-5
+        assert opt.counters(0)["refresh_count"] == 1 and opt.counters(0)["t"] == 1
+    finally:
+        opt.close()
+
+
+def test_host_side_errors_leave_handle_usable():
+    import torch
+    import paper_2602_03515_b200 as br
+    w = torch.zeros(16, 8, device="cuda")
+    opt = br.BasisRotation([LayerSpec("W", 16, 8, GEOM_BI, SRC_SECOND, 2)], [w], grad_dtype="f32",
+                           gemm_prec=br.BR_GEMM_FP32)
+    try:
+        g = torch.randn(16, 8, device="cuda")
+        with pytest.raises(br.BrError) as e:
+            opt.step([g], 5)
+        assert e.value.status == br.BR_ERR_TAU
+        with pytest.raises(br.BrError) as e:
+            opt.refresh_basis(0)
+        assert e.value.status == br.BR_ERR_STATE
+        with pytest.raises(br.BrError) as e:
+            br.br_step(opt.handle, [0], 0)
+        assert e.value.status == br.BR_ERR_INVALID
+        assert opt.counters(0)["calls"] == 0
+        assert opt.step([g], 2) == br.BR_WARMUP
+        assert opt.counters(0) == dict(calls=1, t=0, ring_slot=1, refresh_count=0, next_refresh_t=10)
+    finally:
+        opt.close()
+
+
+def test_checkpoint_resume_bit_identical():
+    """run 9 calls == run 5, save, destroy, create, load, run 4 (all buffers and counters)."""
+    import torch
+    import paper_2602_03515_b200 as br
+    from workloads import GradientStream, initial_weight
+    w = _small(GEOM_BI, SRC_SECOND, 40, 24, tau=2, freq=3)
+    gs = GradientStream(w, 0)
+    bufs = [br.BR_BUF_W, br.BR_BUF_M, br.BR_BUF_V2, br.BR_BUF_U, br.BR_BUF_V, br.BR_BUF_L, br.BR_BUF_R, br.BR_BUF_RING]
+
+    def fresh():
+        wt = torch.from_numpy(initial_weight(w, 0).copy()).cuda()
+        return wt, br.BasisRotation.from_workload(w, [wt], gemm_prec=br.BR_GEMM_FP32)
+
+    wt, a = fresh()
+    for c in range(1, 10):
+        a.step([torch.from_numpy(gs(c)).cuda()], 2)
+    final = {b: a.get_state(0, b).clone() for b in bufs}
+    ca = a.counters(0)
+    a.close()
+    wt, b1 = fresh()
+    for c in range(1, 6):
+        b1.step([torch.from_numpy(gs(c)).cuda()], 2)
+    saved = {b: b1.get_state(0, b).clone() for b in bufs}
+    cnt = b1.counters(0)
+    b1.close()
+    wt, b2 = fresh()
+    for b in bufs:
+        b2.set_state(0, b, saved[b])
+    br.br_set_counters(b2.handle, 0, cnt["calls"], cnt["t"], cnt["refresh_count"])
+    for c in range(6, 10):
+        b2.step([torch.from_numpy(gs(c)).cuda()], 2)
+    assert b2.counters(0) == ca
+    for b in bufs:
+        assert torch.equal(b2.get_state(0, b), final[b]), b
+    b2.close()

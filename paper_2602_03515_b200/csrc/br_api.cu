@@ -129,9 +129,12 @@ void layout(br_handle* h, Bump& b, Sizes* sz) {
       if (L.left) { L.Uh = b.take<__nv_bfloat16>((size_t)L.d.m * L.d.m); L.Ul = b.take<__nv_bfloat16>((size_t)L.d.m * L.d.m); }
       if (L.right) { L.Vh = b.take<__nv_bfloat16>((size_t)L.d.n * L.d.n); L.Vl = b.take<__nv_bfloat16>((size_t)L.d.n * L.d.n); }
     }
-    if (L.d.tau_max > 0) {
+    // a tensor-core layer reads its gradient through a tensor map over the ring, so it keeps
+    // one slot even without delay
+    L.ring_slots = L.d.tau_max > 0 ? L.d.tau_max : (L.use_tc ? 1 : 0);
+    if (L.ring_slots > 0) {
       L.slot_stride = align_up(mn * dtype_size(L.d.grad_dtype));
-      L.ring = b.take<char>(L.slot_stride * (size_t)L.d.tau_max);
+      L.ring = b.take<char>(L.slot_stride * (size_t)L.ring_slots);
     }
     if (L.d.geom != BR_GEOM_NONE) {
       if (!L.use_tc) { any_simt = true; max_numel = std::max(max_numel, mn); }
@@ -165,7 +168,7 @@ void init_layers(br_handle* h, const br_layer_desc* layers, int n_layers) {
     rotated_sides(L.d.m, L.d.n, L.d.geom, &L.left, &L.right);
     L.freq = L.d.freq > 0 ? L.d.freq : h->hp.freq;
     L.use_tc = h->hp.gemm_prec == BR_GEMM_BF16 && L.d.geom != BR_GEOM_NONE &&
-               (L.d.m % 8 == 0) && (L.d.n % 8 == 0) && L.d.grad_dtype == BR_BF16 && false;
+               (L.d.m % 8 == 0) && (L.d.n % 8 == 0) && L.d.grad_dtype == BR_BF16;
   }
 }
 
@@ -316,7 +319,7 @@ size_t buf_bytes(const Layer& L, int which, void** ptr) {
     case BR_BUF_V: *ptr = L.V; return L.V ? 4 * n * n : 0;
     case BR_BUF_L: *ptr = L.L; return L.L ? 4 * m * m : 0;
     case BR_BUF_R: *ptr = L.R; return L.R ? 4 * n * n : 0;
-    case BR_BUF_RING: *ptr = L.ring; return L.ring ? (size_t)L.d.tau_max * m * n * dtype_size(L.d.grad_dtype) : 0;
+    case BR_BUF_RING: *ptr = L.d.tau_max > 0 ? L.ring : nullptr; return L.d.tau_max > 0 ? (size_t)L.d.tau_max * m * n * dtype_size(L.d.grad_dtype) : 0;
     default: *ptr = nullptr; return 0;
   }
 }
@@ -446,13 +449,23 @@ br_status br_step(br_handle* h, const void* const* grads, int tau) {
   // ---- integer state (host) ---------------------------------------------------------------
   h->calls += 1;
   std::vector<const void*> G(nl, nullptr);
+  std::vector<char> stored(nl, 0);
   bool any = false;
   for (int i = 0; i < nl; ++i) {
     Layer& L = h->layers[i];
     const int tl = tau < 0 ? L.d.tau_max : tau;
     const int64_t src_call = h->calls - tl;     // Eq. (delayed_grad)
     if (src_call >= 1) {
-      G[i] = (tl == 0) ? grads[i] : ring_slot_ptr(L, (src_call - 1) % L.d.tau_max);
+      if (tl == 0 && L.use_tc) {
+        // the tensor-core path reads through the ring: store g_c first (no older slot is needed)
+        const size_t bytes = (size_t)L.d.m * L.d.n * dtype_size(L.d.grad_dtype);
+        void* dst = const_cast<void*>(ring_slot_ptr(L, (h->calls - 1) % L.ring_slots));
+        BR_CUDA(h, cudaMemcpyAsync(dst, grads[i], bytes, cudaMemcpyDeviceToDevice, h->stream));
+        G[i] = dst;
+        stored[i] = 1;
+      } else {
+        G[i] = (tl == 0) ? grads[i] : ring_slot_ptr(L, (src_call - 1) % L.ring_slots);
+      }
       L.t += 1;
       any = true;
     }
@@ -478,15 +491,15 @@ br_status br_step(br_handle* h, const void* const* grads, int tau) {
       return (int)refresh_layer(hh, hh->layers[layer]);
     };
     const char* terr = nullptr;
-    int rc = tc_step_run(h->tc, h->layers, G, hp, h->d_status, h->stream, &h->stats, cb, &terr);
+    int rc = tc_step_run(h->tc, h->layers, G, h->calls, tau, hp, h->d_status, h->stream, &h->stats, cb, &terr);
     if (rc != 0) { h->err = terr ? terr : "tensor-core step failed"; return rc < 0 ? (br_status)rc : BR_ERR_CUDA; }
   }
   // ---- store g_c in the ring (after every reader of the slot it may overwrite) --------------
   for (int i = 0; i < nl; ++i) {
     Layer& L = h->layers[i];
-    if (L.d.tau_max <= 0) continue;
+    if (L.ring_slots <= 0 || stored[i]) continue;
     const size_t bytes = (size_t)L.d.m * L.d.n * dtype_size(L.d.grad_dtype);
-    void* dst = const_cast<void*>(ring_slot_ptr(L, (h->calls - 1) % L.d.tau_max));
+    void* dst = const_cast<void*>(ring_slot_ptr(L, (h->calls - 1) % L.ring_slots));
     BR_CUDA(h, cudaMemcpyAsync(dst, grads[i], bytes, cudaMemcpyDeviceToDevice, h->stream));
   }
   return any ? BR_OK : BR_WARMUP;

@@ -79,33 +79,35 @@ enum Epilogue : int32_t {
 };
 
 struct TcOperand {
-  const void* ptr;      // bf16, DEVICE
-  int64_t ld;           // elements
-  int32_t mn_major;     // 1: stored K x MN (MN contiguous); 0: stored MN x K (K contiguous)
+  const void* ptr = nullptr;      // bf16, DEVICE (slot 0 when the operand lives in a ring)
+  int64_t ld = 0;                 // elements
+  int32_t mn_major = 0;           // 1: stored K x MN (MN contiguous); 0: stored MN x K (K contiguous)
+  int32_t ring_slots = 0;         // > 0: the operand is the stale-gradient ring of this many slots
+  int64_t slot_stride_bytes = 0;  // distance between ring slots
 };
 
 struct TcProblem {
-  int64_t Md, Nd, K;
-  int32_t n_pairs;      // 1..3; all pairs share majors and leading dimensions
+  int64_t Md = 0, Nd = 0, K = 0;
+  int32_t n_pairs = 0;            // 1..3; all pairs share majors
   TcOperand A[3], B[3];
-  int32_t epilogue;
-  float alpha, beta, eps;
-  float* D; int64_t ldd;            // fp32 in/out
-  __nv_bfloat16* Dh; __nv_bfloat16* Dl; int64_t ldh;  // bf16 outputs
+  int32_t epilogue = EPI_AXPBY_F32;
+  int32_t tau_max = 0;            // of the layer (delay bookkeeping on the device)
+  int32_t dyn_scalars = 0;        // 1: alpha / beta come from the launch arguments
+  float alpha = 1.f, beta = 0.f, eps = 0.f;
+  float* D = nullptr; int64_t ldd = 0;                                   // fp32 in/out
+  __nv_bfloat16* Dh = nullptr; __nv_bfloat16* Dl = nullptr; int64_t ldh = 0;  // bf16 outputs
 };
 
-struct TcPlan;  // opaque: device problem table + tensor maps, built on the host
+struct TcPlan;  // opaque: device problem table with its tensor maps, built on the host
 
-// Build a plan for a list of problems that can run concurrently in one launch.
+// Build a plan for problems that may run concurrently in one launch.  Synchronises `s` once.
 // Returns nullptr and sets *err on failure.
 TcPlan* tc_plan_create(const TcProblem* problems, int n, int device, cudaStream_t s, const char** err);
 void tc_plan_destroy(TcPlan* p);
-// Scalars may change between launches (eta_t): patch alpha/beta of problem i (host side, copied
-// with the next launch).
-void tc_plan_set_scalars(TcPlan* p, int i, float alpha, float beta);
-// Re-point operands / outputs of problem i (same shapes and strides): used for ring slots.
-int tc_plan_set_operand(TcPlan* p, int i, int pair, int which /*0=A,1=B*/, const void* ptr);
-cudaError_t tc_plan_launch(TcPlan* p, int* status_word, cudaStream_t s);
+// calls / tau: delay bookkeeping (a problem whose layer has calls - tau < 1 is skipped; ring
+// operands read slot (calls - 1 - tau) mod slots; tau < 0 means the layer's tau_max).
+cudaError_t tc_plan_launch(TcPlan* p, long long calls, int tau, float dyn_alpha, float dyn_beta,
+                           int* status_word, cudaStream_t s);
 double tc_plan_flops(const TcPlan* p);
 int tc_supported(int device);
 

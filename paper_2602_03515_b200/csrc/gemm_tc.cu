@@ -1,0 +1,591 @@
+// Grouped bf16 contraction on the 5th-generation tensor cores (sm_100a):
+//   D_tile = sum over operand pairs p and k-blocks of A_p[128 x 64] * B_p[256 x 64]^T
+// TMA (cp.async.bulk.tensor, 128-byte swizzle) stages operand tiles in shared memory, one elected
+// thread issues tcgen05.mma (kind::f16, bf16 operands, fp32 accumulation) into tensor memory,
+// four epilogue warps read the accumulator back with tcgen05.ld and apply a fused epilogue
+// (factor EMA, bf16 hi/lo split, second-moment update, Adam scaling, weight write).
+//
+// One persistent CTA per SM walks a static tile list that spans every problem of a launch
+// (all layers of one phase of the step), so small and large matrices share one launch.
+// Two 256-column accumulators in tensor memory let the epilogue of a tile overlap the main
+// loop of the next one.
+//
+// Operands may be K-major (K contiguous) or MN-major (M / N contiguous); the latter is how the
+// row-major G, U, V enter products that contract over their row index (G^T G, U^T G, T V).
+// Every tensor map is 3-D; the third coordinate selects a ring slot for operands that live in
+// the stale-gradient ring and is 0 otherwise.
+//
+// Every wait on an mbarrier is bounded: when a wait gives up the CTA raises an abort flag,
+// records BR_ERR_TIMEOUT in the status word, leaves its loops, frees its tensor memory and
+// returns; later launches return at once while the status word is negative.
+#include <cuda.h>
+
+#include <cstring>
+#include <mutex>
+#include <string>
+#include <vector>
+
+#include "br_internal.h"
+
+namespace br {
+
+namespace {
+
+constexpr int BM = 128, BN = 256, BK = 64;       // tile (elements); BK*2 bytes = one 128-byte swizzle row
+constexpr int UMMA_K = 16;
+constexpr int STAGES = 4;
+constexpr int A_BYTES = BM * BK * 2;             // 16 KiB
+constexpr int B_BYTES = BN * BK * 2;             // 32 KiB
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024;   // + slack to align the tiles to 1 KiB
+constexpr int TMEM_COLS = 512;
+constexpr int NUM_THREADS = 192;                 // warp 0: TMA, warp 1: MMA, warps 2..5: epilogue
+constexpr int MAX_PAIRS = 3;
+constexpr int GROUP_M = 8;                       // tile rasterisation: 8 row-blocks per column sweep
+
+struct alignas(128) DevProblem {
+  CUtensorMap mapA[MAX_PAIRS];
+  CUtensorMap mapB[MAX_PAIRS];
+  int32_t Md, Nd, K, n_pairs;
+  int32_t a_mn, b_mn, epilogue, tiles_m;
+  int32_t tiles_n, tile_begin, tile_count, tau_max;
+  int32_t ring_slots, a_ring_mask, b_ring_mask, dyn_scalars;
+  float alpha, beta, eps, pad_;
+  float* D;
+  long long ldd;
+  __nv_bfloat16* Dh;
+  __nv_bfloat16* Dl;
+  long long ldh;
+  long long pad2_;
+};
+
+// ---------------------------------------------------------------------------------------------
+// PTX wrappers
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok;
+}
+__device__ __forceinline__ uint64_t global_timer_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+
+constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s: far above any legitimate wait
+
+// Bounded wait.  Returns false when the wait gave up or another role raised the abort flag.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          int* status) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = global_timer_ns();
+  uint32_t spins = 0;
+  while (true) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((++spins & 0xFF) == 0) {
+      if (*abort_flag) return false;
+      if (global_timer_ns() - t0 > kWaitLimitNs) {
+        *abort_flag = 1;
+        atomicMin(status, (int)BR_ERR_TIMEOUT);
+        return false;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar,
+                                            int x, int y, int z) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(x), "r"(y), "r"(z)
+      : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// Arrive on an mbarrier once every tcgen05.mma issued so far by this thread has completed.
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle.  lbo / sbo in bytes.
+//   K-major : rows of 128 bytes (64 elements of K); 8-row groups 1024 bytes apart (sbo); lbo unused.
+//   MN-major: rows of 128 bytes (64 elements of M/N), one row per k; 8-k groups sbo apart,
+//             64-element M/N blocks lbo apart.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)((lbo >> 4) & 0x3FFFu) << 16;
+  d |= (uint64_t)((sbo >> 4) & 0x3FFFu) << 32;
+  d |= 1ull << 46;     // descriptor version of this architecture
+  d |= 2ull << 61;     // 128-byte swizzle
+  return d;
+}
+
+// Instruction descriptor of kind::f16: fp32 accumulator, bf16 A and B, M = 128, N = 256.
+__device__ __forceinline__ uint32_t make_idesc(int a_mn, int b_mn) {
+  uint32_t d = 0;
+  d |= 1u << 4;                       // accumulator format: fp32
+  d |= 1u << 7;                       // A format: bf16
+  d |= 1u << 10;                      // B format: bf16
+  d |= (uint32_t)(a_mn ? 1 : 0) << 15;
+  d |= (uint32_t)(b_mn ? 1 : 0) << 16;
+  d |= (uint32_t)(BN >> 3) << 17;
+  d |= (uint32_t)(BM >> 4) << 24;
+  return d;
+}
+
+__device__ __forceinline__ uint32_t pack2_bf16(float a, float b) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+struct TileInfo {
+  const DevProblem* p;
+  int m0, n0, z;
+  bool active;
+};
+
+// tile index -> problem (binary search over tile_begin) and block coordinates
+__device__ __forceinline__ TileInfo locate_tile(const DevProblem* probs, int n_probs, int tile,
+                                                long long calls, int tau) {
+  int lo = 0, hi = n_probs - 1;
+  while (lo < hi) {
+    int mid = (lo + hi + 1) >> 1;
+    if (probs[mid].tile_begin <= tile) lo = mid; else hi = mid - 1;
+  }
+  const DevProblem* p = probs + lo;
+  TileInfo ti;
+  ti.p = p;
+  const int local = tile - p->tile_begin;
+  const int per_group = GROUP_M * p->tiles_n;
+  const int group = local / per_group;
+  const int first_m = group * GROUP_M;
+  const int gsz = min(p->tiles_m - first_m, GROUP_M);
+  const int in_group = local - group * per_group;
+  ti.m0 = (first_m + in_group % gsz) * BM;
+  ti.n0 = (in_group / gsz) * BN;
+  // delayed-gradient bookkeeping: the layer is active once call - tau >= 1; the gradient to
+  // apply sits in ring slot (calls - 1 - tau) mod slots
+  const int tl = tau < 0 ? p->tau_max : tau;
+  ti.active = (calls - tl >= 1);
+  ti.z = 0;
+  if (p->ring_slots > 0 && ti.active) ti.z = (int)((calls - 1 - tl) % p->ring_slots);
+  return ti;
+}
+
+// ---------------------------------------------------------------------------------------------
+// The kernel
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+k_tc_gemm(const DevProblem* __restrict__ probs, int n_probs, int total_tiles, long long calls,
+          int tau, float dyn_alpha, float dyn_beta, int* status) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ alignas(8) uint64_t bars[2 * STAGES + 4];
+  __shared__ uint32_t tmem_slot;
+  __shared__ int abort_word;
+  volatile int* abort_flag = &abort_word;
+
+  if (*reinterpret_cast<volatile int*>(status) < 0) return;   // an earlier launch failed
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  auto sA = [&](int s) { return tiles_base + (uint32_t)s * A_BYTES; };
+  auto sB = [&](int s) { return tiles_base + (uint32_t)STAGES * A_BYTES + (uint32_t)s * B_BYTES; };
+  const uint32_t bar0 = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
+  auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + a); };
+  auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + 2 + a); };
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
+    abort_word = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&tmem_slot);
+
+  if (warp == 0) {
+    // ======================= TMA producer =======================
+    if (lane == 0) {
+      int stage = 0; uint32_t phase = 0;
+      for (int tile = blockIdx.x; tile < total_tiles && !*abort_flag; tile += gridDim.x) {
+        const TileInfo ti = locate_tile(probs, n_probs, tile, calls, tau);
+        if (!ti.active) continue;
+        const DevProblem* p = ti.p;
+        const int nkb = (p->K + BK - 1) / BK;
+        bool ok = true;
+        for (int pr = 0; pr < p->n_pairs && ok; ++pr) {
+          const CUtensorMap* ma = &p->mapA[pr];
+          const CUtensorMap* mb = &p->mapB[pr];
+          const int za = ((p->a_ring_mask >> pr) & 1) ? ti.z : 0;
+          const int zb = ((p->b_ring_mask >> pr) & 1) ? ti.z : 0;
+          for (int kb = 0; kb < nkb; ++kb) {
+            if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, status)) { ok = false; break; }
+            mbar_expect_tx(full_bar(stage), STAGE_BYTES);
+            const int k0 = kb * BK;
+            if (p->a_mn) {
+#pragma unroll
+              for (int j = 0; j < BM / 64; ++j)
+                tma_load_3d(sA(stage) + j * (BK * 128), ma, full_bar(stage), ti.m0 + 64 * j, k0, za);
+            } else {
+              tma_load_3d(sA(stage), ma, full_bar(stage), k0, ti.m0, za);
+            }
+            if (p->b_mn) {
+#pragma unroll
+              for (int j = 0; j < BN / 64; ++j)
+                tma_load_3d(sB(stage) + j * (BK * 128), mb, full_bar(stage), ti.n0 + 64 * j, k0, zb);
+            } else {
+              tma_load_3d(sB(stage), mb, full_bar(stage), k0, ti.n0, zb);
+            }
+            if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+          }
+        }
+        if (!ok) break;
+      }
+    }
+  } else if (warp == 1) {
+    // ======================= MMA issuer =======================
+    if (lane == 0) {
+      int stage = 0; uint32_t phase = 0;
+      int acc = 0; uint32_t acc_phase = 0;
+      for (int tile = blockIdx.x; tile < total_tiles && !*abort_flag; tile += gridDim.x) {
+        const TileInfo ti = locate_tile(probs, n_probs, tile, calls, tau);
+        if (!ti.active) continue;
+        const DevProblem* p = ti.p;
+        const int nkb = (p->K + BK - 1) / BK;
+        const uint32_t idesc = make_idesc(p->a_mn, p->b_mn);
+        // K-major: advance 32 bytes per 16-element k step inside the swizzle row;
+        // MN-major: 16 k rows = two 8-row groups of 1024 bytes.
+        const uint32_t a_lbo = p->a_mn ? BK * 128 : 0, a_adv = p->a_mn ? 2048 : 32;
+        const uint32_t b_lbo = p->b_mn ? BK * 128 : 0, b_adv = p->b_mn ? 2048 : 32;
+        if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, status)) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)acc * BN;
+        uint32_t accumulate = 0;
+        bool ok = true;
+        for (int it = 0; it < p->n_pairs * nkb; ++it) {
+          if (!mbar_wait(full_bar(stage), phase, abort_flag, status)) { ok = false; break; }
+          tc_fence_after();
+          const uint64_t adesc = make_smem_desc(sA(stage), a_lbo, 1024);
+          const uint64_t bdesc = make_smem_desc(sB(stage), b_lbo, 1024);
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k) {
+            umma_bf16(d_tmem, adesc + (uint64_t)((k * a_adv) >> 4), bdesc + (uint64_t)((k * b_adv) >> 4),
+                      idesc, accumulate);
+            accumulate = 1;
+          }
+          umma_commit(empty_bar(stage));          // frees the stage once these MMAs have read it
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        umma_commit(tfull_bar(acc));              // accumulator complete
+        acc ^= 1;
+        if (acc == 0) acc_phase ^= 1u;
+      }
+    }
+  } else {
+    // ======================= epilogue warps =======================
+    const int quad = warp & 3;                    // tensor-memory lane quadrant this warp may read
+    int acc = 0; uint32_t acc_phase = 0;
+    for (int tile = blockIdx.x; tile < total_tiles && !*abort_flag; tile += gridDim.x) {
+      const TileInfo ti = locate_tile(probs, n_probs, tile, calls, tau);
+      if (!ti.active) continue;
+      const DevProblem* p = ti.p;
+      if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag, status)) break;
+      tc_fence_after();
+      const int row = ti.m0 + quad * 32 + lane;
+      const bool row_ok = row < p->Md;
+      const float alpha = p->dyn_scalars ? dyn_alpha : p->alpha;
+      const float beta = p->dyn_scalars ? dyn_beta : p->beta;
+      const float eps = p->eps;
+      const int epi = p->epilogue;
+#pragma unroll 1
+      for (int c0 = 0; c0 < BN; c0 += 32) {
+        if (ti.n0 + c0 >= p->Nd) break;           // uniform across the warp
+        float v[32];
+        tmem_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * BN + c0), v);
+        if (!row_ok) continue;
+        const int col0 = ti.n0 + c0;
+        if (epi == EPI_AXPBY_F32) {
+          float* d = p->D + (long long)row * p->ldd + col0;
+#pragma unroll
+          for (int j = 0; j < 32; j += 4) {
+            if (col0 + j >= p->Nd) break;
+            float4 o = make_float4(alpha * v[j], alpha * v[j + 1], alpha * v[j + 2], alpha * v[j + 3]);
+            if (beta != 0.0f) {
+              const float4 old = *reinterpret_cast<const float4*>(d + j);
+              o.x = fmaf(beta, old.x, o.x); o.y = fmaf(beta, old.y, o.y);
+              o.z = fmaf(beta, old.z, o.z); o.w = fmaf(beta, old.w, o.w);
+            }
+            *reinterpret_cast<float4*>(d + j) = o;
+          }
+        } else if (epi == EPI_SECOND_MOMENT) {
+          float* d = p->D + (long long)row * p->ldd + col0;
+#pragma unroll
+          for (int j = 0; j < 32; j += 4) {
+            if (col0 + j >= p->Nd) break;
+            float4 s = *reinterpret_cast<const float4*>(d + j);
+            s.x = fmaf(beta, s.x, alpha * v[j] * v[j]);
+            s.y = fmaf(beta, s.y, alpha * v[j + 1] * v[j + 1]);
+            s.z = fmaf(beta, s.z, alpha * v[j + 2] * v[j + 2]);
+            s.w = fmaf(beta, s.w, alpha * v[j + 3] * v[j + 3]);
+            *reinterpret_cast<float4*>(d + j) = s;
+          }
+        } else if (epi == EPI_SCALE_BF16) {
+          const float* d = p->D + (long long)row * p->ldd + col0;
+          __nv_bfloat16* xh = p->Dh + (long long)row * p->ldh + col0;
+#pragma unroll
+          for (int j = 0; j < 32; j += 8) {
+            if (col0 + j >= p->Nd) break;
+            const float4 s0 = *reinterpret_cast<const float4*>(d + j);
+            const float4 s1 = *reinterpret_cast<const float4*>(d + j + 4);
+            uint4 o;
+            o.x = pack2_bf16(v[j] / sqrtf(s0.x + eps), v[j + 1] / sqrtf(s0.y + eps));
+            o.y = pack2_bf16(v[j + 2] / sqrtf(s0.z + eps), v[j + 3] / sqrtf(s0.w + eps));
+            o.z = pack2_bf16(v[j + 4] / sqrtf(s1.x + eps), v[j + 5] / sqrtf(s1.y + eps));
+            o.w = pack2_bf16(v[j + 6] / sqrtf(s1.z + eps), v[j + 7] / sqrtf(s1.w + eps));
+            *reinterpret_cast<uint4*>(xh + j) = o;
+          }
+        } else {  // EPI_SPLIT_BF16
+          __nv_bfloat16* dh = p->Dh + (long long)row * p->ldh + col0;
+          __nv_bfloat16* dl = p->Dl ? p->Dl + (long long)row * p->ldh + col0 : nullptr;
+#pragma unroll
+          for (int j = 0; j < 32; j += 8) {
+            if (col0 + j >= p->Nd) break;
+            float h[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) h[e] = __bfloat162float(__float2bfloat16_rn(v[j + e]));
+            uint4 o;
+            o.x = pack2_bf16(h[0], h[1]); o.y = pack2_bf16(h[2], h[3]);
+            o.z = pack2_bf16(h[4], h[5]); o.w = pack2_bf16(h[6], h[7]);
+            *reinterpret_cast<uint4*>(dh + j) = o;
+            if (dl) {
+              uint4 l;
+              l.x = pack2_bf16(v[j] - h[0], v[j + 1] - h[1]);
+              l.y = pack2_bf16(v[j + 2] - h[2], v[j + 3] - h[3]);
+              l.z = pack2_bf16(v[j + 4] - h[4], v[j + 5] - h[5]);
+              l.w = pack2_bf16(v[j + 6] - h[6], v[j + 7] - h[7]);
+              *reinterpret_cast<uint4*>(dl + j) = l;
+            }
+          }
+        }
+      }
+      // all tcgen05.ld of this warp have completed (wait::ld): hand the accumulator back
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar(acc));
+      acc ^= 1;
+      if (acc == 0) acc_phase ^= 1u;
+    }
+  }
+
+  // teardown: every role has left its loop (all waits are bounded)
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Host side: tensor-map encoding and plans
+// ---------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  });
+  return fn;
+}
+
+// rows = extent of the M / N index, K = contraction extent.
+bool encode_operand(CUtensorMap* map, const TcOperand& op, int64_t rows, int64_t K, int box_rows,
+                    std::string* err) {
+  EncodeTiledFn enc = get_encode_fn();
+  if (!enc) { *err = "cuTensorMapEncodeTiled is not available from the driver"; return false; }
+  const int64_t inner = op.mn_major ? rows : K;
+  const int64_t outer = op.mn_major ? K : rows;
+  const int slots = op.ring_slots > 0 ? op.ring_slots : 1;
+  const uint64_t slot_stride = op.ring_slots > 0 ? (uint64_t)op.slot_stride_bytes
+                                                 : (uint64_t)op.ld * 2ull * (uint64_t)outer;
+  if ((reinterpret_cast<uintptr_t>(op.ptr) & 15) || (op.ld % 8) || (slot_stride % 16)) {
+    *err = "tensor-core operand is not 16-byte aligned (pointer, leading dimension or slot stride)";
+    return false;
+  }
+  cuuint64_t dims[3] = {(cuuint64_t)inner, (cuuint64_t)outer, (cuuint64_t)slots};
+  cuuint64_t strides[2] = {(cuuint64_t)op.ld * 2ull, (cuuint64_t)slot_stride};
+  cuuint32_t box[3] = {64u, (cuuint32_t)(op.mn_major ? BK : box_rows), 1u};
+  cuuint32_t estr[3] = {1u, 1u, 1u};
+  CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(op.ptr), dims, strides, box,
+                   estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    *err = "cuTensorMapEncodeTiled failed with code " + std::to_string((int)r);
+    return false;
+  }
+  return true;
+}
+
+}  // namespace
+
+struct TcPlan {
+  DevProblem* d_probs = nullptr;
+  int n = 0;
+  int total_tiles = 0;
+  double flops = 0.0;
+  int sm_count = 148;
+  std::string err;
+};
+
+int tc_supported(int device) {
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return 0;
+  return prop.major == 10 && get_encode_fn() != nullptr;
+}
+
+TcPlan* tc_plan_create(const TcProblem* problems, int n, int device, cudaStream_t s, const char** err) {
+  static thread_local std::string last;
+  auto fail = [&](const std::string& m) -> TcPlan* { last = m; if (err) *err = last.c_str(); return nullptr; };
+  if (n <= 0) return fail("empty plan");
+  std::vector<DevProblem> host(n);
+  int tile_begin = 0;
+  double flops = 0.0;
+  for (int i = 0; i < n; ++i) {
+    const TcProblem& q = problems[i];
+    DevProblem& d = host[i];
+    std::memset(&d, 0, sizeof d);
+    if (q.n_pairs < 1 || q.n_pairs > MAX_PAIRS || q.Md < 1 || q.Nd < 1 || q.K < 1 ||
+        (q.Md % 8) || (q.Nd % 8) || (q.K % 8) || q.Md > (1ll << 30) || q.Nd > (1ll << 30) || q.K > (1ll << 30))
+      return fail("tensor-core problem: dimensions must be positive multiples of 8");
+    std::string e;
+    for (int p = 0; p < q.n_pairs; ++p) {
+      if (q.A[p].mn_major != q.A[0].mn_major || q.B[p].mn_major != q.B[0].mn_major)
+        return fail("tensor-core problem: all pairs must share operand majors");
+      if (!encode_operand(&d.mapA[p], q.A[p], q.Md, q.K, BM, &e)) return fail(e);
+      if (!encode_operand(&d.mapB[p], q.B[p], q.Nd, q.K, BN, &e)) return fail(e);
+      if (q.A[p].ring_slots > 0) { d.a_ring_mask |= 1 << p; d.ring_slots = q.A[p].ring_slots; }
+      if (q.B[p].ring_slots > 0) { d.b_ring_mask |= 1 << p; d.ring_slots = q.B[p].ring_slots; }
+    }
+    d.Md = (int32_t)q.Md; d.Nd = (int32_t)q.Nd; d.K = (int32_t)q.K; d.n_pairs = q.n_pairs;
+    d.a_mn = q.A[0].mn_major; d.b_mn = q.B[0].mn_major; d.epilogue = q.epilogue;
+    d.tiles_m = (int32_t)((q.Md + BM - 1) / BM);
+    d.tiles_n = (int32_t)((q.Nd + BN - 1) / BN);
+    d.tile_begin = tile_begin;
+    d.tile_count = d.tiles_m * d.tiles_n;
+    tile_begin += d.tile_count;
+    d.tau_max = q.tau_max;
+    d.dyn_scalars = q.dyn_scalars;
+    d.alpha = q.alpha; d.beta = q.beta; d.eps = q.eps;
+    d.D = q.D; d.ldd = q.ldd; d.Dh = q.Dh; d.Dl = q.Dl; d.ldh = q.ldh;
+    const bool need_D = q.epilogue != EPI_SPLIT_BF16;
+    const bool need_H = q.epilogue == EPI_SPLIT_BF16 || q.epilogue == EPI_SCALE_BF16;
+    if ((need_D && (!q.D || (q.ldd % 4) || (reinterpret_cast<uintptr_t>(q.D) & 15))) ||
+        (need_H && (!q.Dh || (q.ldh % 8) || (reinterpret_cast<uintptr_t>(q.Dh) & 15))) ||
+        (q.Dl && (reinterpret_cast<uintptr_t>(q.Dl) & 15)))
+      return fail("tensor-core problem: output pointer missing or misaligned");
+    flops += 2.0 * (double)q.Md * (double)q.Nd * (double)q.K * q.n_pairs;
+  }
+  TcPlan* plan = new TcPlan();
+  plan->n = n;
+  plan->total_tiles = tile_begin;
+  plan->flops = flops;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) == cudaSuccess) plan->sm_count = prop.multiProcessorCount;
+  cudaError_t ce = cudaMalloc(&plan->d_probs, sizeof(DevProblem) * n);
+  if (ce == cudaSuccess)
+    ce = cudaMemcpyAsync(plan->d_probs, host.data(), sizeof(DevProblem) * n, cudaMemcpyHostToDevice, s);
+  if (ce == cudaSuccess) ce = cudaStreamSynchronize(s);   // `host` goes out of scope
+  if (ce != cudaSuccess) {
+    if (plan->d_probs) cudaFree(plan->d_probs);
+    delete plan;
+    return fail(std::string("plan upload: ") + cudaGetErrorString(ce));
+  }
+  static std::once_flag attr_once;
+  std::call_once(attr_once, [] {
+    cudaFuncSetAttribute(k_tc_gemm, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+  });
+  return plan;
+}
+
+void tc_plan_destroy(TcPlan* p) {
+  if (!p) return;
+  if (p->d_probs) cudaFree(p->d_probs);
+  delete p;
+}
+
+double tc_plan_flops(const TcPlan* p) { return p ? p->flops : 0.0; }
+
+cudaError_t tc_plan_launch(TcPlan* p, long long calls, int tau, float dyn_alpha, float dyn_beta,
+                           int* status_word, cudaStream_t s) {
+  const int grid = p->total_tiles < p->sm_count ? p->total_tiles : p->sm_count;
+  // per-device attribute: set again when another device is current (cheap, idempotent)
+  cudaFuncSetAttribute(k_tc_gemm, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+  k_tc_gemm<<<grid, NUM_THREADS, SMEM_BYTES, s>>>(p->d_probs, p->n, p->total_tiles, calls, tau, dyn_alpha,
+                                                  dyn_beta, status_word);
+  return cudaGetLastError();
+}
+
+}  // namespace br

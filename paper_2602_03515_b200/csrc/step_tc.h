@@ -15,6 +15,7 @@ struct Layer {
   float *M = nullptr, *V2 = nullptr, *U = nullptr, *V = nullptr, *L = nullptr, *R = nullptr;
   __nv_bfloat16 *Uh = nullptr, *Ul = nullptr, *Vh = nullptr, *Vl = nullptr;  // bf16 hi/lo of U, V
   char* ring = nullptr;
+  int ring_slots = 0;                 // physical slots: tau_max, or 1 for a tensor-core layer without delay
   size_t slot_stride = 0;             // bytes between ring slots
   int64_t t = 0, refresh_count = 0;
 };
@@ -40,8 +41,8 @@ TcStep* tc_step_create(std::vector<Layer>& layers, const br_hparams& hp, char* s
                        int device, cudaStream_t s, const char** err);
 // Enqueue the updates of every tensor-core layer whose G[i] is non-null.  0 on success,
 // a negative br_status otherwise (message in *err).
-int tc_step_run(TcStep* t, std::vector<Layer>& layers, const std::vector<const void*>& G,
-                const br_hparams& hp, int* d_status, cudaStream_t s, LaunchStats* stats,
+int tc_step_run(TcStep* t, std::vector<Layer>& layers, const std::vector<const void*>& G, long long calls,
+                int tau, const br_hparams& hp, int* d_status, cudaStream_t s, LaunchStats* stats,
                 const TcStepCallbacks& cb, const char** err);
 void tc_step_destroy(TcStep* t);
 

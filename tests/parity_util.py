@@ -29,7 +29,11 @@ class SideBySide:
         self.streams = [GradientStream(w, i) for i in range(len(w.layers))]
         w0 = [initial_weight(w, i) for i in range(len(w.layers))]
         self.weights = [torch.from_numpy(x.copy()).to(self.device) for x in w0]
-        self.oracle = O.make_oracle(w, w0, accum=accum, power_iters=power_iters)
+        # the C-ABI takes its hyper-parameters as fp32: hand the oracle exactly those values
+        f32 = lambda x: float(np.float32(x))
+        self.oracle = O.make_oracle(w, w0, accum=accum, power_iters=power_iters, lr=f32(w.lr),
+                                    beta1=f32(w.beta1), beta2=f32(w.beta2), eps=f32(w.eps),
+                                    weight_decay=f32(w.weight_decay))
         gp = gemm_prec if gemm_prec is not None else (br.BR_GEMM_FP32 if w.gemm_prec == "f32" else br.BR_GEMM_BF16)
         self.opt = br.BasisRotation.from_workload(
             w, self.weights, gemm_prec=gp, power_iters=power_iters,

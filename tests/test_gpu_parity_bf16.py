@@ -1,0 +1,76 @@
+"""GPU parity of the tensor-core (bf16 operands, fp32 accumulation) path against the float64
+oracle through the C-ABI.  Tolerances: per-step parameter update relative L2 <= 2e-2; bases
+(sign-normalised) max-abs <= 1e-3 where the refresh is fed identical factors (teacher-forced);
+integer state bit-exact."""
+from dataclasses import replace
+
+import numpy as np
+import pytest
+
+from workloads import get_workload, LayerSpec, Workload
+from workloads.configs import GEOM_BI, GEOM_UNI, SRC_FIRST, SRC_SECOND, scaled
+
+pytestmark = pytest.mark.gpu
+
+TOL_DW = 2e-2
+
+
+def _run(w, calls, tau=-1, tol=TOL_DW, **kw):
+    from tests.parity_util import SideBySide, rel_l2
+    import paper_2602_03515_b200 as br
+    sbs = SideBySide(w, gemm_prec=br.BR_GEMM_BF16, **kw)
+    worst = 0.0
+    try:
+        for c in range(calls):
+            st_g, st_o, dg, do = sbs.step(tau)
+            assert st_g == st_o, (c, st_g, st_o)
+            for li, (a, b) in enumerate(zip(dg, do)):
+                if b is None:
+                    assert not np.any(a)
+                    continue
+                e = rel_l2(a, b)
+                worst = max(worst, e)
+                assert e <= tol, (c, li, e)
+            for li in range(len(w.layers)):
+                assert sbs.opt.counters(li) == sbs.oracle.counters(li)
+        assert sbs.opt.sync_status() == br.BR_OK
+        for li, lay in enumerate(sbs.oracle.layers):
+            assert rel_l2(sbs.state(li, br.BR_BUF_M), lay.M) < 1e-5
+            if lay.L is not None:
+                assert rel_l2(sbs.state(li, br.BR_BUF_L), lay.L) < 1e-4
+            if lay.R is not None:
+                assert rel_l2(sbs.state(li, br.BR_BUF_R), lay.R) < 1e-4
+    finally:
+        sbs.close()
+    return worst
+
+
+def test_c2_block_quarter_size_bilateral_second():
+    """Transformer block at d_model=256, ffn=1024 (C2 divided by 4), rank-16 signal + 0.1 noise,
+    tau=4, refresh every 10: 24 calls cover warm-up, two refreshes and ragged tiles."""
+    w = scaled(get_workload("c2"), 4)
+    _run(w, 24, tau=4)
+
+
+def test_c3_block_quarter_size_unilateral_first():
+    w = scaled(get_workload("c3"), 4)
+    _run(w, 22, tau=8)
+
+
+def test_ragged_multiple_of_8_shapes_and_tau0():
+    layers = [LayerSpec("a", 136, 200, GEOM_BI, SRC_SECOND, 0), LayerSpec("b", 264, 72, GEOM_UNI, SRC_SECOND, 0),
+              LayerSpec("c", 72, 264, GEOM_UNI, SRC_SECOND, 0), LayerSpec("d", 37, 53, GEOM_BI, SRC_SECOND, 0)]
+    w = Workload("ragged", layers, "bf16", "iid_normal", 0.02, tau=0, freq=3, calls=8, seed=2)
+    _run(w, 8, tau=0)
+
+
+def test_student_t_gradients_per_layer_tau():
+    layers = [LayerSpec("a", 256, 256, GEOM_BI, SRC_SECOND, 3), LayerSpec("e", 1000, 128, GEOM_UNI, SRC_SECOND, 1)]
+    w = Workload("t", layers, "bf16", "student_t", 1e-3, tau=3, freq=4, calls=10, seed=4)
+    _run(w, 10, tau=-1)
+
+
+def test_on_refresh_accumulation_tensor_core():
+    w = Workload("sq", [LayerSpec("a", 128, 128, GEOM_BI, SRC_SECOND, 0)], "bf16", "iid_normal", 0.02, tau=0,
+                 freq=2, calls=6, seed=6)
+    _run(w, 6, tau=0, accum="on_refresh")

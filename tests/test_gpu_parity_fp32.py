@@ -55,8 +55,8 @@ def test_c1_full_trajectory():
     _run(w, w.calls, tau=2)
 
 
-def _small(geom, src, m, n, dtype="f32", kind="iid_normal", tau=1, freq=3, **kw):
-    return Workload("small", [LayerSpec("W", m, n, geom, src, tau)], dtype, kind, 0.05, 4, tau=tau,
+def _small(geom, src, m, n, dtype="f32", kind="iid_normal", tau=1, freq=3, scale=0.05, **kw):
+    return Workload("small", [LayerSpec("W", m, n, geom, src, tau)], dtype, kind, scale, 4, tau=tau,
                     freq=freq, calls=10, gemm_prec="f32", seed=3, **kw)
 
 
@@ -70,12 +70,17 @@ def test_strategy_grid_ragged_shapes(geom, src, m, n):
 
 
 def test_bf16_gradients_lowrank_fp32_gemm():
-    w = _small(GEOM_BI, SRC_SECOND, 72, 104, dtype="bf16", kind="lowrank_noise", tau=2, freq=4)
+    # noise 0.5 against a rank-4 signal: the first refresh then has min_j R_jj/|a_j| ~ 4e-3, so the
+    # fp32 rounding of the stored factors (1e-7 relative) stays below the 1e-4 update tolerance.
+    # (With noise 0.05 the same quantity is 4e-5 and fp32 factor state alone costs ~5e-4.)
+    w = _small(GEOM_BI, SRC_SECOND, 72, 104, dtype="bf16", kind="lowrank_noise", tau=2, freq=4, scale=0.5)
     _run(w, 12, tau=2)
 
 
 def test_weight_decay_and_on_refresh_accumulation():
-    w = _small(GEOM_BI, SRC_SECOND, 48, 24, tau=0, freq=2, weight_decay=0.1)
+    # square, so that one gradient already gives full-rank factors (the literal placement of the
+    # accumulation inside the refresh feeds only every freq-th gradient into L and R)
+    w = _small(GEOM_BI, SRC_SECOND, 32, 32, tau=0, freq=2, weight_decay=0.1)
     _run(w, 8, tau=0, accum="on_refresh")
 
 

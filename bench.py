@@ -1,0 +1,398 @@
+#!/usr/bin/env python
+"""Benchmark of the delayed rotated-Adam step (one step = one br_step over the whole layer set).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c5] [--impl reference]
+
+Prints ONE JSON line.  `value` is whole-job parameters/s (steps/s x parameters of the layer set)
+with gradients resident in HBM; `e2e` is the same metric through the C-ABI with the gradients in
+pinned host memory (host->device copy and a device->host read inside the timed region).
+With N > 1 every rank runs an independent replica of the workload (the path has no exchange
+step); times are the maximum over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from workloads import get_workload  # noqa: E402
+from workloads.configs import GEOM_BI, GEOM_NONE, GEOM_UNI, SRC_SECOND  # noqa: E402
+
+METRIC = "rotated_adam_params_per_sec"
+UNIT = "params/s"
+
+
+# ---------------------------------------------------------------------------------------------
+def algorithmic_flops_per_step(w) -> float:
+    """Contraction work the method itself prescribes per step (Alg. 1 lines 8-11 and the factor
+    EMAs of Alg. 2): bilateral/2nd 8mn(m+n); one-sided on side s: 8 s^2 max (2nd) or 6 s^2 max (1st)."""
+    f = 0.0
+    for l in w.layers:
+        m, n = l.m, l.n
+        if l.geom == GEOM_BI:
+            f += (8.0 if l.src == SRC_SECOND else 6.0) * m * n * (m + n)
+        elif l.geom == GEOM_UNI:
+            s, b = min(m, n), max(m, n)
+            f += (8.0 if l.src == SRC_SECOND else 6.0) * s * s * b
+    return f
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm=d["hbm_gbs"], tf_burst=d["bf16_tflops"], tf_sustained=d.get("bf16_tflops_sustained", d["bf16_tflops"]),
+                    source="measured (MEASURED_PEAKS.json)")
+    return dict(hbm=6650.0, tf_burst=1590.0, tf_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "200", "-i", str(index)],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, power, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.splitlines():
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1])); power.append(float(parts[2]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, parts[3:7]):
+                if v == "Active":
+                    reasons.add(nm)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ---------------------------------------------------------------------------------------------
+def device_gradients(w, device, torch):
+    """One synthetic gradient per layer, generated on the device with the value structure of the
+    workload (throughput runs only; parity runs use the CPU streams of workloads.gradients)."""
+    grads = []
+    for i, l in enumerate(w.layers):
+        g = torch.Generator(device=device)
+        g.manual_seed(1000003 * (w.seed + 1) + i)
+        if w.grad_kind == "lowrank_noise":
+            A = torch.randn(l.m, w.grad_rank, device=device, generator=g)
+            B = torch.randn(l.n, w.grad_rank, device=device, generator=g)
+            x = A @ B.t()
+            x.add_(torch.randn(l.m, l.n, device=device, generator=g), alpha=w.grad_scale)
+        elif w.grad_kind == "student_t":
+            z = torch.randn(l.m, l.n, device=device, generator=g)
+            c = torch.zeros(l.m, l.n, device=device)
+            for _ in range(3):
+                c.addcmul_(*(2 * [torch.randn(l.m, l.n, device=device, generator=g)]))
+            x = z.div_(c.div_(3.0).sqrt_()).mul_(w.grad_scale)
+        else:
+            x = torch.randn(l.m, l.n, device=device, generator=g).mul_(w.grad_scale)
+        grads.append(x.to(torch.bfloat16) if w.grad_dtype == "bf16" else x)
+        del x
+    return grads
+
+
+def fit_tau(w_name, n_layers, tau_req, gemm_prec, free_bytes, margin, br):
+    """Largest ring depth <= tau_req whose state fits the device (ring bytes are linear in tau)."""
+    def total(tau):
+        w = get_workload(w_name, n_layers=n_layers, tau=tau)
+        descs = [br.BrLayerDesc(m=l.m, n=l.n, geom=l.geom, src=l.src, grad_dtype=br.BR_BF16 if w.grad_dtype == "bf16" else br.BR_F32,
+                                tau_max=l.tau_max, freq=0, reserved=0, weight=0) for l in w.layers]
+        hp = br.BrHparams(lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps, weight_decay=0.0, beta_factor=-1.0, freq=w.freq,
+                          power_iters=1, accum=0, gemm_prec=gemm_prec, flags=0, reserved=0, scratch_limit_bytes=0)
+        return br.br_state_bytes(descs, hp)[0]
+    tau = tau_req
+    while tau > 1 and total(tau) > free_bytes - margin:
+        tau -= 1
+    return tau, total(tau)
+
+
+# ---------------------------------------------------------------------------------------------
+def cpu_oracle_sample(w, shapes, reps=1):
+    """Time the float64 oracle (as it stands) on one steady step of each given layer shape."""
+    import numpy as np
+    from oracle import br_oracle as O
+    from dataclasses import replace
+    import threadpoolctl
+    np.ones((256, 256)) @ np.ones((256, 256))
+    total_t, total_params = 0.0, 0
+    for (m, n, geom, src) in shapes:
+        rng = np.random.default_rng(0)
+        lay = O.OracleLayer(np.zeros((m, n)), geom, src, 0)
+        orc = O.Oracle([lay], O.Hyper(lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps, freq=10 ** 9))
+        g = rng.standard_normal((m, n))
+        best = None
+        for _ in range(reps):
+            t0 = time.perf_counter()
+            orc.step([g], 0)
+            dt = time.perf_counter() - t0
+            best = dt if best is None else min(best, dt)
+        total_t += best
+        total_params += m * n
+    try:
+        threads = max(p["num_threads"] for p in threadpoolctl.threadpool_info() if p.get("user_api") == "blas")
+    except Exception:
+        threads = len(os.sched_getaffinity(0))
+    return total_params / total_t, total_t, threads
+
+
+def sample_shapes(w, small: bool):
+    """Distinct (m, n, geom, src) of the workload, largest first; `small` keeps only the cheapest."""
+    seen = []
+    for l in w.layers:
+        key = (l.m, l.n, l.geom, l.src)
+        if l.geom != GEOM_NONE and key not in seen:
+            seen.append(key)
+    seen.sort(key=lambda k: k[0] * k[1] * (k[0] + k[1]))
+    # bounded: drop shapes whose float64 step is beyond ~1.5e12 flop (e.g. a 32000-row embedding factor)
+    seen = [k for k in seen if 8.0 * k[0] * k[1] * (k[0] + k[1]) <= 1.5e12] or seen[:1]
+    return seen[:1] if small else seen[:2]
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = get_workload(args.workload)
+    shapes = sample_shapes(w, small=True)
+    times = []
+    for i in range(args.warmup + args.steps):
+        v, t, threads = cpu_oracle_sample(w, shapes)
+        if i >= args.warmup:
+            times.append(t)
+    ms = 1e3 * sum(times) / len(times)
+    params = sum(m * n for m, n, _, _ in shapes)
+    value = params / (ms / 1e3)
+    sample = "one steady (refresh-free) oracle step of a %dx%d matrix of %s per step" % (shapes[0][0], shapes[0][1], w.name)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64", "data": "synthetic", "config": {"workload": w.name, "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ---------------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="c5")
+    ap.add_argument("--impl", default="ours")
+    ap.add_argument("--layers", type=int, default=None, help="decoder depth override (c4/c5)")
+    ap.add_argument("--tau", type=int, default=None, help="ring depth override")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--scratch-gib", type=float, default=0.0)
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    import paper_2602_03515_b200 as br
+    from paper_2602_03515_b200 import build as _build
+    _build.build()
+    br.load_library()
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    peaks = measured_peaks()
+
+    # ---- workload and memory plan -------------------------------------------------------------
+    w0 = get_workload(args.workload, n_layers=args.layers, tau=args.tau)
+    gemm_prec = br.BR_GEMM_FP32 if w0.gemm_prec == "f32" else br.BR_GEMM_BF16
+    tau_req = w0.tau
+    free0, total_mem = torch.cuda.mem_get_info(dev)
+    n_params0 = w0.n_params
+    gbytes = 2 if w0.grad_dtype == "bf16" else 4
+    reserve = n_params0 * (4 + gbytes) + (6 << 30)       # caller's weights and gradient buffers + headroom
+    if args.workload in ("c4", "c5"):
+        tau, state_bytes = fit_tau(args.workload, args.layers, tau_req, gemm_prec, free0, reserve, br)
+        w = get_workload(args.workload, n_layers=args.layers, tau=tau)
+    else:
+        w, tau = w0, tau_req
+        state_bytes = None
+    n_params = w.n_params
+
+    weights = [torch.empty(l.m, l.n, device=dev).normal_(0.0, 0.02) for l in w.layers]
+    grads = device_gradients(w, dev, torch)
+    stream = torch.cuda.Stream(device=dev)
+    opt = br.BasisRotation.from_workload(w, weights, stream=stream,
+                                         scratch_limit_bytes=int(args.scratch_gib * 2 ** 30))
+    if state_bytes is None:
+        state_bytes = opt.state_bytes()[0]
+
+    def sync_all():
+        torch.cuda.synchronize(dev)
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize(dev)
+
+    with torch.cuda.stream(stream):
+        # ---- priming (untimed): fill the ring, apply one update, refresh every basis once -------
+        for _ in range(tau + 1):
+            opt.step(grads, tau)
+        opt.refresh_basis(-1)
+        assert opt.sync_status() >= 0
+        for _ in range(args.warmup):
+            opt.step(grads, tau)
+        sync_all()
+
+        # ---- timed region: exactly K steps, events on the launching stream -----------------------
+        l0, _ = opt.launch_stats()
+        sampler = ClockSampler(local)
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+        is_refresh = []
+        evs[0].record(stream)
+        for k in range(args.steps):
+            opt.step(grads, tau)
+            is_refresh.append(opt.counters(0)["t"] % w.freq == 0)     # every layer shares tau and freq here
+            evs[k + 1].record(stream)
+        sync_all()
+        clocks = sampler.stop()
+        l1, _ = opt.launch_stats()
+        step_ms = [evs[k].elapsed_time(evs[k + 1]) for k in range(args.steps)]
+        total_ms = evs[0].elapsed_time(evs[-1])
+
+        # ---- one full refresh (every layer), timed on its own --------------------------------------
+        r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        r0.record(stream)
+        opt.refresh_basis(-1)
+        r1.record(stream)
+        sync_all()
+        refresh_ms = r0.elapsed_time(r1)
+
+        # ---- per-kernel device time (separate, profiled steps) -------------------------------------
+        opt.profile(True)
+        prof_steps = 2
+        for _ in range(prof_steps):
+            opt.step(grads, tau)
+        opt.profile(False)
+        prof = opt.get_profile()
+        assert opt.sync_status() >= 0
+
+    steady = [t for t, r in zip(step_ms, is_refresh) if not r] or step_ms
+    steady_ms = sum(steady) / len(steady)
+    amortised_ms = steady_ms + refresh_ms / w.freq
+    times = torch.tensor([amortised_ms, steady_ms, refresh_ms, total_ms / args.steps], device=dev, dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    amortised_ms, steady_ms, refresh_ms, raw_ms = [float(x) for x in times.tolist()]
+    value = world * n_params / (amortised_ms / 1e3)
+
+    # ---- end to end through the C-ABI with host buffers ------------------------------------------
+    e2e = None
+    if args.e2e_steps > 0:
+        host = [torch.empty(g.shape, dtype=g.dtype, pin_memory=True) for g in grads]
+        for h_, g in zip(host, grads):
+            h_.copy_(g)
+        w_host = torch.empty(weights[0].shape, dtype=torch.float32, pin_memory=True)
+        h2d = sum(h_.numel() * h_.element_size() for h_ in host)
+        d2h = w_host.numel() * 4 + 4
+        sync_all()
+        t0 = time.perf_counter()
+        with torch.cuda.stream(stream):
+            for _ in range(args.e2e_steps):
+                for h_, g in zip(host, grads):
+                    g.copy_(h_, non_blocking=True)
+                opt.step(grads, tau)
+                w_host.copy_(weights[0], non_blocking=True)
+                st = opt.sync_status()          # waits for the stream and reads the status word back
+                assert st >= 0
+        sync_all()
+        e2e_ms = 1e3 * (time.perf_counter() - t0) / args.e2e_steps + refresh_ms / w.freq
+        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
+        if world > 1:
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e = {"value": world * n_params / (float(t.item()) / 1e3), "unit": UNIT, "ms_per_step": float(t.item()),
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": args.e2e_steps}
+        del host
+
+    # ---- rooflines -------------------------------------------------------------------------------
+    alg_flops = algorithmic_flops_per_step(w)
+    roofline = None
+    roofline_elem = None
+    if prof["tc_launches"] > 0:
+        tc_ms_step = prof["tc_ms"] / prof_steps
+        achieved = alg_flops / (tc_ms_step / 1e3) / 1e12
+        executed = prof["tc_flops"] / (prof["tc_ms"] / 1e3) / 1e12
+        roofline = {"bound": "tensor", "kernel": "k_tc_gemm", "achieved": achieved, "peak": peaks["tf_sustained"],
+                    "unit": "TFLOP/s", "frac": achieved / peaks["tf_sustained"], "traffic": None,
+                    "executed_tflops": executed, "executed_frac": executed / peaks["tf_sustained"],
+                    "launches_per_step": prof["tc_launches"] / prof_steps, "ms_per_step_in_kernel": tc_ms_step,
+                    "avg_launch_ms": prof["tc_ms"] / prof["tc_launches"],
+                    "peak_source": peaks["source"] + ", bf16 sustained"}
+        if prof["ema_launches"] > 0:
+            gbs = prof["ema_bytes"] / (prof["ema_ms"] / 1e3) / 1e9
+            roofline_elem = {"bound": "hbm", "kernel": "k_ema_momentum", "achieved": gbs, "peak": peaks["hbm"], "unit": "GB/s",
+                             "frac": gbs / peaks["hbm"], "traffic": None, "ms_per_step_in_kernel": prof["ema_ms"] / prof_steps}
+
+    # ---- CPU baseline: the oracle on a bounded sample (rank 0, N = 1 only) -----------------------------
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        shapes = sample_shapes(w, small=False)
+        v, t, threads = cpu_oracle_sample(w, shapes)
+        cpu = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "seconds": t,
+               "sample": "one steady (refresh-free) float64 oracle step of each of " +
+                         ", ".join(f"{m}x{n}" for m, n, _, _ in shapes) + f" from {w.name}"}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": amortised_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16" if gemm_prec == br.BR_GEMM_BF16 else "f32", "data": "synthetic",
+            "steps_per_sec": 1e3 / amortised_ms,
+            "ms_steady_step": steady_ms, "ms_full_refresh": refresh_ms, "ms_raw_mean_of_timed_steps": raw_ms,
+            "timing": "ms_per_step = mean steady step + (one refresh of every basis)/freq; refresh steps inside the timed region are excluded from the steady mean",
+            "config": {"workload": w.name, "layers": len(w.layers), "params": n_params, "geometry": "bilateral+unilateral embedding" if args.workload in ("c4", "c5") else "see workloads/configs.py",
+                       "tau": tau, "tau_requested": tau_req, "freq": w.freq, "grad_dtype": w.grad_dtype, "state_bytes": state_bytes,
+                       "l2": "inputs larger than L2 (no flush needed)" if n_params * 2 > (126 << 20) else "inputs smaller than L2",
+                       "replicas": world, "gradients": "one device-resident synthetic gradient set reused every step"},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": int(l1 - l0),
+            "roofline": roofline, "roofline_elementwise": roofline_elem, "cpu_baseline": cpu,
+            "algorithmic_flops_per_step": alg_flops,
+        }
+        print(json.dumps(line), flush=True)
+    opt.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

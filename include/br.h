@@ -169,6 +169,23 @@ BR_API br_status br_set_state(br_handle* h, int layer, int which, const void* ho
  * contraction kernels since creation (for benchmarks). */
 BR_API br_status br_get_launch_stats(br_handle* h, int64_t* kernel_launches, double* gemm_flops);
 
+/* Device-side timing of the library's own launches, by class, with CUDA events on the handle's
+ * stream.  br_profile(h, 1) starts recording, br_profile(h, 0) stops; br_get_profile waits for the
+ * stream, sums what was recorded since the last call and clears it. */
+typedef struct {
+  double tc_ms;          /* tensor-core contraction launches                                  */
+  double tc_flops;       /* floating-point operations those launches issued                   */
+  int64_t tc_launches;
+  double ema_ms;         /* momentum EMA launches (Alg. 1 line 4, with the bf16 hi/lo of M)    */
+  double ema_bytes;      /* bytes those launches must move (gradient, M in and out, hi/lo)    */
+  int64_t ema_launches;
+  double refresh_ms;     /* Power() spans: power product + QR + conversions                   */
+  double refresh_flops;
+  int64_t refresh_spans;
+} br_profile_stats;
+BR_API br_status br_profile(br_handle* h, int enable);
+BR_API br_status br_get_profile(br_handle* h, br_profile_stats* out);
+
 /* Free everything the handle allocated.  NULL is accepted.  Synchronises the stream. */
 BR_API br_status br_destroy(br_handle* h);
 

@@ -47,6 +47,15 @@ class BrCounters(C.Structure):
         return {k: int(getattr(self, k)) for k, _ in self._fields_}
 
 
+class BrProfileStats(C.Structure):
+    _fields_ = [("tc_ms", C.c_double), ("tc_flops", C.c_double), ("tc_launches", C.c_int64),
+                ("ema_ms", C.c_double), ("ema_bytes", C.c_double), ("ema_launches", C.c_int64),
+                ("refresh_ms", C.c_double), ("refresh_flops", C.c_double), ("refresh_spans", C.c_int64)]
+
+    def as_dict(self):
+        return {k: getattr(self, k) for k, _ in self._fields_}
+
+
 _ALLOC_FN = C.CFUNCTYPE(C.c_void_p, C.c_size_t, C.c_void_p)
 _FREE_FN = C.CFUNCTYPE(None, C.c_void_p, C.c_void_p)
 
@@ -82,6 +91,8 @@ def load_library():
         "br_get_state": ([H, C.c_int, C.c_int, C.c_void_p, C.c_size_t], C.c_int),
         "br_set_state": ([H, C.c_int, C.c_int, C.c_void_p, C.c_size_t], C.c_int),
         "br_get_launch_stats": ([H, C.POINTER(C.c_int64), C.POINTER(C.c_double)], C.c_int),
+        "br_profile": ([H, C.c_int], C.c_int),
+        "br_get_profile": ([H, C.POINTER(BrProfileStats)], C.c_int),
         "br_destroy": ([H], C.c_int),
         "br_strerror": ([C.c_int], C.c_char_p),
         "br_last_error": ([H], C.c_char_p),
@@ -171,6 +182,16 @@ def br_get_launch_stats(handle):
     n, f = C.c_int64(0), C.c_double(0.0)
     _check(load_library().br_get_launch_stats(handle, C.byref(n), C.byref(f)), handle)
     return int(n.value), float(f.value)
+
+
+def br_profile(handle, enable: bool) -> int:
+    return _check(load_library().br_profile(handle, 1 if enable else 0), handle)
+
+
+def br_get_profile(handle) -> dict:
+    st = BrProfileStats()
+    _check(load_library().br_get_profile(handle, C.byref(st)), handle)
+    return st.as_dict()
 
 
 def br_destroy(handle) -> int:
@@ -264,6 +285,12 @@ class BasisRotation:
 
     def launch_stats(self):
         return br_get_launch_stats(self.handle)
+
+    def profile(self, enable: bool):
+        return br_profile(self.handle, enable)
+
+    def get_profile(self) -> dict:
+        return br_get_profile(self.handle)
 
     def _buf_shape(self, layer: int, which: int):
         s = self.specs[layer]

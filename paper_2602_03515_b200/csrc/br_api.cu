@@ -222,8 +222,11 @@ br_status refresh_side(br_handle* h, Layer& L, bool left_side) {
 
 br_status refresh_layer(br_handle* h, Layer& L) {
   br_status st;
+  const double f0 = h->stats.gemm_flops;
+  const int span = h->stats.prof.begin(PROF_REFRESH, h->stream);
   if (L.left && (st = refresh_side(h, L, true)) != BR_OK) return st;
   if (L.right && (st = refresh_side(h, L, false)) != BR_OK) return st;
+  h->stats.prof.end(span, h->stream, h->stats.gemm_flops - f0);
   L.refresh_count += 1;
   return BR_OK;
 }
@@ -615,11 +618,43 @@ br_status br_get_launch_stats(br_handle* h, int64_t* kernel_launches, double* ge
   return BR_OK;
 }
 
+br_status br_profile(br_handle* h, int enable) {
+  if (!h) return BR_ERR_INVALID;
+  h->stats.prof.on = enable != 0;
+  return BR_OK;
+}
+
+br_status br_get_profile(br_handle* h, br_profile_stats* out) {
+  br_status st = check_handle(h);
+  if (st != BR_OK) return st;
+  if (!out) return BR_ERR_INVALID;
+  BR_CUDA(h, cudaStreamSynchronize(h->stream));
+  std::memset(out, 0, sizeof *out);
+  Profiler& P = h->stats.prof;
+  for (auto& sp : P.spans) {
+    float ms = 0.f;
+    cudaEventElapsedTime(&ms, sp.a, sp.b);
+    if (sp.cls == PROF_TC) { out->tc_ms += ms; out->tc_launches += 1; }
+    else if (sp.cls == PROF_EMA) { out->ema_ms += ms; out->ema_launches += 1; }
+    else { out->refresh_ms += ms; out->refresh_spans += 1; }
+    P.free_events.push_back(sp.a);
+    P.free_events.push_back(sp.b);
+  }
+  P.spans.clear();
+  out->tc_flops = P.units[PROF_TC];
+  out->ema_bytes = P.units[PROF_EMA];
+  out->refresh_flops = P.units[PROF_REFRESH];
+  P.units[0] = P.units[1] = P.units[2] = 0.0;
+  return BR_OK;
+}
+
 br_status br_destroy(br_handle* h) {
   if (!h) return BR_OK;
   cudaSetDevice(h->device);
   cudaStreamSynchronize(h->stream);
   if (h->tc) tc_step_destroy(h->tc);
+  for (auto& sp : h->stats.prof.spans) { cudaEventDestroy(sp.a); cudaEventDestroy(sp.b); }
+  for (auto e : h->stats.prof.free_events) cudaEventDestroy(e);
   if (h->slab) {
     if (h->alloc.alloc) h->alloc.free(h->slab, h->alloc.ctx); else cudaFree(h->slab);
   }

@@ -6,6 +6,8 @@
 #include <stdint.h>
 #include <stddef.h>
 
+#include <vector>
+
 #include "br.h"
 
 namespace br {
@@ -13,9 +15,40 @@ namespace br {
 // ---------------------------------------------------------------------------------------------
 // Launch accounting (reported through br_get_launch_stats)
 // ---------------------------------------------------------------------------------------------
+// Optional per-class device timing: CUDA events recorded around the library's own launches on
+// the handle's stream (classes: tensor-core contraction, momentum EMA, refresh).
+enum ProfClass { PROF_TC = 0, PROF_EMA = 1, PROF_REFRESH = 2, PROF_NCLASS = 3 };
+
+struct Profiler {
+  bool on = false;
+  struct Span { cudaEvent_t a, b; int cls; };
+  std::vector<Span> spans;
+  std::vector<cudaEvent_t> free_events;
+  double units[PROF_NCLASS] = {0, 0, 0};     // flops (TC, refresh) or bytes (EMA) issued while on
+  cudaEvent_t get() {
+    cudaEvent_t e;
+    if (!free_events.empty()) { e = free_events.back(); free_events.pop_back(); return e; }
+    cudaEventCreate(&e);
+    return e;
+  }
+  int begin(int cls, cudaStream_t s) {
+    if (!on) return -1;
+    Span sp{get(), get(), cls};
+    cudaEventRecord(sp.a, s);
+    spans.push_back(sp);
+    return (int)spans.size() - 1;
+  }
+  void end(int idx, cudaStream_t s, double u) {
+    if (idx < 0) return;
+    cudaEventRecord(spans[idx].b, s);
+    units[spans[idx].cls] += u;
+  }
+};
+
 struct LaunchStats {
   int64_t launches = 0;
   double gemm_flops = 0.0;
+  Profiler prof;
 };
 
 // ---------------------------------------------------------------------------------------------

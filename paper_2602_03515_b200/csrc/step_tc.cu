@@ -271,14 +271,18 @@ int tc_step_run(TcStep* t, std::vector<Layer>& layers, const std::vector<const v
       if (!g) continue;
       any = true;
       // Alg. 1 line 4, with the bf16 hi/lo pair of the new M for the rotation
+      const int span = stats->prof.begin(PROF_EMA, s);
       cudaError_t e = ema_momentum(L.M, g, 1, L.d.m * L.d.n, hp.beta1, nullptr, c.scr[j].Mh, c.scr[j].Ml, s);
+      stats->prof.end(span, s, 14.0 * (double)L.d.m * (double)L.d.n);
       if (e != cudaSuccess) return cuda_fail("ema_momentum", e);
       stats->launches += 1;
     }
     if (!any) continue;
     auto launch = [&](TcPlan* p, const char* what) -> int {
       if (!p) return 0;
+      const int span = stats->prof.begin(PROF_TC, s);
       cudaError_t e = tc_plan_launch(p, calls, tau, dyn_alpha, dyn_beta, d_status, s);
+      stats->prof.end(span, s, tc_plan_flops(p));
       if (e != cudaSuccess) return cuda_fail(what, e);
       stats->launches += 1;
       stats->gemm_flops += tc_plan_flops(p);

@@ -78,9 +78,10 @@ def test_bf16_gradients_lowrank_fp32_gemm():
 
 
 def test_weight_decay_and_on_refresh_accumulation():
-    # square, so that one gradient already gives full-rank factors (the literal placement of the
-    # accumulation inside the refresh feeds only every freq-th gradient into L and R)
-    w = _small(GEOM_BI, SRC_SECOND, 32, 32, tau=0, freq=2, weight_decay=0.1)
+    # The literal placement of the accumulation inside the refresh feeds only every freq-th
+    # gradient into the factor, so the first refresh sees a single G G^T: a wide unilateral layer
+    # (24 x 96, left factor) keeps that factor full rank and well conditioned.
+    w = _small(GEOM_UNI, SRC_SECOND, 24, 96, tau=0, freq=2, weight_decay=0.1)
     _run(w, 8, tau=0, accum="on_refresh")
 
 

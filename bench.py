@@ -25,6 +25,9 @@ sys.path.insert(0, ROOT)
 from workloads import get_workload  # noqa: E402
 from workloads.configs import GEOM_BI, GEOM_NONE, GEOM_UNI, SRC_SECOND  # noqa: E402
 
+# profiles/k_tc_gemm_c5_4layers.md: 13.8e9 B of DRAM traffic per launch at 3.45e12 executed flop per launch
+NCU_DRAM_BYTES_PER_EXECUTED_FLOP = 13.8e9 / 3.45e12
+
 METRIC = "rotated_adam_params_per_sec"
 UNIT = "params/s"
 
@@ -213,6 +216,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--scratch-gib", type=float, default=0.0)
+    ap.add_argument("--no-refresh", action="store_true",
+                    help="profiling captures only: skip the basis refresh (priming and timing); the line is then not a bench value")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     if args.impl == "reference":
@@ -268,7 +273,8 @@ def main():
         # ---- priming (untimed): fill the ring, apply one update, refresh every basis once -------
         for _ in range(tau + 1):
             opt.step(grads, tau)
-        opt.refresh_basis(-1)
+        if not args.no_refresh:
+            opt.refresh_basis(-1)
         assert opt.sync_status() >= 0
         for _ in range(args.warmup):
             opt.step(grads, tau)
@@ -293,7 +299,8 @@ def main():
         # ---- one full refresh (every layer), timed on its own --------------------------------------
         r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         r0.record(stream)
-        opt.refresh_basis(-1)
+        if not args.no_refresh:
+            opt.refresh_basis(-1)
         r1.record(stream)
         sync_all()
         refresh_ms = r0.elapsed_time(r1)
@@ -352,8 +359,12 @@ def main():
         tc_ms_step = prof["tc_ms"] / prof_steps
         achieved = alg_flops / (tc_ms_step / 1e3) / 1e12
         executed = prof["tc_flops"] / (prof["tc_ms"] / 1e3) / 1e12
+        # DRAM bytes per launch: dram__bytes_read+write of an ncu capture of a small case of this
+        # workload (profiles/), scaled to this run's launches by executed flop per launch
+        traffic = NCU_DRAM_BYTES_PER_EXECUTED_FLOP * prof["tc_flops"] / prof["tc_launches"]
         roofline = {"bound": "tensor", "kernel": "k_tc_gemm", "achieved": achieved, "peak": peaks["tf_sustained"],
-                    "unit": "TFLOP/s", "frac": achieved / peaks["tf_sustained"], "traffic": None,
+                    "unit": "TFLOP/s", "frac": achieved / peaks["tf_sustained"], "traffic": traffic,
+                    "traffic_source": "ncu capture of the 4-layer case, scaled by executed flop per launch",
                     "executed_tflops": executed, "executed_frac": executed / peaks["tf_sustained"],
                     "launches_per_step": prof["tc_launches"] / prof_steps, "ms_per_step_in_kernel": tc_ms_step,
                     "avg_launch_ms": prof["tc_ms"] / prof["tc_launches"],
@@ -383,7 +394,7 @@ def main():
             "config": {"workload": w.name, "layers": len(w.layers), "params": n_params, "geometry": "bilateral+unilateral embedding" if args.workload in ("c4", "c5") else "see workloads/configs.py",
                        "tau": tau, "tau_requested": tau_req, "freq": w.freq, "grad_dtype": w.grad_dtype, "state_bytes": state_bytes,
                        "l2": "inputs larger than L2 (no flush needed)" if n_params * 2 > (126 << 20) else "inputs smaller than L2",
-                       "replicas": world, "gradients": "one device-resident synthetic gradient set reused every step"},
+                       "replicas": world, "refresh_skipped_not_a_bench_value": bool(args.no_refresh), "gradients": "one device-resident synthetic gradient set reused every step"},
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(l1 - l0),
             "roofline": roofline, "roofline_elementwise": roofline_elem, "cpu_baseline": cpu,
             "algorithmic_flops_per_step": alg_flops,

@@ -57,12 +57,14 @@ class SideBySide:
         self.call += 1
         host, dev = self.grads_for(self.call)
         before = [w.detach().cpu().numpy().astype(np.float64) for w in self.weights]
+        before_o = [l.W.copy() for l in self.oracle.layers]
         st_g = self.opt.step(dev, tau)
         st_o = self.oracle.step(host, tau)
         self.torch.cuda.synchronize()
         after = [w.detach().cpu().numpy().astype(np.float64) for w in self.weights]
         dW_g = [a - b for a, b in zip(after, before)]
-        dW_o = [l.last_dW for l in self.oracle.layers]
+        # the whole change of the weights (update plus decoupled decay), None on warm-up calls
+        dW_o = [None if l.last_dW is None else l.W - b for l, b in zip(self.oracle.layers, before_o)]
         return st_g, st_o, dW_g, dW_o
 
     def state(self, layer, which):

@@ -206,6 +206,30 @@ BR_API br_status br_gemm_bf16(void* cuda_stream, int64_t Md, int64_t Nd, int64_t
                        const void* const* A, const void* const* B, int a_mn, int b_mn,
                        int64_t lda, int64_t ldb, float* D, int64_t ldd, float alpha, float beta);
 
+/*
+ * One Power(F, Q) application without any allocation.  (The paper has no counterpart: this is a
+ * library convenience around the Power() step it describes.)
+ *
+ * For callers that cannot allocate device memory when they need a refresh: processes whose
+ * framework already owns all of HBM, services that forbid allocation after start-up, loops that
+ * cannot afford the device-wide synchronisation of cudaMalloc / cudaFree.  Q (k x k fp32, DEVICE,
+ * row-major) is replaced by the Q factor, with a positive diagonal of R, of the fp64 product F*Q;
+ * F is k x k fp32, DEVICE, read only.  The caller owns F and Q.  device_flag, if not NULL, is a
+ * DEVICE int that receives 0 or BR_WARN_RANK_DEFICIENT.
+ *
+ * Scratch lives in a fixed array inside the library's device image (about 3.4 MB on every GPU
+ * that loads the library, held until the process exits), so k is limited to 512: larger orders
+ * return BR_ERR_SHAPE and must use br_create / br_refresh_basis.  The call itself, and everything
+ * it calls, performs no cudaMalloc, cudaFree or other allocating routine.  The first call on a
+ * device looks the array's address up (once per device); make that first call outside any stream
+ * capture.  All calls on a GPU share the one array, which keeps the previous call's contents: the
+ * call clears what must start at zero, and two calls whose work overlaps on the GPU (different
+ * streams, or different threads) race on it -- serialise them.  Enqueues on cuda_stream (the
+ * device of that stream must be current) and does not synchronise.
+ */
+BR_API br_status br_power_static(void* cuda_stream, const float* F, float* Q, int64_t k,
+                                 int* device_flag);
+
 #ifdef __cplusplus
 }
 #endif

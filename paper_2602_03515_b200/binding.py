@@ -94,6 +94,7 @@ def load_library():
         "br_profile": ([H, C.c_int], C.c_int),
         "br_get_profile": ([H, C.POINTER(BrProfileStats)], C.c_int),
         "br_destroy": ([H], C.c_int),
+        "br_power_static": ([C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p], C.c_int),
         "br_strerror": ([C.c_int], C.c_char_p),
         "br_last_error": ([H], C.c_char_p),
         "br_gemm_bf16": ([C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_int, C.POINTER(C.c_void_p), C.POINTER(C.c_void_p), C.c_int, C.c_int, C.c_int64, C.c_int64, C.c_void_p, C.c_int64, C.c_float, C.c_float], C.c_int),
@@ -204,6 +205,16 @@ def br_gemm_bf16(stream_ptr, Md, Nd, K, A_ptrs, B_ptrs, a_mn, b_mn, lda, ldb, D_
     B = (C.c_void_p * n)(*[C.c_void_p(p) for p in B_ptrs])
     return _check(load_library().br_gemm_bf16(C.c_void_p(stream_ptr), Md, Nd, K, n, A, B, int(a_mn), int(b_mn),
                                               lda, ldb, C.c_void_p(D_ptr), ldd, float(alpha), float(beta)))
+
+
+def br_power_static(stream_ptr: int, F_ptr: int, Q_ptr: int, k: int, device_flag_ptr: int = 0) -> int:
+    """Q <- qr(F Q).Q on the device without allocating; see include/br.h for the limits (k <= 512,
+    one shared scratch array per GPU, calls must not overlap on the GPU)."""
+    st = load_library().br_power_static(C.c_void_p(stream_ptr), C.c_void_p(F_ptr), C.c_void_p(Q_ptr), int(k),
+                                        C.c_void_p(device_flag_ptr) if device_flag_ptr else None)
+    if st < 0:
+        raise BrError(st, br_strerror(st) + (": order above 512 does not fit the fixed scratch" if st == BR_ERR_SHAPE else ""))
+    return st
 
 
 # ---- convenience object: torch tensors in, pointers out ----------------------------------------------

@@ -91,6 +91,12 @@ cudaError_t sdgemm(int ta, int tb, int64_t M, int64_t N, int64_t K, double alpha
 cudaError_t dgemm(int ta, int tb, int64_t M, int64_t N, int64_t K, double alpha, const double* A,
                   int64_t lda, const double* B, int64_t ldb, double beta, double* C, int64_t ldc,
                   cudaStream_t s);
+// As dgemm, with the contraction split into nsplit ranges of K whose partial products (nsplit * M * N
+// doubles in `partial`) are added in a fixed order by a second kernel, and with an optional DEVICE
+// flag that cancels the launches when it is non-zero at the time they run.
+cudaError_t dgemm_ex(int ta, int tb, int64_t M, int64_t N, int64_t K, double alpha, const double* A,
+                     int64_t lda, const double* B, int64_t ldb, double beta, double* C, int64_t ldc,
+                     int nsplit, double* partial, const int* skip, cudaStream_t s);
 
 // ---------------------------------------------------------------------------------------------
 // QR with positive diagonal in fp64 (qr.cu).  A (k x k, row-major, ld = k) is overwritten by

@@ -1,7 +1,6 @@
-// SIMT (FFMA / DFMA) contractions: the accurate path.  Used for BR_GEMM_FP32, for layers whose
-// shapes the tensor-core tiles do not take, and -- in fp64 -- for the basis refresh, where
-// Power(A, Q) must be resolved far below the fp32 rounding level (the first refresh of a
-// low-rank-plus-noise stream has a column-scaled condition number of 1e4..1e5).
+// SIMT (FFMA) contractions: the accurate fp32 path.  Used for BR_GEMM_FP32 and for layers whose
+// shapes the tensor-core tiles do not take.  (The fp64 contractions of the basis refresh live in
+// dgemm.cu.)
 //
 // C = alpha * op(A) op(B) + beta * C, all row-major.  op(A) is M x K, op(B) is K x N.
 #include "br_internal.h"
@@ -107,24 +106,6 @@ cudaError_t sgemm(int ta, int tb, int64_t M, int64_t N, int64_t K, float alpha, 
                   int64_t lda, const float* B, int64_t ldb, float beta, float* C, int64_t ldc,
                   cudaStream_t s) {
   return launch<float, float, float>(ta, tb, M, N, K, alpha, A, lda, B, ldb, beta, C, ldc, s);
-}
-
-cudaError_t sdgemm(int ta, int tb, int64_t M, int64_t N, int64_t K, double alpha, const float* A,
-                   int64_t lda, const float* B, int64_t ldb, double beta, double* C, int64_t ldc,
-                   cudaStream_t s) {
-  return launch<float, float, double>(ta, tb, M, N, K, alpha, A, lda, B, ldb, beta, C, ldc, s);
-}
-
-cudaError_t fdgemm(int ta, int tb, int64_t M, int64_t N, int64_t K, double alpha, const float* A,
-                   int64_t lda, const double* B, int64_t ldb, double beta, double* C, int64_t ldc,
-                   cudaStream_t s) {
-  return launch<float, double, double>(ta, tb, M, N, K, alpha, A, lda, B, ldb, beta, C, ldc, s);
-}
-
-cudaError_t dgemm(int ta, int tb, int64_t M, int64_t N, int64_t K, double alpha, const double* A,
-                  int64_t lda, const double* B, int64_t ldb, double beta, double* C, int64_t ldc,
-                  cudaStream_t s) {
-  return launch<double, double, double>(ta, tb, M, N, K, alpha, A, lda, B, ldb, beta, C, ldc, s);
 }
 
 }  // namespace br

@@ -113,7 +113,8 @@ def test_variable_tau_per_call():
 
 def test_qr_many_panels_teacher_forced():
     """Forced refresh from a given L, U (set through the API) against the oracle's Power():
-    k = 200 spans 7 panels with a ragged last one; the factor has a 1e4 spread of eigenvalues."""
+    k = 200 spans 4 panels of 64 columns with a ragged last one; the factor has a 1e4 spread of
+    eigenvalues."""
     import torch
     import paper_2602_03515_b200 as br
     from oracle import br_oracle as O
@@ -142,6 +143,45 @@ def test_qr_many_panels_teacher_forced():
         assert np.max(np.abs(U.T @ U - np.eye(k))) < 1e-5
         assert basis_err(U, ref) < 1e-5
         assert opt.counters(0)["refresh_count"] == 1 and opt.counters(0)["t"] == 1
+    finally:
+        opt.close()
+
+
+@pytest.mark.parametrize("start", ["identity", "tracking"])
+def test_qr_wide_panels_split_contractions(start):
+    """k = 1160: nine 128-column panels and a ragged 8-column one, contractions split over K.
+    "identity": Power(F, I) for a factor with a 1e5 spread of eigenvalues, the ill-conditioned
+    first refresh (every column of F is dominated by the leading eigenvectors; both Cholesky-QR
+    passes run).  "tracking": the basis already holds approximate eigenvectors, so the columns of
+    F Q are nearly orthogonal and the second pass is cancelled by the device-side flag."""
+    import torch
+    import paper_2602_03515_b200 as br
+    from oracle import br_oracle as O
+    from tests.parity_util import basis_err
+    k, n = 1160, 8
+    rng = np.random.default_rng(5)
+    Qe, _ = np.linalg.qr(rng.standard_normal((k, k)))
+    lam = np.logspace(0, -5, k)
+    F = ((Qe * lam) @ Qe.T).astype(np.float32)
+    if start == "identity":
+        U0 = np.eye(k, dtype=np.float32)
+    else:
+        pert, _ = np.linalg.qr(np.eye(k) + 1e-3 * rng.standard_normal((k, k)))
+        U0 = (Qe @ pert).astype(np.float32)
+    w = torch.zeros(k, n, device="cuda")
+    opt = br.BasisRotation([LayerSpec("W", k, n, GEOM_BI, SRC_SECOND, 0)], [w], grad_dtype="f32",
+                           gemm_prec=br.BR_GEMM_FP32, freq=1000)
+    try:
+        assert opt.step([torch.randn(k, n, device="cuda") * 0.01], 0) == br.BR_OK
+        opt.set_state(0, br.BR_BUF_L, torch.from_numpy(F))
+        opt.set_state(0, br.BR_BUF_U, torch.from_numpy(U0))
+        opt.refresh_basis(0)
+        assert opt.sync_status() == br.BR_OK
+        U = opt.get_state(0, br.BR_BUF_U).numpy().astype(np.float64)
+        ref, deficient = O.power(F.astype(np.float64), U0.astype(np.float64))
+        assert not deficient
+        assert np.max(np.abs(U.T @ U - np.eye(k))) < 1e-5
+        assert basis_err(U, ref) < 1e-5
     finally:
         opt.close()
 

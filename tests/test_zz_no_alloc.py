@@ -29,7 +29,7 @@ def test_static_scratch_power_matches_handle_path_twice():
     import paper_2602_03515_b200 as br
     from workloads import LayerSpec
     from tests.parity_util import basis_err
-    k = 200                                    # 7 panels of 32 columns, the last one ragged
+    k = 200                                    # several panels, the last one ragged
     w = torch.zeros(k, 16, device="cuda")
     opt = br.BasisRotation([LayerSpec("W", k, 16, br.BR_GEOM_BILATERAL, br.BR_SRC_SECOND, 0)], [w],
                            grad_dtype="f32", gemm_prec=br.BR_GEMM_FP32, freq=10 ** 6)

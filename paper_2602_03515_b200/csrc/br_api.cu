@@ -92,7 +92,7 @@ struct br_handle {
   // scratch of the SIMT path (one layer at a time)
   float *sG = nullptr, *sT = nullptr, *sGt = nullptr, *sMt = nullptr;
   // scratch of the refresh
-  double *rA = nullptr, *rZ = nullptr, *rWork = nullptr;
+  double *rA = nullptr, *rZ = nullptr, *rWork = nullptr, *rF = nullptr, *rQ = nullptr;
   // tensor-core path
   TcStep* tc = nullptr;
   LaunchStats stats;
@@ -151,6 +151,8 @@ void layout(br_handle* h, Bump& b, Sizes* sz) {
   }
   if (max_k) {
     h->rA = b.take<double>(max_k * max_k);
+    h->rF = b.take<double>(max_k * max_k);
+    h->rQ = b.take<double>(max_k * max_k);
     h->rWork = b.take<double>(qr_work_doubles((int64_t)max_k));
     if (max_z) h->rZ = b.take<double>(max_z);
   }
@@ -196,8 +198,11 @@ br_status refresh_side(br_handle* h, Layer& L, bool left_side) {
   for (int it = 0; it < h->hp.power_iters; ++it) {
     if (L.d.src == BR_SRC_SECOND) {
       const float* F = left_side ? L.L : L.R;
-      BR_CUDA(h, sdgemm(0, 0, k, k, k, 1.0, F, k, Q, k, 0.0, h->rA, k, s));
-      count(h); h->stats.gemm_flops += 2.0 * k * k * k;
+      // widen once, then a pure fp64 product (the products are exact either way)
+      BR_CUDA(h, f32_to_f64(F, h->rF, k * k, s));
+      BR_CUDA(h, f32_to_f64(Q, h->rQ, k * k, s));
+      BR_CUDA(h, dgemm(0, 0, k, k, k, 1.0, h->rF, k, h->rQ, k, 0.0, h->rA, k, s));
+      count(h, 3); h->stats.gemm_flops += 2.0 * k * k * k;
     } else if (left_side) {
       // (M M^T) U = M (M^T U)
       BR_CUDA(h, sdgemm(1, 0, n, m, m, 1.0, L.M, n, Q, m, 0.0, h->rZ, m, s));

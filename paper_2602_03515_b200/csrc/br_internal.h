@@ -76,6 +76,7 @@ cudaError_t split_bf16(const float* X, __nv_bfloat16* hi, __nv_bfloat16* lo, int
 cudaError_t widen_bf16(const __nv_bfloat16* X, float* out, int64_t numel, cudaStream_t s);
 // out(double) <- in(float) ; out(float) <- in(double)
 cudaError_t f64_to_f32(const double* X, float* out, int64_t numel, cudaStream_t s);
+cudaError_t f32_to_f64(const float* X, double* out, int64_t numel, cudaStream_t s);
 
 // ---------------------------------------------------------------------------------------------
 // SIMT contractions (gemm_simt.cu):  C = alpha * op(A) op(B) + beta * C, row-major.

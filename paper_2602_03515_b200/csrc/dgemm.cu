@@ -7,7 +7,8 @@
 //
 // 128 x 128 x 16 tiles, 8 warps, each warp a 32 x 64 sub-tile as 4 x 8 mma.sync.m8n8k4.f64
 // fragments (64 accumulator doubles per thread), two shared-memory stages with the next tile
-// prefetched into registers during the math.  fp32 operands are widened while they are staged,
+// prefetched into registers during the math.  Transposed operands are staged in a second
+// shared-memory layout instead of being transposed on the way.  fp32 operands are widened while they are staged,
 // so every product is exact and only the fp64 accumulation rounds.  A contraction that is long
 // and narrow (Gram matrices, panel projections) is split over K into partial sums that a second
 // kernel adds in a fixed order, which keeps the result reproducible from run to run.
@@ -18,8 +19,14 @@ namespace br {
 namespace {
 
 constexpr int BM = 128, BN = 128, BK = 16;
-constexpr int LDS = 136;                  // padded row of a staged tile (doubles): 136 = 8 mod 16
-constexpr int STAGE = 2 * BK * LDS;       // doubles per stage (A tile + B tile)
+// A staged operand tile holds 128 (i) x 16 (kk) doubles in one of two layouts, chosen so that the
+// copy from global memory needs no transposition and both the copy and the fragment loads are free
+// of bank conflicts:
+//   k-major  S[kk * 136 + i]   for an operand whose i index is contiguous in global memory
+//   i-major  S[i * 20 + kk]    for an operand whose contraction index is contiguous
+constexpr int LDK = 136, LDI = 20;
+constexpr int TILE = BM * LDI;            // doubles reserved per operand tile (>= BK * LDK)
+constexpr int STAGE = 2 * TILE;           // doubles per stage (A tile + B tile)
 constexpr int SMEM_BYTES = 2 * STAGE * (int)sizeof(double);
 
 __device__ __forceinline__ void dmma(double& c0, double& c1, double a, double b) {
@@ -34,6 +41,7 @@ template <> struct Vec2<float> { using type = float2; };
 // One operand tile of 128 (i) x 16 (kk) elements, fetched into 8 registers per thread.
 //   direct : element (kk, i) at X[(k0 + kk) * ld + i0 + i]   (contraction index is the slow one)
 //   scatter: element (i, kk) at X[(i0 + i) * ld + k0 + kk]   (contraction index is contiguous)
+// Either way 8 (float: 16) consecutive threads read one contiguous 128-byte (64-byte) run.
 // `fast` = the tile is interior and 2-element vector loads are aligned.
 template <typename T>
 __device__ __forceinline__ void tile_load(double (&r)[8], const T* __restrict__ X, int64_t ld, bool scatter,
@@ -59,41 +67,39 @@ __device__ __forceinline__ void tile_load(double (&r)[8], const T* __restrict__ 
       }
     }
   } else {
-    const int w = t >> 5, lane = t & 31;
-    const T* col = X + (i0 + lane) * ld + k0 + 2 * w;
+    const int li = t >> 3, lk = (t & 7) * 2;      // rows li + 32 q, columns k0 + lk, k0 + lk + 1
+    const T* p = X + (i0 + li) * ld + k0 + lk;
     if (fast) {
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
-        const V v = *reinterpret_cast<const V*>(col + (int64_t)32 * q * ld);
+        const V v = *reinterpret_cast<const V*>(p + (int64_t)32 * q * ld);
         r[2 * q] = (double)v.x; r[2 * q + 1] = (double)v.y;
       }
     } else {
-      const bool k0ok = (k0 + 2 * w) < Kend, k1ok = (k0 + 2 * w + 1) < Kend;
+      const bool k0ok = (k0 + lk) < Kend, k1ok = (k0 + lk + 1) < Kend;
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
-        const bool iok = (i0 + lane + 32 * q) < I;
-        r[2 * q] = (iok && k0ok) ? (double)col[(int64_t)32 * q * ld] : 0.0;
-        r[2 * q + 1] = (iok && k1ok) ? (double)col[(int64_t)32 * q * ld + 1] : 0.0;
+        const bool iok = (i0 + li + 32 * q) < I;
+        r[2 * q] = (iok && k0ok) ? (double)p[(int64_t)32 * q * ld] : 0.0;
+        r[2 * q + 1] = (iok && k1ok) ? (double)p[(int64_t)32 * q * ld + 1] : 0.0;
       }
     }
   }
 }
 
-// Registers -> staged tile S[kk][i] (row length LDS).  Both forms store without bank conflicts.
+// Registers -> staged tile (k-major for a direct operand, i-major for a scatter operand).
 __device__ __forceinline__ void tile_store(double* __restrict__ S, const double (&r)[8], bool scatter) {
   const int t = threadIdx.x;
   if (!scatter) {
     const int lk = t >> 4, li = (t & 15) * 2;
 #pragma unroll
     for (int q = 0; q < 4; ++q)
-      *reinterpret_cast<double2*>(S + lk * LDS + li + 32 * q) = make_double2(r[2 * q], r[2 * q + 1]);
+      *reinterpret_cast<double2*>(S + lk * LDK + li + 32 * q) = make_double2(r[2 * q], r[2 * q + 1]);
   } else {
-    const int w = t >> 5, lane = t & 31;
+    const int li = t >> 3, lk = (t & 7) * 2;
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      S[(2 * w) * LDS + lane + 32 * q] = r[2 * q];
-      S[(2 * w + 1) * LDS + lane + 32 * q] = r[2 * q + 1];
-    }
+    for (int q = 0; q < 4; ++q)
+      *reinterpret_cast<double2*>(S + (li + 32 * q) * LDI + lk) = make_double2(r[2 * q], r[2 * q + 1]);
   }
 }
 
@@ -125,9 +131,14 @@ k_dgemm(int ta, int tb, int64_t M, int64_t N, int64_t K, double alpha, const TA*
     tile_load<TA>(pa, A, lda, a_scatter, a_int && kfull, m0, kbeg, M, kend);
     tile_load<TB>(pb, B, ldb, b_scatter, b_int && kfull, n0, kbeg, N, kend);
     tile_store(sm, pa, a_scatter);
-    tile_store(sm + BK * LDS, pb, b_scatter);
+    tile_store(sm + TILE, pb, b_scatter);
   }
   __syncthreads();
+  // fragment addressing: element (i, kk) of a staged tile sits at i * si + kk * sk
+  const int a_si = a_scatter ? LDI : 1, a_sk = a_scatter ? 1 : LDK;
+  const int b_si = b_scatter ? LDI : 1, b_sk = b_scatter ? 1 : LDK;
+  const int a_base = (32 * wm + g) * a_si + tig * a_sk;
+  const int b_base = (64 * wn + g) * b_si + tig * b_sk;
   for (int64_t kt = 0; kt < nk; ++kt) {
     const int st = (int)(kt & 1);
     if (kt + 1 < nk) {
@@ -136,15 +147,15 @@ k_dgemm(int ta, int tb, int64_t M, int64_t N, int64_t K, double alpha, const TA*
       tile_load<TA>(pa, A, lda, a_scatter, a_int && kfull, m0, k0, M, kend);
       tile_load<TB>(pb, B, ldb, b_scatter, b_int && kfull, n0, k0, N, kend);
     }
-    const double* As = sm + st * STAGE;
-    const double* Bs = As + BK * LDS;
+    const double* As = sm + st * STAGE + a_base;
+    const double* Bs = sm + st * STAGE + TILE + b_base;
 #pragma unroll
     for (int k4 = 0; k4 < BK; k4 += 4) {
       double a[4], b[8];
 #pragma unroll
-      for (int mi = 0; mi < 4; ++mi) a[mi] = As[(k4 + tig) * LDS + 32 * wm + 8 * mi + g];
+      for (int mi = 0; mi < 4; ++mi) a[mi] = As[8 * mi * a_si + k4 * a_sk];
 #pragma unroll
-      for (int ni = 0; ni < 8; ++ni) b[ni] = Bs[(k4 + tig) * LDS + 64 * wn + 8 * ni + g];
+      for (int ni = 0; ni < 8; ++ni) b[ni] = Bs[8 * ni * b_si + k4 * b_sk];
 #pragma unroll
       for (int mi = 0; mi < 4; ++mi)
 #pragma unroll
@@ -153,7 +164,7 @@ k_dgemm(int ta, int tb, int64_t M, int64_t N, int64_t K, double alpha, const TA*
     if (kt + 1 < nk) {
       double* Sn = sm + (st ^ 1) * STAGE;
       tile_store(Sn, pa, a_scatter);
-      tile_store(Sn + BK * LDS, pb, b_scatter);
+      tile_store(Sn + TILE, pb, b_scatter);
     }
     __syncthreads();
   }

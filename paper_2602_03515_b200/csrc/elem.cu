@@ -196,6 +196,13 @@ k_widen_bf16(const __nv_bfloat16* __restrict__ X, float* __restrict__ out, int64
 }
 
 __global__ void __launch_bounds__(kThreads)
+k_f32_to_f64(const float* __restrict__ X, double* __restrict__ out, int64_t numel) {
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < numel; i += stride)
+    out[i] = (double)X[i];
+}
+
+__global__ void __launch_bounds__(kThreads)
 k_f64_to_f32(const double* __restrict__ X, float* __restrict__ out, int64_t numel) {
   const int64_t stride = (int64_t)gridDim.x * blockDim.x;
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < numel; i += stride)
@@ -244,6 +251,11 @@ cudaError_t split_bf16(const float* X, __nv_bfloat16* hi, __nv_bfloat16* lo, int
 
 cudaError_t widen_bf16(const __nv_bfloat16* X, float* out, int64_t numel, cudaStream_t s) {
   k_widen_bf16<<<grid_for((numel + 3) / 4), kThreads, 0, s>>>(X, out, numel);
+  return cudaGetLastError();
+}
+
+cudaError_t f32_to_f64(const float* X, double* out, int64_t numel, cudaStream_t s) {
+  k_f32_to_f64<<<grid_for(numel), kThreads, 0, s>>>(X, out, numel);
   return cudaGetLastError();
 }
 

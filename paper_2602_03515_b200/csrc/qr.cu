@@ -1,16 +1,27 @@
 // QR orthonormalisation for Power(A, Q) = qr(A Q).Q (Sec. 3.2 of the paper), fp64, in place.
 //
 // The factorisation wanted is the unique one with a positive diagonal of R.  It is computed by
-// a right-looking block Gram-Schmidt whose floating-point work is almost entirely fp64 matrix
-// products (dgemm.cu): for each panel P of up to 128 columns
-//   1. orthonormalise the panel by Cholesky-QR: Gram matrix S = P^T P (split over the rows),
-//      Cholesky factor S = R^T R and its inverse in one CTA, P <- P R^-1.  The Cholesky factor
-//      has a positive diagonal, so the signs come out as required.  The step is repeated once
-//      unless the first Cholesky factorisation showed the panel to be nearly orthogonal already
-//      (see k_chol_inverse), which is the usual case once the basis tracks the factor;
-//   2. project the panel out of all trailing columns: C = P^T A_trail, A_trail -= P C.
-// In fp64 the loss of orthogonality of this scheme is ~ cond * 1e-16, far below the fp32
-// rounding of the stored bases, and the result agrees with Householder QR to the same level.
+// a recursive block Gram-Schmidt whose floating-point work is almost entirely large fp64 matrix
+// products (dgemm.cu):
+//   orth(columns):  if the block is at most one panel (128 columns) wide, orthonormalise it by
+//                   Cholesky-QR; otherwise orth(left half), project the left half out of the right
+//                   half (C = Q_l^T A_r, A_r -= Q_l C), orth(right half).
+//   Cholesky-QR of a panel P: Gram matrix S = P^T P (split over the rows), Cholesky factor
+//   S = R^T R and its inverse in one CTA, P <- P R^-1.  The Cholesky factor has a positive
+//   diagonal, so the signs come out as required.  The step is repeated once unless the first
+//   factorisation showed the panel to be nearly orthogonal already (see k_chol_inverse).
+// Half of the floating-point work is in the two products of the top level and three quarters in
+// the top two, which is what lets the matrix unit run close to its peak.
+//
+// A block projection takes all its coefficients from the same right-hand side (as classical
+// Gram-Schmidt does), so one sweep loses orthogonality like cond^2 * 1e-16, with cond the condition
+// number of the column-scaled input.  Once the basis tracks the factor the columns of A Q are
+// nearly orthogonal and one sweep is accurate to rounding.  The first refresh of a low-rank-plus-
+// noise factor is different (cond ~ 1e5): there the whole orthonormalisation is run a second time
+// on its own output ("twice is enough"), which restores orthogonality to the rounding level.  The
+// second sweep is decided on the device: the first sweep compares the squared norm each column has
+// left when its panel is reached with the squared norm it started with, and clears a flag when the
+// ratio falls below 1e-4; every launch of the second sweep returns at once while the flag is set.
 // All reductions are done in a fixed order, so the result is bit-reproducible from run to run.
 #include <algorithm>
 
@@ -25,169 +36,266 @@ constexpr double kDefectLimit = 0.1;
 inline int64_t cdiv(int64_t a, int64_t b) { return (a + b - 1) / b; }
 inline int panel_width(int64_t k) { return k >= 1024 ? 128 : 64; }
 inline int gram_splits(int64_t k) { return (int)std::min<int64_t>(64, std::max<int64_t>(1, cdiv(k, 128))); }
-inline int proj_splits_max(int64_t k) { return k >= 1024 ? 8 : 2; }
+inline int proj_splits_max(int64_t k) { return k >= 1024 ? 64 : 1; }
+constexpr double kIllRatio = 1e-4;   // squared-norm ratio below which the second sweep runs
 // sub-buffers of the work area start on 256-byte boundaries
 inline int64_t pad32(int64_t doubles) { return (doubles + 31) / 32 * 32; }
 
 // Cholesky factorisation S = R^T R of a bw x bw Gram matrix (bw <= 128) and R^-1, in one CTA.
 //
-// The matrix lives in registers: thread (ty, tx) of the 16 x 16 grid owns rows ty + 16 a and
-// columns tx + 16 b (a, b < 8), a cyclic distribution that keeps every thread busy while the
-// elimination shrinks the active part.  Step c scales row c by 1 / R_cc, shares it through shared
-// memory and subtracts R_ci times it from every row i > c.  The same row operations applied to the
-// identity give R^-T; because column j of the Gram matrix is dead once step j is done and column j
-// of R^-T is still a unit vector until then, both share one register array: entry (i, j) holds the
-// Gram entry while j > c and the entry of R^-T afterwards.
+// The matrix lives in registers: thread (ty, tx) of the 32 x 16 grid owns rows ty + 32 a (a < 4)
+// and columns tx + 16 b (b < 8), a cyclic distribution that keeps every thread busy while the
+// elimination shrinks the active part.  Row c reaches the other threads through shared memory,
+// posted by its owners at the end of step c - 1; in step c every thread derives 1 / R_cc from it
+// (redundantly, so no thread waits for another inside a step), scales the row and subtracts R_ci
+// times it from each of its rows i > c.  The same row operations applied to the identity give
+// R^-T; because column j of the Gram matrix is dead once step j is done and column j of R^-T is
+// still a unit vector until then, both share one register array: entry (i, j) holds the Gram
+// entry while j > c and the entry of R^-T afterwards.  Row c of R^-T is final after step c and is
+// written out (as column c of R^-1) straight from the scaled row.
 //
 // A pivot that underflows 1e-24 of the column's squared norm is clamped and reported as a
 // numerically rank-deficient factor.  defect = sum_c (1 - pivot_c / S_cc) bounds the squared
 // Frobenius distance of the column-scaled Gram matrix from the identity (up to a factor ~2): when
 // it is small the panel was close to orthogonal and one Cholesky-QR pass is accurate to rounding,
-// so *skip_next is set and the kernels of the second pass return at once.
-__global__ void __launch_bounds__(256)
+// so *skip_next is set and the kernels of the second pass return at once.  norm0 (optional):
+// squared norms the panel's columns had before any projection; a column that has lost more than
+// 1 - kIllRatio of it marks the input as ill-conditioned by clearing *ill_clear.
+__global__ void __launch_bounds__(512)
 k_chol_inverse(const double* __restrict__ S, int bw, double* __restrict__ Rinv, int* __restrict__ status,
-               int* __restrict__ skip_next, const int* __restrict__ skip_self) {
-  if (skip_self && *skip_self) return;
-  __shared__ double rowZ[2][kB];
-  __shared__ double defect_sm;
-  const int t = threadIdx.x, ty = t >> 4, tx = t & 15, lane = t & 31;
-  double Z[8][8];
-  double d0[8];
+               int* __restrict__ skip_next, const int* __restrict__ skip_self,
+               const double* __restrict__ norm0, int* __restrict__ ill_clear) {
+  if (skip_self && *skip_self) {
+    if (skip_next && threadIdx.x == 0) *skip_next = 1;
+    return;
+  }
+  __shared__ double rowS[2][kB];
+  __shared__ double diag0[kB], diag0_inv[kB], nrm_floor[kB];
+  const int t = threadIdx.x, ty = t >> 4, tx = t & 15;
+  if (t < kB) nrm_floor[t] = (norm0 && t < bw) ? kIllRatio * norm0[t] : 0.0;
+  double Z[4][8];
 #pragma unroll
-  for (int a = 0; a < 8; ++a) {
-    const int i = ty + 16 * a;
+  for (int a = 0; a < 4; ++a) {
+    const int i = ty + 32 * a;
 #pragma unroll
     for (int b = 0; b < 8; ++b) {
       const int j = tx + 16 * b;
-      Z[a][b] = (i < bw && j < bw) ? S[(int64_t)i * bw + j] : (i == j ? 1.0 : 0.0);
+      const double v = (i < bw && j < bw) ? S[(int64_t)i * bw + j] : (i == j ? 1.0 : 0.0);
+      Z[a][b] = v;
+      if (i == j) { diag0[i] = v; diag0_inv[i] = v > 0.0 ? 1.0 / v : 0.0; }
     }
-    d0[a] = Z[a][a];        // meaningful on the diagonal threads (ty == tx) only
   }
-  if (t == 0) defect_sm = 0.0;
+  if (ty == 0) {
+#pragma unroll
+    for (int b = 0; b < 8; ++b) rowS[0][tx + 16 * b] = Z[0][b];
+  }
   __syncthreads();
+  double defect = 0.0;       // accumulated by thread 0 (every thread sees every pivot)
+  bool ill = false;
 
   for (int c = 0; c < bw; ++c) {
-    const int buf = c & 1, ca = c >> 4, cr = c & 15;
-    if (ty == cr) {
-      // the 16 owners of row c are one half of a warp
-      double zr[8];
+    const int buf = c & 1;
+    const double orig = diag0[c];
+    double piv = rowS[buf][c];
+    double floor_ = orig * 1e-24;
+    if (!(floor_ > 1e-300)) floor_ = 1e-300;
+    const bool clamped = !(piv > floor_);
+    if (clamped) piv = floor_;
+    if (t == 0) {
+      if (clamped) atomicMax(status, (int)BR_WARN_RANK_DEFICIENT);
+      defect += fmax(0.0, 1.0 - piv * diag0_inv[c]);
+      if (orig < nrm_floor[c]) ill = true;
+    }
+    const double inv_d = rsqrt(piv);
+    double rj[8];
 #pragma unroll
-      for (int a = 0; a < 8; ++a)
-        if (a == ca) {
-#pragma unroll
-          for (int b = 0; b < 8; ++b) zr[b] = Z[a][b];
-        }
-      double piv = 0.0;
-      if (tx == cr) {
-        double orig = 0.0;
-#pragma unroll
-        for (int b = 0; b < 8; ++b)
-          if (b == ca) { piv = zr[b]; orig = d0[b]; }
-        double floor_ = orig * 1e-24;
-        if (!(floor_ > 1e-300)) floor_ = 1e-300;
-        if (!(piv > floor_)) {
-          piv = floor_;
-          atomicMax(status, (int)BR_WARN_RANK_DEFICIENT);
-        }
-        defect_sm += (orig > 0.0) ? fmax(0.0, 1.0 - piv / orig) : 1.0;
-      }
-      const unsigned half = (lane < 16) ? 0x0000FFFFu : 0xFFFF0000u;
-      piv = __shfl_sync(half, piv, (lane & 16) | cr);
-      const double inv_d = 1.0 / sqrt(piv);
+    for (int b = 0; b < 8; ++b) {
+      const int j = tx + 16 * b;
+      rj[b] = (j == c) ? inv_d : rowS[buf][j] * inv_d;
+    }
+    // row c of R^-T is final: column c of R^-1 (zero below the diagonal)
+    if (ty == 0) {
 #pragma unroll
       for (int b = 0; b < 8; ++b) {
         const int j = tx + 16 * b;
-        const double v = (j == c) ? inv_d : zr[b] * inv_d;
-        zr[b] = v;
-        rowZ[buf][j] = v;
+        if (j < bw) Rinv[(int64_t)j * bw + c] = (j <= c) ? rj[b] : 0.0;
       }
+    }
+    double f[4];
 #pragma unroll
-      for (int a = 0; a < 8; ++a)
-        if (a == ca) {
+    for (int a = 0; a < 4; ++a) {
+      const int i = ty + 32 * a;
+      f[a] = (i > c) ? rowS[buf][i] * inv_d : 0.0;   // R_ci (row c of R, by symmetry); 0 leaves dead rows alone
 #pragma unroll
-          for (int b = 0; b < 8; ++b) Z[a][b] = zr[b];
-        }
+      for (int b = 0; b < 8; ++b) Z[a][b] = fma(-f[a], rj[b], Z[a][b]);
+    }
+    // column c turns from a Gram column into a column of R^-T: entry (i, c) = -R_ci / R_cc
+    if (tx == (c & 15)) {
+      switch (c >> 4) {
+#define BR_FIX(B)                                                          \
+  case B:                                                                  \
+    _Pragma("unroll") for (int a = 0; a < 4; ++a) Z[a][B] = -f[a] * inv_d; \
+    break;
+        BR_FIX(0) BR_FIX(1) BR_FIX(2) BR_FIX(3) BR_FIX(4) BR_FIX(5) BR_FIX(6) BR_FIX(7)
+#undef BR_FIX
+      }
+    }
+    // post row c + 1 for the next step
+    if (ty == ((c + 1) & 31)) {
+      switch ((c + 1) >> 5) {
+#define BR_POST(A)                                                                          \
+  case A:                                                                                   \
+    _Pragma("unroll") for (int b = 0; b < 8; ++b) rowS[buf ^ 1][tx + 16 * b] = Z[A][b];     \
+    break;
+        BR_POST(0) BR_POST(1) BR_POST(2) BR_POST(3)
+#undef BR_POST
+      }
     }
     __syncthreads();
-    double rj[8];
-#pragma unroll
-    for (int b = 0; b < 8; ++b) rj[b] = rowZ[buf][tx + 16 * b];
-#pragma unroll
-    for (int a = 0; a < 8; ++a) {
-      const int i = ty + 16 * a;
-      if (i > c) {
-        const double f = rowZ[buf][i];        // R_ci (row c of R, by symmetry of the Gram matrix)
-#pragma unroll
-        for (int b = 0; b < 8; ++b) {
-          const double old = (tx + 16 * b == c) ? 0.0 : Z[a][b];
-          Z[a][b] = fma(-f, rj[b], old);
-        }
-      }
-    }
   }
-  __syncthreads();
-  if (t == 0 && skip_next) *skip_next = (defect_sm <= kDefectLimit) ? 1 : 0;
-  // Z holds R^-T in its lower triangle: R^-1 (i, j) = Z (j, i)
-#pragma unroll
-  for (int a = 0; a < 8; ++a) {
-    const int i = ty + 16 * a;
-#pragma unroll
-    for (int b = 0; b < 8; ++b) {
-      const int j = tx + 16 * b;
-      if (i < bw && j < bw) Rinv[(int64_t)j * bw + i] = (j <= i) ? Z[a][b] : 0.0;
-    }
+  if (t == 0) {
+    if (skip_next) *skip_next = (defect <= kDefectLimit) ? 1 : 0;
+    if (ill && ill_clear) *ill_clear = 0;
   }
+}
+
+// part[z][j] = sum over the row chunk z of A[i][j]^2 (rows in order)
+constexpr int kNormChunks = 32;
+__global__ void __launch_bounds__(256)
+k_column_norms_partial(const double* __restrict__ A, int64_t k, int64_t rows_per_chunk, double* __restrict__ part) {
+  const int64_t j = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  if (j >= k) return;
+  const int64_t r0 = (int64_t)blockIdx.y * rows_per_chunk;
+  const int64_t r1 = (r0 + rows_per_chunk < k) ? r0 + rows_per_chunk : k;
+  double s0 = 0.0, s1 = 0.0;
+  int64_t i = r0;
+  for (; i + 1 < r1; i += 2) {
+    const double a0 = A[i * k + j], a1 = A[(i + 1) * k + j];
+    s0 = fma(a0, a0, s0); s1 = fma(a1, a1, s1);
+  }
+  if (i < r1) { const double a0 = A[i * k + j]; s0 = fma(a0, a0, s0); }
+  part[(int64_t)blockIdx.y * k + j] = s0 + s1;
+}
+// norm0[j] = sum_z part[z][j] in chunk order; *flag = 1
+__global__ void __launch_bounds__(256)
+k_column_norms_sum(const double* __restrict__ part, int64_t k, int nchunks, double* __restrict__ norm0,
+                   int* __restrict__ flag) {
+  const int64_t j = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  if (j == 0) *flag = 1;
+  if (j >= k) return;
+  double s = 0.0;
+  for (int z = 0; z < nchunks; ++z) s += part[(int64_t)z * k + j];
+  norm0[j] = s;
+}
+
+struct Sweep {
+  double* A; int64_t k; int b, sg, sp_max;
+  double *gram_part, *S, *Rinv, *norm0, *C, *proj_part;
+  int *skip2, *sweep2_skip;
+  int* status;
+  cudaStream_t s;
+  const int* skip;        // non-null: every launch of this sweep returns while *skip != 0
+  bool first;             // first sweep: watch the column norms
+  int64_t launches = 0;
+  double flops = 0.0;
+  cudaError_t err = cudaSuccess;
+};
+
+// Cholesky-QR (at most twice) of the panel of columns [j0, j0 + bw).
+void leaf(Sweep& q, int64_t j0, int bw) {
+  double* P = q.A + j0;
+  const int64_t k = q.k;
+  for (int pass = 0; pass < 2 && q.err == cudaSuccess; ++pass) {
+    const int* skip = pass ? q.skip2 : q.skip;
+    cudaError_t e = dgemm_ex(1, 0, bw, bw, k, 1.0, P, k, P, k, 0.0, q.S, bw, q.sg, q.gram_part, skip, q.s);
+    if (e != cudaSuccess) { q.err = e; return; }
+    k_chol_inverse<<<1, 512, 0, q.s>>>(q.S, bw, q.Rinv, q.status, pass ? nullptr : q.skip2, skip,
+                                       (q.first && !pass) ? q.norm0 + j0 : nullptr, q.sweep2_skip);
+    // P <- P R^-1 (in place: a CTA reads only the rows it writes, and writes after its last read)
+    e = dgemm_ex(0, 0, k, bw, bw, 1.0, P, k, q.Rinv, bw, 0.0, P, k, 1, nullptr, skip, q.s);
+    if (e != cudaSuccess) { q.err = e; return; }
+    q.launches += 3 + (q.sg > 1 ? 1 : 0);
+    if (q.first && !pass) q.flops += 4.0 * (double)k * bw * bw;
+  }
+}
+
+// A[:, jt : jt + wt] -= Q (Q^T A[:, jt : jt + wt]) with Q = A[:, jp : jp + wp] orthonormal.
+void project(Sweep& q, int64_t jp, int64_t wp, int64_t jt, int64_t wt) {
+  if (q.err != cudaSuccess) return;
+  const int64_t k = q.k;
+  const int64_t tiles = cdiv(wp, 128) * cdiv(wt, 128);
+  int sp = 1;
+  if (tiles < 148) sp = (int)std::max<int64_t>(1, std::min<int64_t>(std::min<int64_t>(cdiv(296, tiles), q.sp_max), k / 128));
+  cudaError_t e = dgemm_ex(1, 0, wp, wt, k, 1.0, q.A + jp, k, q.A + jt, k, 0.0, q.C, wt, sp, q.proj_part, q.skip, q.s);
+  if (e == cudaSuccess)
+    e = dgemm_ex(0, 0, k, wt, wp, -1.0, q.A + jp, k, q.C, wt, 1.0, q.A + jt, k, 1, nullptr, q.skip, q.s);
+  if (e != cudaSuccess) { q.err = e; return; }
+  q.launches += 2 + (sp > 1 ? 1 : 0);
+  if (q.first) q.flops += 4.0 * (double)k * wp * wt;
+}
+
+void orth(Sweep& q, int64_t j0, int64_t w) {
+  if (q.err != cudaSuccess) return;
+  if (w <= q.b) { leaf(q, j0, (int)w); return; }
+  const int64_t h = cdiv(w, 2 * q.b) * q.b;     // left part: a whole number of panels
+  orth(q, j0, h);
+  project(q, j0, h, j0 + h, w - h);
+  orth(q, j0 + h, w - h);
+}
+
+inline int64_t proj_part_doubles(int64_t k) {
+  const int sp = proj_splits_max(k);
+  if (sp <= 1) return 0;
+  // a projection is split only while it has fewer than 148 tiles of 128 x 128
+  return std::min<int64_t>((int64_t)sp * ((k + 1) / 2) * ((k + 1) / 2), (int64_t)(296 + 148) * 128 * 128);
 }
 
 }  // namespace
 
 size_t qr_work_doubles(int64_t k) {
   const int64_t b = std::min<int64_t>(panel_width(k), k);
-  return (size_t)(pad32((int64_t)gram_splits(k) * b * b) + 2 * pad32(b * b) + 64 +
-                  pad32((int64_t)proj_splits_max(k) * b * k) + pad32(b * k));
+  return (size_t)(pad32((int64_t)gram_splits(k) * b * b) + 2 * pad32(b * b) + 64 + pad32(k) +
+                  pad32(((k + 1) / 2) * ((k + 1) / 2)) + pad32(proj_part_doubles(k)));
 }
 
 cudaError_t qr_pos_inplace(double* A, int64_t k, double* work, int* status, cudaStream_t s,
                            int64_t* launches, double* flops) {
-  const int64_t b = std::min<int64_t>(panel_width(k), k);
-  const int sg = gram_splits(k);
-  double* gram_part = work;
-  double* S = gram_part + pad32((int64_t)sg * b * b);
-  double* Rinv = S + pad32(b * b);
-  int* skip2 = reinterpret_cast<int*>(Rinv + pad32(b * b));      // 64 doubles reserved for flags
-  double* proj_part = Rinv + pad32(b * b) + 64;
-  double* C = proj_part + pad32((int64_t)proj_splits_max(k) * b * k);
-  int64_t nl = 0;
-  double fl = 0.0;
-  cudaError_t e = cudaSuccess;
-  for (int64_t j0 = 0; j0 < k; j0 += b) {
-    const int bw = (int)std::min<int64_t>(b, k - j0);
-    double* P = A + j0;
-    for (int pass = 0; pass < 2; ++pass) {
-      const int* skip = pass ? skip2 : nullptr;
-      // S = P^T P
-      if ((e = dgemm_ex(1, 0, bw, bw, k, 1.0, P, k, P, k, 0.0, S, bw, sg, gram_part, skip, s)) != cudaSuccess) return e;
-      k_chol_inverse<<<1, 256, 0, s>>>(S, bw, Rinv, status, pass ? nullptr : skip2, skip);
-      // P <- P R^-1 (in place: a CTA reads only the rows it writes, and writes after its last read)
-      if ((e = dgemm_ex(0, 0, k, bw, bw, 1.0, P, k, Rinv, bw, 0.0, P, k, 1, nullptr, skip, s)) != cudaSuccess) return e;
-      nl += 3 + (sg > 1 ? 1 : 0);
-      fl += 4.0 * (double)k * bw * bw;
-    }
-    const int64_t jt0 = j0 + bw, ntrail = k - jt0;
-    if (ntrail > 0) {
-      int sp = (int)cdiv(296, cdiv(ntrail, 128));
-      sp = std::max(1, std::min(sp, std::min(proj_splits_max(k), (int)std::max<int64_t>(1, k / 256))));
-      // C = P^T A_trail ; A_trail -= P C
-      if ((e = dgemm_ex(1, 0, bw, ntrail, k, 1.0, P, k, A + jt0, k, 0.0, C, ntrail, sp, proj_part, nullptr, s)) != cudaSuccess) return e;
-      if ((e = dgemm_ex(0, 0, k, ntrail, bw, -1.0, P, k, C, ntrail, 1.0, A + jt0, k, 1, nullptr, nullptr, s)) != cudaSuccess) return e;
-      nl += 2 + (sp > 1 ? 1 : 0);
-      fl += 4.0 * (double)k * bw * ntrail;
-    }
-    e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
+  Sweep q;
+  q.A = A; q.k = k; q.s = s; q.status = status;
+  q.b = (int)std::min<int64_t>(panel_width(k), k);
+  q.sg = gram_splits(k);
+  q.sp_max = proj_splits_max(k);
+  const int64_t b = q.b;
+  q.gram_part = work;
+  q.S = q.gram_part + pad32((int64_t)q.sg * b * b);
+  q.Rinv = q.S + pad32(b * b);
+  int* flags = reinterpret_cast<int*>(q.Rinv + pad32(b * b));      // 64 doubles reserved for flags
+  q.skip2 = flags;
+  q.sweep2_skip = flags + 1;
+  q.norm0 = q.Rinv + pad32(b * b) + 64;
+  q.C = q.norm0 + pad32(k);
+  q.proj_part = q.C + pad32(((k + 1) / 2) * ((k + 1) / 2));
+  // first sweep, watching how much of its norm each column keeps
+  {
+    // the partial sums borrow the (still unused) projection buffer: kNormChunks * k <= (k + 1)^2 / 4 for k >= 128
+    const int nchunks = (int)std::min<int64_t>(kNormChunks, std::max<int64_t>(1, k / 4));
+    const int64_t rows_per_chunk = cdiv(k, nchunks);
+    const int used = (int)cdiv(k, rows_per_chunk);
+    dim3 grid((unsigned)cdiv(k, 256), (unsigned)used);
+    k_column_norms_partial<<<grid, 256, 0, s>>>(A, k, rows_per_chunk, q.C);
+    k_column_norms_sum<<<(unsigned)cdiv(k, 256), 256, 0, s>>>(q.C, k, used, q.norm0, q.sweep2_skip);
   }
-  if (launches) *launches += nl;
-  if (flops) *flops += fl;
+  q.skip = nullptr; q.first = true;
+  orth(q, 0, k);
+  if (q.err != cudaSuccess) return q.err;
+  // second sweep, cancelled on the device unless the first one met an ill-conditioned input
+  q.skip = q.sweep2_skip; q.first = false;
+  orth(q, 0, k);
+  if (q.err != cudaSuccess) return q.err;
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  if (launches) *launches += q.launches + 2;
+  if (flops) *flops += q.flops;
   return cudaSuccess;
 }
 

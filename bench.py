@@ -97,29 +97,44 @@ class ClockSampler:
 
 
 # ---------------------------------------------------------------------------------------------
-def device_gradients(w, device, torch):
-    """One synthetic gradient per layer, generated on the device with the value structure of the
-    workload (throughput runs only; parity runs use the CPU streams of workloads.gradients)."""
-    grads = []
-    for i, l in enumerate(w.layers):
-        g = torch.Generator(device=device)
-        g.manual_seed(1000003 * (w.seed + 1) + i)
+class DeviceGradients:
+    """Synthetic gradients generated on the device with the value structure of the workload
+    (throughput runs only; parity runs use the CPU streams of workloads.gradients).  The signal
+    factors of a low-rank-plus-noise layer are drawn once, the noise is drawn afresh by every call of
+    `fresh()`, as the workload prescribes: the factor EMAs then have full rank and the basis refresh
+    sees the conditioning of a real stream (a refresh takes device-side decisions that depend on it)."""
+
+    def __init__(self, w, device, torch):
+        self.w, self.device, self.torch = w, device, torch
+        self.gen = torch.Generator(device=device)
+        self.gen.manual_seed(1000003 * (w.seed + 1))
+        self.factors = []
+        dt = torch.bfloat16 if w.grad_dtype == "bf16" else torch.float32
+        self.grads = [torch.empty(l.m, l.n, device=device, dtype=dt) for l in w.layers]
         if w.grad_kind == "lowrank_noise":
-            A = torch.randn(l.m, w.grad_rank, device=device, generator=g)
-            B = torch.randn(l.n, w.grad_rank, device=device, generator=g)
-            x = A @ B.t()
-            x.add_(torch.randn(l.m, l.n, device=device, generator=g), alpha=w.grad_scale)
-        elif w.grad_kind == "student_t":
-            z = torch.randn(l.m, l.n, device=device, generator=g)
-            c = torch.zeros(l.m, l.n, device=device)
-            for _ in range(3):
-                c.addcmul_(*(2 * [torch.randn(l.m, l.n, device=device, generator=g)]))
-            x = z.div_(c.div_(3.0).sqrt_()).mul_(w.grad_scale)
-        else:
-            x = torch.randn(l.m, l.n, device=device, generator=g).mul_(w.grad_scale)
-        grads.append(x.to(torch.bfloat16) if w.grad_dtype == "bf16" else x)
-        del x
-    return grads
+            for l in w.layers:
+                self.factors.append((torch.randn(l.m, w.grad_rank, device=device, generator=self.gen),
+                                     torch.randn(l.n, w.grad_rank, device=device, generator=self.gen)))
+        self.fresh()
+
+    def fresh(self):
+        torch, w = self.torch, self.w
+        for i, l in enumerate(w.layers):
+            if w.grad_kind == "lowrank_noise":
+                A, B = self.factors[i]
+                x = torch.randn(l.m, l.n, device=self.device, generator=self.gen).mul_(w.grad_scale)
+                x.addmm_(A, B.t())
+            elif w.grad_kind == "student_t":
+                z = torch.randn(l.m, l.n, device=self.device, generator=self.gen)
+                c = torch.zeros(l.m, l.n, device=self.device)
+                for _ in range(3):
+                    c.addcmul_(*(2 * [torch.randn(l.m, l.n, device=self.device, generator=self.gen)]))
+                x = z.div_(c.div_(3.0).sqrt_()).mul_(w.grad_scale)
+            else:
+                x = torch.randn(l.m, l.n, device=self.device, generator=self.gen).mul_(w.grad_scale)
+            self.grads[i].copy_(x)
+            del x
+        return self.grads
 
 
 def fit_tau(w_name, n_layers, tau_req, gemm_prec, free_bytes, margin, br):
@@ -256,8 +271,10 @@ def main():
     n_params = w.n_params
 
     weights = [torch.empty(l.m, l.n, device=dev).normal_(0.0, 0.02) for l in w.layers]
-    grads = device_gradients(w, dev, torch)
     stream = torch.cuda.Stream(device=dev)
+    with torch.cuda.stream(stream):
+        gen = DeviceGradients(w, dev, torch)
+    grads = gen.grads
     opt = br.BasisRotation.from_workload(w, weights, stream=stream,
                                          scratch_limit_bytes=int(args.scratch_gib * 2 ** 30))
     if state_bytes is None:
@@ -272,44 +289,49 @@ def main():
     with torch.cuda.stream(stream):
         # ---- priming (untimed): fill the ring, apply one update, refresh every basis once -------
         for _ in range(tau + 1):
-            opt.step(grads, tau)
+            opt.step(gen.fresh(), tau)
         if not args.no_refresh:
             opt.refresh_basis(-1)
         assert opt.sync_status() >= 0
         for _ in range(args.warmup):
-            opt.step(grads, tau)
+            opt.step(gen.fresh(), tau)
         sync_all()
 
         # ---- timed region: exactly K steps, events on the launching stream -----------------------
         l0, _ = opt.launch_stats()
         sampler = ClockSampler(local)
-        evs = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+        # (the gradients of a step are drawn before its first event: generating inputs is not timed)
+        ev0 = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+        ev1 = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
         is_refresh = []
-        evs[0].record(stream)
         for k in range(args.steps):
+            gen.fresh()
+            ev0[k].record(stream)
             opt.step(grads, tau)
+            ev1[k].record(stream)
             is_refresh.append(opt.counters(0)["t"] % w.freq == 0)     # every layer shares tau and freq here
-            evs[k + 1].record(stream)
         sync_all()
         clocks = sampler.stop()
         l1, _ = opt.launch_stats()
-        step_ms = [evs[k].elapsed_time(evs[k + 1]) for k in range(args.steps)]
-        total_ms = evs[0].elapsed_time(evs[-1])
+        step_ms = [ev0[k].elapsed_time(ev1[k]) for k in range(args.steps)]
+        total_ms = sum(step_ms)
 
         # ---- one full refresh (every layer), timed on its own --------------------------------------
         r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        sampler_r = ClockSampler(local)
         r0.record(stream)
         if not args.no_refresh:
             opt.refresh_basis(-1)
         r1.record(stream)
         sync_all()
+        clocks_refresh = sampler_r.stop()
         refresh_ms = r0.elapsed_time(r1)
 
         # ---- per-kernel device time (separate, profiled steps) -------------------------------------
         opt.profile(True)
         prof_steps = 2
         for _ in range(prof_steps):
-            opt.step(grads, tau)
+            opt.step(gen.fresh(), tau)
         opt.profile(False)
         prof = opt.get_profile()
         assert opt.sync_status() >= 0
@@ -394,8 +416,8 @@ def main():
             "config": {"workload": w.name, "layers": len(w.layers), "params": n_params, "geometry": "bilateral+unilateral embedding" if args.workload in ("c4", "c5") else "see workloads/configs.py",
                        "tau": tau, "tau_requested": tau_req, "freq": w.freq, "grad_dtype": w.grad_dtype, "state_bytes": state_bytes,
                        "l2": "inputs larger than L2 (no flush needed)" if n_params * 2 > (126 << 20) else "inputs smaller than L2",
-                       "replicas": world, "refresh_skipped_not_a_bench_value": bool(args.no_refresh), "gradients": "one device-resident synthetic gradient set reused every step"},
-            "clocks": clocks, "e2e": e2e, "gpu_launches": int(l1 - l0),
+                       "replicas": world, "refresh_skipped_not_a_bench_value": bool(args.no_refresh), "gradients": "device-generated; signal factors fixed per layer, noise drawn afresh before every step (untimed)"},
+            "clocks": clocks, "clocks_during_refresh": clocks_refresh, "e2e": e2e, "gpu_launches": int(l1 - l0),
             "roofline": roofline, "roofline_elementwise": roofline_elem, "cpu_baseline": cpu,
             "algorithmic_flops_per_step": alg_flops,
         }

@@ -5,6 +5,7 @@
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <string>
 #include <vector>
@@ -91,8 +92,20 @@ struct br_handle {
   int* d_status = nullptr;
   // scratch of the SIMT path (one layer at a time)
   float *sG = nullptr, *sT = nullptr, *sGt = nullptr, *sMt = nullptr;
-  // scratch of the refresh
-  double *rA = nullptr, *rZ = nullptr, *rWork = nullptr, *rF = nullptr, *rQ = nullptr;
+  // The refresh runs independent Power() applications (one per layer and side) on a few lanes at
+  // once: lane 0 is the handle's own stream, the others are internal streams that wait for the
+  // handle's stream before they start and that the handle's stream waits for when they are done.
+  // The orthonormalisation is a chain of short dependent launches between large products; with
+  // several chains in flight the short ones fill the gaps of the others.
+  struct Lane {
+    cudaStream_t stream = nullptr;
+    cudaEvent_t done = nullptr;
+    double *rA = nullptr, *rF = nullptr, *rQ = nullptr, *rZ = nullptr, *rWork = nullptr;
+  };
+  static constexpr int kMaxLanes = 3;
+  Lane lanes[kMaxLanes];
+  int n_lanes = 1;
+  cudaEvent_t ev_begin = nullptr;
   // tensor-core path
   TcStep* tc = nullptr;
   LaunchStats stats;
@@ -114,7 +127,7 @@ struct Bump {
 // Lays out every buffer of the handle in one slab.  With base == nullptr only sizes are computed.
 void layout(br_handle* h, Bump& b, Sizes* sz) {
   const br_hparams& hp = h->hp;
-  size_t max_numel = 0, max_k = 0, max_z = 0;
+  size_t max_numel = 0, max_k = 0, max_z = 0, n_sides = 0;
   bool any_simt = false;
   for (Layer& L : h->layers) {
     const size_t mn = (size_t)L.d.m * L.d.n;
@@ -138,8 +151,8 @@ void layout(br_handle* h, Bump& b, Sizes* sz) {
     }
     if (L.d.geom != BR_GEOM_NONE) {
       if (!L.use_tc) { any_simt = true; max_numel = std::max(max_numel, mn); }
-      if (L.left) max_k = std::max(max_k, (size_t)L.d.m);
-      if (L.right) max_k = std::max(max_k, (size_t)L.d.n);
+      if (L.left) { max_k = std::max(max_k, (size_t)L.d.m); ++n_sides; }
+      if (L.right) { max_k = std::max(max_k, (size_t)L.d.n); ++n_sides; }
       if (!second) max_z = std::max(max_z, mn);
     }
   }
@@ -150,11 +163,20 @@ void layout(br_handle* h, Bump& b, Sizes* sz) {
     h->sMt = b.take<float>(max_numel);
   }
   if (max_k) {
-    h->rA = b.take<double>(max_k * max_k);
-    h->rF = b.take<double>(max_k * max_k);
-    h->rQ = b.take<double>(max_k * max_k);
-    h->rWork = b.take<double>(qr_work_doubles((int64_t)max_k));
-    if (max_z) h->rZ = b.take<double>(max_z);
+    h->n_lanes = (int)std::min<size_t>(br_handle::kMaxLanes, std::max<size_t>(1, n_sides));
+    // tuning aid: BR_REFRESH_LANES=1..3 caps the number of concurrent refresh lanes
+    if (const char* env = std::getenv("BR_REFRESH_LANES")) {
+      const int v = std::atoi(env);
+      if (v >= 1 && v < h->n_lanes) h->n_lanes = v;
+    }
+    for (int i = 0; i < h->n_lanes; ++i) {
+      br_handle::Lane& ln = h->lanes[i];
+      ln.rA = b.take<double>(max_k * max_k);
+      ln.rF = b.take<double>(max_k * max_k);
+      ln.rQ = b.take<double>(max_k * max_k);
+      ln.rWork = b.take<double>(qr_work_doubles((int64_t)max_k));
+      if (max_z) ln.rZ = b.take<double>(max_z);
+    }
   }
   h->d_status = b.take<int>(64);
   (void)hp;
@@ -190,8 +212,8 @@ const void* ring_slot_ptr(const Layer& L, int64_t slot) {
 }
 
 // ---- refresh of one side: Q <- qr(F Q).Q in fp64, F = L | R (S=2nd) or M M^T | M^T M (S=1st) ----
-br_status refresh_side(br_handle* h, Layer& L, bool left_side) {
-  cudaStream_t s = h->stream;
+br_status refresh_side(br_handle* h, Layer& L, bool left_side, br_handle::Lane& ln) {
+  cudaStream_t s = ln.stream;
   const int64_t m = L.d.m, n = L.d.n;
   const int64_t k = left_side ? m : n;
   float* Q = left_side ? L.U : L.V;
@@ -199,23 +221,23 @@ br_status refresh_side(br_handle* h, Layer& L, bool left_side) {
     if (L.d.src == BR_SRC_SECOND) {
       const float* F = left_side ? L.L : L.R;
       // widen once, then a pure fp64 product (the products are exact either way)
-      BR_CUDA(h, f32_to_f64(F, h->rF, k * k, s));
-      BR_CUDA(h, f32_to_f64(Q, h->rQ, k * k, s));
-      BR_CUDA(h, dgemm(0, 0, k, k, k, 1.0, h->rF, k, h->rQ, k, 0.0, h->rA, k, s));
+      BR_CUDA(h, f32_to_f64(F, ln.rF, k * k, s));
+      BR_CUDA(h, f32_to_f64(Q, ln.rQ, k * k, s));
+      BR_CUDA(h, dgemm(0, 0, k, k, k, 1.0, ln.rF, k, ln.rQ, k, 0.0, ln.rA, k, s));
       count(h, 3); h->stats.gemm_flops += 2.0 * k * k * k;
     } else if (left_side) {
       // (M M^T) U = M (M^T U)
-      BR_CUDA(h, sdgemm(1, 0, n, m, m, 1.0, L.M, n, Q, m, 0.0, h->rZ, m, s));
-      BR_CUDA(h, fdgemm(0, 0, m, m, n, 1.0, L.M, n, h->rZ, m, 0.0, h->rA, m, s));
+      BR_CUDA(h, sdgemm(1, 0, n, m, m, 1.0, L.M, n, Q, m, 0.0, ln.rZ, m, s));
+      BR_CUDA(h, fdgemm(0, 0, m, m, n, 1.0, L.M, n, ln.rZ, m, 0.0, ln.rA, m, s));
       count(h, 2); h->stats.gemm_flops += 4.0 * m * m * n;
     } else {
       // (M^T M) V = M^T (M V)
-      BR_CUDA(h, sdgemm(0, 0, m, n, n, 1.0, L.M, n, Q, n, 0.0, h->rZ, n, s));
-      BR_CUDA(h, fdgemm(1, 0, n, n, m, 1.0, L.M, n, h->rZ, n, 0.0, h->rA, n, s));
+      BR_CUDA(h, sdgemm(0, 0, m, n, n, 1.0, L.M, n, Q, n, 0.0, ln.rZ, n, s));
+      BR_CUDA(h, fdgemm(1, 0, n, n, m, 1.0, L.M, n, ln.rZ, n, 0.0, ln.rA, n, s));
       count(h, 2); h->stats.gemm_flops += 4.0 * n * n * m;
     }
-    BR_CUDA(h, qr_pos_inplace(h->rA, k, h->rWork, h->d_status, s, &h->stats.launches, &h->stats.gemm_flops));
-    BR_CUDA(h, f64_to_f32(h->rA, Q, k * k, s));
+    BR_CUDA(h, qr_pos_inplace(ln.rA, k, ln.rWork, h->d_status, s, &h->stats.launches, &h->stats.gemm_flops));
+    BR_CUDA(h, f64_to_f32(ln.rA, Q, k * k, s));
     count(h);
   }
   if (L.use_tc) {
@@ -225,15 +247,58 @@ br_status refresh_side(br_handle* h, Layer& L, bool left_side) {
   return BR_OK;
 }
 
-br_status refresh_layer(br_handle* h, Layer& L) {
-  br_status st;
+// Refresh the bases of the given layers: every (layer, side) is an independent job; jobs are
+// dealt to the lanes largest first, each to the lane with the least work so far.
+br_status refresh_layers(br_handle* h, const int* ids, int n_ids) {
+  struct Job { int layer; bool left; double cost; };
+  std::vector<Job> jobs;
+  for (int j = 0; j < n_ids; ++j) {
+    const Layer& L = h->layers[ids[j]];
+    if (L.left) jobs.push_back({ids[j], true, (double)L.d.m * L.d.m * L.d.m});
+    if (L.right) jobs.push_back({ids[j], false, (double)L.d.n * L.d.n * L.d.n});
+  }
+  if (jobs.empty()) return BR_OK;
+  std::stable_sort(jobs.begin(), jobs.end(), [](const Job& a, const Job& b) { return a.cost > b.cost; });
+  const int nl = (int)std::min<size_t>((size_t)h->n_lanes, jobs.size());
+  std::vector<std::vector<Job>> per_lane(nl);
+  std::vector<double> load(nl, 0.0);
+  for (const Job& jb : jobs) {
+    int best = 0;
+    for (int i = 1; i < nl; ++i) if (load[i] < load[best]) best = i;
+    per_lane[best].push_back(jb);
+    load[best] += jb.cost;
+  }
   const double f0 = h->stats.gemm_flops;
   const int span = h->stats.prof.begin(PROF_REFRESH, h->stream);
-  if (L.left && (st = refresh_side(h, L, true)) != BR_OK) return st;
-  if (L.right && (st = refresh_side(h, L, false)) != BR_OK) return st;
+  if (nl > 1) {
+    BR_CUDA(h, cudaEventRecord(h->ev_begin, h->stream));
+    for (int i = 1; i < nl; ++i) BR_CUDA(h, cudaStreamWaitEvent(h->lanes[i].stream, h->ev_begin, 0));
+  }
+  // interleave the enqueueing so that every lane has work early
+  size_t longest = 0;
+  for (auto& v : per_lane) longest = std::max(longest, v.size());
+  for (size_t r = 0; r < longest; ++r)
+    for (int i = 0; i < nl; ++i) {
+      if (r >= per_lane[i].size()) continue;
+      const Job& jb = per_lane[i][r];
+      br_status st = refresh_side(h, h->layers[jb.layer], jb.left, h->lanes[i]);
+      if (st != BR_OK) return st;
+    }
+  for (int i = 1; i < nl; ++i) {
+    BR_CUDA(h, cudaEventRecord(h->lanes[i].done, h->lanes[i].stream));
+    BR_CUDA(h, cudaStreamWaitEvent(h->stream, h->lanes[i].done, 0));
+  }
   h->stats.prof.end(span, h->stream, h->stats.gemm_flops - f0);
-  L.refresh_count += 1;
+  for (int j = 0; j < n_ids; ++j) {
+    Layer& L = h->layers[ids[j]];
+    if (L.left || L.right) L.refresh_count += 1;
+  }
   return BR_OK;
+}
+
+br_status refresh_layer(br_handle* h, Layer& L) {
+  const int id = (int)(&L - h->layers.data());
+  return refresh_layers(h, &id, 1);
 }
 
 // L <- beta L + (1-beta) G G^T ; R <- beta R + (1-beta) G^T G   (Alg. 2), fp32 FFMA
@@ -425,6 +490,12 @@ br_status br_create(br_handle** out, const br_layer_desc* layers, int n_layers, 
       if (L.V && (e = split_bf16(L.V, L.Vh, L.Vl, L.d.n * L.d.n, s)) != cudaSuccess) return fail("split_bf16", e);
     }
   }
+  h->lanes[0].stream = s;
+  for (int i = 1; i < h->n_lanes; ++i) {
+    if ((e = cudaStreamCreateWithFlags(&h->lanes[i].stream, cudaStreamNonBlocking)) != cudaSuccess) return fail("cudaStreamCreate", e);
+    if ((e = cudaEventCreateWithFlags(&h->lanes[i].done, cudaEventDisableTiming)) != cudaSuccess) return fail("cudaEventCreate", e);
+  }
+  if ((e = cudaEventCreateWithFlags(&h->ev_begin, cudaEventDisableTiming)) != cudaSuccess) return fail("cudaEventCreate", e);
   const char* tc_err = nullptr;
   h->tc = tc_step_create(h->layers, h->hp, h->slab + sz.total, tc_bytes, device, s, &tc_err);
   if (!h->tc && tc_err) {
@@ -494,9 +565,8 @@ br_status br_step(br_handle* h, const void* const* grads, int tau) {
   if (h->tc) {
     TcStepCallbacks cb;
     cb.ctx = h;
-    cb.refresh = [](void* ctx, int layer) -> int {
-      br_handle* hh = static_cast<br_handle*>(ctx);
-      return (int)refresh_layer(hh, hh->layers[layer]);
+    cb.refresh = [](void* ctx, const int* ids, int n) -> int {
+      return (int)refresh_layers(static_cast<br_handle*>(ctx), ids, n);
     };
     const char* terr = nullptr;
     int rc = tc_step_run(h->tc, h->layers, G, h->calls, tau, hp, h->d_status, h->stream, &h->stats, cb, &terr);
@@ -533,12 +603,10 @@ br_status br_refresh_basis(br_handle* h, int layer) {
       return BR_ERR_STATE;
     }
   }
-  for (int i = lo; i < hi; ++i) {
-    Layer& L = h->layers[i];
-    if (L.d.geom == BR_GEOM_NONE) continue;
-    if ((st = refresh_layer(h, L)) != BR_OK) return st;
-  }
-  return BR_OK;
+  std::vector<int> ids;
+  for (int i = lo; i < hi; ++i)
+    if (h->layers[i].d.geom != BR_GEOM_NONE) ids.push_back(i);
+  return refresh_layers(h, ids.data(), (int)ids.size());
 }
 
 br_status br_sync_status(br_handle* h) {
@@ -658,6 +726,11 @@ br_status br_destroy(br_handle* h) {
   cudaSetDevice(h->device);
   cudaStreamSynchronize(h->stream);
   if (h->tc) tc_step_destroy(h->tc);
+  for (int i = 1; i < br_handle::kMaxLanes; ++i) {
+    if (h->lanes[i].stream) { cudaStreamSynchronize(h->lanes[i].stream); cudaStreamDestroy(h->lanes[i].stream); }
+    if (h->lanes[i].done) cudaEventDestroy(h->lanes[i].done);
+  }
+  if (h->ev_begin) cudaEventDestroy(h->ev_begin);
   for (auto& sp : h->stats.prof.spans) { cudaEventDestroy(sp.a); cudaEventDestroy(sp.b); }
   for (auto e : h->stats.prof.free_events) cudaEventDestroy(e);
   if (h->slab) {

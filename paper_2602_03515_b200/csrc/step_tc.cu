@@ -290,11 +290,15 @@ int tc_step_run(TcStep* t, std::vector<Layer>& layers, const std::vector<const v
     };
     int rc;
     if ((rc = launch(c.factors, "factor launch"))) return rc;
+    std::vector<int> due;
     for (int i : c.ids) {
       Layer& L = layers[i];
       if (!G[i] || L.t % L.freq != 0) continue;
       if (t->factor_plan[i] && (rc = launch(t->factor_plan[i], "factor launch"))) return rc;
-      rc = cb.refresh(cb.ctx, i);
+      due.push_back(i);
+    }
+    if (!due.empty()) {
+      rc = cb.refresh(cb.ctx, due.data(), (int)due.size());
       if (rc != 0) { if (err) *err = nullptr; return rc; }
     }
     if ((rc = launch(c.fwd1, "first-side rotation launch"))) return rc;

@@ -31,7 +31,8 @@ cudaError_t fdgemm(int ta, int tb, int64_t M, int64_t N, int64_t K, double alpha
 struct TcStep;
 struct TcStepCallbacks {
   void* ctx = nullptr;
-  int (*refresh)(void* ctx, int layer) = nullptr;   // runs Power() for a layer, returns br_status
+  // runs Power() for the given layers (independent of one another), returns br_status
+  int (*refresh)(void* ctx, const int* layers, int n) = nullptr;
 };
 
 // Transient scratch (bytes) the tensor-core step needs for these layers.

@@ -288,7 +288,9 @@ def main():
 
     with torch.cuda.stream(stream):
         # ---- priming (untimed): fill the ring, apply one update, refresh every basis once -------
-        for _ in range(tau + 1):
+        # (eight updates before the first refresh: the factor EMAs must have full rank, which takes
+        # ceil(max(m, n) / min(m, n)) gradients; in a real run the first refresh comes at t = freq)
+        for _ in range(tau + 8):
             opt.step(gen.fresh(), tau)
         if not args.no_refresh:
             opt.refresh_basis(-1)

@@ -116,13 +116,19 @@ typedef struct {
 
 typedef enum {
   BR_BUF_W = 0,   /* m*n fp32                                         */
-  BR_BUF_M = 1,   /* m*n fp32, original space                         */
+  BR_BUF_M = 1,   /* m*n fp32, original space (tensor-core layers: U M~ V^T, see BR_BUF_MROT) */
   BR_BUF_V2 = 2,  /* m*n fp32, V~ in the rotated space                */
   BR_BUF_U = 3,   /* m*m fp32 (absent when the left side is unrotated) */
   BR_BUF_V = 4,   /* n*n fp32 (absent when the right side is unrotated) */
   BR_BUF_L = 5,   /* m*m fp32 (S=2nd, left side rotated)              */
   BR_BUF_R = 6,   /* n*n fp32 (S=2nd, right side rotated)             */
-  BR_BUF_RING = 7 /* tau_max * m*n gradients in grad_dtype, slot-major */
+  BR_BUF_RING = 7, /* tau_max * m*n gradients in grad_dtype, slot-major */
+  /* m*n fp32: the momentum in rotated coordinates, M~ = U^T M V.  Between two refreshes
+   * M~_t = beta1 M~_{t-1} + (1-beta1) U^T G_t V holds exactly (Alg. 1 line 4 is linear), and this is
+   * what layers on the tensor-core path store; BR_BUF_M converts on the way in and out with fp32
+   * products.  A checkpoint that must resume bit-identically saves and restores this buffer (after
+   * U and V) instead of BR_BUF_M.  Absent for layers on the fp32 path. */
+  BR_BUF_MROT = 8
 } br_buf;
 
 /* Bytes of device memory br_create would request for these layers (state, ring, operand
@@ -161,7 +167,10 @@ BR_API br_status br_get_counters(br_handle* h, int layer, br_counters* out);
 BR_API br_status br_set_counters(br_handle* h, int layer, const br_counters* in);
 
 /* Copy a state buffer to / from HOST memory; `bytes` must equal the buffer's size.
- * Both synchronise the stream.  Setting U or V also refreshes the operand shadows. */
+ * Both synchronise the stream.  Setting U or V also refreshes the operand shadows and leaves the
+ * momentum of the original space unchanged (a tensor-core layer re-expresses its M~ for the new
+ * basis).  BR_BUF_M of a tensor-core layer needs 8*m*n bytes of temporary device memory from the
+ * handle's allocator for the duration of the call. */
 BR_API br_status br_get_state(br_handle* h, int layer, int which, void* host_dst, size_t bytes);
 BR_API br_status br_set_state(br_handle* h, int layer, int which, const void* host_src, size_t bytes);
 

@@ -17,7 +17,7 @@ BR_SRC_FIRST, BR_SRC_SECOND = 1, 2
 BR_F32, BR_BF16 = 0, 1
 BR_GEMM_FP32, BR_GEMM_BF16 = 0, 2
 BR_ACCUM_EVERY_STEP, BR_ACCUM_ON_REFRESH = 0, 1
-BR_BUF_W, BR_BUF_M, BR_BUF_V2, BR_BUF_U, BR_BUF_V, BR_BUF_L, BR_BUF_R, BR_BUF_RING = range(8)
+BR_BUF_W, BR_BUF_M, BR_BUF_V2, BR_BUF_U, BR_BUF_V, BR_BUF_L, BR_BUF_R, BR_BUF_RING, BR_BUF_MROT = range(9)
 
 
 class BrError(RuntimeError):
@@ -306,7 +306,7 @@ class BasisRotation:
     def _buf_shape(self, layer: int, which: int):
         s = self.specs[layer]
         torch = self._torch
-        if which in (BR_BUF_W, BR_BUF_M, BR_BUF_V2):
+        if which in (BR_BUF_W, BR_BUF_M, BR_BUF_V2, BR_BUF_MROT):
             return (s.m, s.n), torch.float32
         if which in (BR_BUF_U, BR_BUF_L):
             return (s.m, s.m), torch.float32

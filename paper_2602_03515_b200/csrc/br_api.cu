@@ -132,6 +132,7 @@ void layout(br_handle* h, Bump& b, Sizes* sz) {
   for (Layer& L : h->layers) {
     const size_t mn = (size_t)L.d.m * L.d.n;
     L.M = b.take<float>(mn);
+    if (L.use_tc && L.d.src == BR_SRC_FIRST) L.Morig = b.take<float>(mn);
     L.V2 = b.take<float>(mn);
     const bool second = L.d.src == BR_SRC_SECOND;
     if (L.left) { L.U = b.take<float>((size_t)L.d.m * L.d.m); sz->overhead += 4 * (size_t)L.d.m * L.d.m; }
@@ -217,6 +218,9 @@ br_status refresh_side(br_handle* h, Layer& L, bool left_side, br_handle::Lane& 
   const int64_t m = L.d.m, n = L.d.n;
   const int64_t k = left_side ? m : n;
   float* Q = left_side ? L.U : L.V;
+  // S = 1st reads the momentum in the original space: the state buffer itself on the fp32 path, the
+  // copy the caller prepared on the tensor-core path (whose state is the rotated momentum)
+  const float* Mo = L.Morig ? L.Morig : L.M;
   for (int it = 0; it < h->hp.power_iters; ++it) {
     if (L.d.src == BR_SRC_SECOND) {
       const float* F = left_side ? L.L : L.R;
@@ -227,13 +231,13 @@ br_status refresh_side(br_handle* h, Layer& L, bool left_side, br_handle::Lane& 
       count(h, 3); h->stats.gemm_flops += 2.0 * k * k * k;
     } else if (left_side) {
       // (M M^T) U = M (M^T U)
-      BR_CUDA(h, sdgemm(1, 0, n, m, m, 1.0, L.M, n, Q, m, 0.0, ln.rZ, m, s));
-      BR_CUDA(h, fdgemm(0, 0, m, m, n, 1.0, L.M, n, ln.rZ, m, 0.0, ln.rA, m, s));
+      BR_CUDA(h, sdgemm(1, 0, n, m, m, 1.0, Mo, n, Q, m, 0.0, ln.rZ, m, s));
+      BR_CUDA(h, fdgemm(0, 0, m, m, n, 1.0, Mo, n, ln.rZ, m, 0.0, ln.rA, m, s));
       count(h, 2); h->stats.gemm_flops += 4.0 * m * m * n;
     } else {
       // (M^T M) V = M^T (M V)
-      BR_CUDA(h, sdgemm(0, 0, m, n, n, 1.0, L.M, n, Q, n, 0.0, ln.rZ, n, s));
-      BR_CUDA(h, fdgemm(1, 0, n, n, m, 1.0, L.M, n, ln.rZ, n, 0.0, ln.rA, n, s));
+      BR_CUDA(h, sdgemm(0, 0, m, n, n, 1.0, Mo, n, Q, n, 0.0, ln.rZ, n, s));
+      BR_CUDA(h, fdgemm(1, 0, n, n, m, 1.0, Mo, n, ln.rZ, n, 0.0, ln.rA, n, s));
       count(h, 2); h->stats.gemm_flops += 4.0 * n * n * m;
     }
     BR_CUDA(h, qr_pos_inplace(ln.rA, k, ln.rWork, h->d_status, s, &h->stats.launches, &h->stats.gemm_flops));
@@ -334,6 +338,36 @@ br_status rotate_simt(br_handle* h, Layer& L, const float* X, float* tmp, float*
   return BR_OK;
 }
 
+// out = U X V^T with the identity on an unrotated side; tmp is scratch
+br_status rotate_back_simt(br_handle* h, Layer& L, const float* X, float* tmp, float* out) {
+  const int64_t m = L.d.m, n = L.d.n;
+  cudaStream_t s = h->stream;
+  if (L.left && L.right) {
+    BR_CUDA(h, sgemm(0, 0, m, n, m, 1.f, L.U, m, X, n, 0.f, tmp, n, s));
+    BR_CUDA(h, sgemm(0, 1, m, n, n, 1.f, tmp, n, L.V, n, 0.f, out, n, s));
+    count(h, 2);
+  } else if (L.left) {
+    BR_CUDA(h, sgemm(0, 0, m, n, m, 1.f, L.U, m, X, n, 0.f, out, n, s));
+    count(h);
+  } else {
+    BR_CUDA(h, sgemm(0, 1, m, n, n, 1.f, X, n, L.V, n, 0.f, out, n, s));
+    count(h);
+  }
+  return BR_OK;
+}
+
+// Temporary device memory for the state accessors (synchronising calls; not used by br_step).
+float* tmp_alloc(br_handle* h, size_t bytes) {
+  void* p = nullptr;
+  if (h->alloc.alloc) return static_cast<float*>(h->alloc.alloc(bytes, h->alloc.ctx));
+  if (cudaMalloc(&p, bytes) != cudaSuccess) { (void)cudaGetLastError(); return nullptr; }
+  return static_cast<float*>(p);
+}
+void tmp_free(br_handle* h, void* p) {
+  if (!p) return;
+  if (h->alloc.alloc) h->alloc.free(p, h->alloc.ctx); else cudaFree(p);
+}
+
 // One update of one layer on the accurate (fp32 FFMA) path.  G: the gradient to apply.
 br_status update_layer_simt(br_handle* h, Layer& L, const void* G) {
   const br_hparams& hp = h->hp;
@@ -392,6 +426,7 @@ size_t buf_bytes(const Layer& L, int which, void** ptr) {
     case BR_BUF_V: *ptr = L.V; return L.V ? 4 * n * n : 0;
     case BR_BUF_L: *ptr = L.L; return L.L ? 4 * m * m : 0;
     case BR_BUF_R: *ptr = L.R; return L.R ? 4 * n * n : 0;
+    case BR_BUF_MROT: *ptr = L.use_tc ? L.M : nullptr; return L.use_tc ? 4 * m * n : 0;
     case BR_BUF_RING: *ptr = L.d.tau_max > 0 ? L.ring : nullptr; return L.d.tau_max > 0 ? (size_t)L.d.tau_max * m * n * dtype_size(L.d.grad_dtype) : 0;
     default: *ptr = nullptr; return 0;
   }
@@ -603,10 +638,29 @@ br_status br_refresh_basis(br_handle* h, int layer) {
       return BR_ERR_STATE;
     }
   }
-  std::vector<int> ids;
-  for (int i = lo; i < hi; ++i)
-    if (h->layers[i].d.geom != BR_GEOM_NONE) ids.push_back(i);
-  return refresh_layers(h, ids.data(), (int)ids.size());
+  std::vector<int> ids, tc_ids;
+  for (int i = lo; i < hi; ++i) {
+    if (h->layers[i].d.geom == BR_GEOM_NONE) continue;
+    ids.push_back(i);
+    if (h->layers[i].use_tc) tc_ids.push_back(i);
+  }
+  // tensor-core layers keep the rotated momentum: back to the original space with the old basis,
+  // forward again with the new one
+  const char* terr = nullptr;
+  if (!tc_ids.empty()) {
+    int rc = tc_step_reexpress(h->tc, h->layers, tc_ids.data(), (int)tc_ids.size(), 0, h->d_status, h->stream, &h->stats, &terr);
+    if (rc != 0) { h->err = terr ? terr : "re-expression failed"; return (br_status)rc; }
+    for (int i : tc_ids) {
+      Layer& L = h->layers[i];
+      if (L.Morig) BR_CUDA(h, cudaMemcpyAsync(L.Morig, L.M, 4 * (size_t)L.d.m * L.d.n, cudaMemcpyDeviceToDevice, h->stream));
+    }
+  }
+  if ((st = refresh_layers(h, ids.data(), (int)ids.size())) != BR_OK) return st;
+  if (!tc_ids.empty()) {
+    int rc = tc_step_reexpress(h->tc, h->layers, tc_ids.data(), (int)tc_ids.size(), 1, h->d_status, h->stream, &h->stats, &terr);
+    if (rc != 0) { h->err = terr ? terr : "re-expression failed"; return (br_status)rc; }
+  }
+  return BR_OK;
 }
 
 br_status br_sync_status(br_handle* h) {
@@ -653,7 +707,19 @@ br_status br_get_state(br_handle* h, int layer, int which, void* host_dst, size_
   if (!p || want == 0) { h->err = "this layer has no such buffer"; return BR_ERR_STATE; }
   if (bytes != want) { h->err = format("buffer is %zu bytes, caller passed %zu", want, bytes); return BR_ERR_SHAPE; }
   BR_CUDA(h, cudaStreamSynchronize(h->stream));
-  if (which == BR_BUF_RING) {
+  if (which == BR_BUF_M && L.use_tc) {
+    // the state is M~: hand out M = U M~ V^T, computed with fp32 FFMA products into temporaries
+    float* tmp = tmp_alloc(h, 2 * bytes);
+    if (!tmp) { h->err = format("allocation of %zu bytes failed", 2 * bytes); return BR_ERR_OOM; }
+    Layer& Lm = h->layers[layer];
+    float* out = tmp + (size_t)L.d.m * L.d.n;
+    st = rotate_back_simt(h, Lm, L.M, tmp, out);
+    cudaError_t ce = cudaStreamSynchronize(h->stream);
+    if (st == BR_OK && ce == cudaSuccess) ce = cudaMemcpy(host_dst, out, bytes, cudaMemcpyDeviceToHost);
+    tmp_free(h, tmp);
+    if (st != BR_OK) return st;
+    if (ce != cudaSuccess) { h->err = format("get_state: %s", cudaGetErrorString(ce)); return BR_ERR_CUDA; }
+  } else if (which == BR_BUF_RING) {
     const size_t row = (size_t)L.d.m * L.d.n * dtype_size(L.d.grad_dtype);
     BR_CUDA(h, cudaMemcpy2D(host_dst, row, p, L.slot_stride, row, L.d.tau_max, cudaMemcpyDeviceToHost));
   } else {
@@ -672,7 +738,37 @@ br_status br_set_state(br_handle* h, int layer, int which, const void* host_src,
   if (!p || want == 0) { h->err = "this layer has no such buffer"; return BR_ERR_STATE; }
   if (bytes != want) { h->err = format("buffer is %zu bytes, caller passed %zu", want, bytes); return BR_ERR_SHAPE; }
   BR_CUDA(h, cudaStreamSynchronize(h->stream));
-  if (which == BR_BUF_RING) {
+  const size_t mn_bytes = 4 * (size_t)L.d.m * L.d.n;
+  if (L.use_tc && (which == BR_BUF_M || which == BR_BUF_U || which == BR_BUF_V)) {
+    // The state of a tensor-core layer is M~ = U^T M V.  Setting M stores its rotation; setting a
+    // basis keeps M (original space) as it is, so M~ is carried over: M~' = U'^T (U M~) or (M~ V^T) V'.
+    float* tmp = tmp_alloc(h, 2 * mn_bytes);
+    if (!tmp) { h->err = format("allocation of %zu bytes failed", 2 * mn_bytes); return BR_ERR_OOM; }
+    float* tmp2 = tmp + (size_t)L.d.m * L.d.n;
+    const int64_t m = L.d.m, n = L.d.n;
+    cudaStream_t s = h->stream;
+    cudaError_t ce = cudaSuccess;
+    if (which == BR_BUF_M) {
+      ce = cudaMemcpy(tmp, host_src, bytes, cudaMemcpyHostToDevice);
+      if (ce == cudaSuccess) st = rotate_simt(h, L, tmp, tmp2, L.M);
+    } else if (which == BR_BUF_U) {
+      ce = sgemm(0, 0, m, n, m, 1.f, L.U, m, L.M, n, 0.f, tmp, n, s);                 // U_old M~
+      if (ce == cudaSuccess) ce = cudaStreamSynchronize(s);
+      if (ce == cudaSuccess) ce = cudaMemcpy(L.U, host_src, bytes, cudaMemcpyHostToDevice);
+      if (ce == cudaSuccess) ce = sgemm(1, 0, m, n, m, 1.f, L.U, m, tmp, n, 0.f, L.M, n, s);   // U_new^T (.)
+      count(h, 2);
+    } else {
+      ce = sgemm(0, 1, m, n, n, 1.f, L.M, n, L.V, n, 0.f, tmp, n, s);                 // M~ V_old^T
+      if (ce == cudaSuccess) ce = cudaStreamSynchronize(s);
+      if (ce == cudaSuccess) ce = cudaMemcpy(L.V, host_src, bytes, cudaMemcpyHostToDevice);
+      if (ce == cudaSuccess) ce = sgemm(0, 0, m, n, n, 1.f, tmp, n, L.V, n, 0.f, L.M, n, s);   // (.) V_new
+      count(h, 2);
+    }
+    if (ce == cudaSuccess) ce = cudaStreamSynchronize(s);
+    tmp_free(h, tmp);
+    if (st != BR_OK) return st;
+    if (ce != cudaSuccess) { h->err = format("set_state: %s", cudaGetErrorString(ce)); return BR_ERR_CUDA; }
+  } else if (which == BR_BUF_RING) {
     const size_t row = (size_t)L.d.m * L.d.n * dtype_size(L.d.grad_dtype);
     BR_CUDA(h, cudaMemcpy2D(p, L.slot_stride, host_src, row, row, L.d.tau_max, cudaMemcpyHostToDevice));
   } else {

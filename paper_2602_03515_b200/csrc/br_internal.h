@@ -77,6 +77,9 @@ cudaError_t widen_bf16(const __nv_bfloat16* X, float* out, int64_t numel, cudaSt
 // out(double) <- in(float) ; out(float) <- in(double)
 cudaError_t f64_to_f32(const double* X, float* out, int64_t numel, cudaStream_t s);
 cudaError_t f32_to_f64(const float* X, double* out, int64_t numel, cudaStream_t s);
+// out <- beta1 M + (1-beta1) G (out-of-place form of Alg. 1 line 4)
+cudaError_t ema_out(float* out, const float* M, const void* G, int g_is_bf16, int64_t numel, float beta1,
+                    cudaStream_t s);
 
 // ---------------------------------------------------------------------------------------------
 // SIMT contractions (gemm_simt.cu):  C = alpha * op(A) op(B) + beta * C, row-major.
@@ -115,7 +118,10 @@ enum Epilogue : int32_t {
   EPI_AXPBY_F32 = 0,    // D <- alpha*acc + beta*D                 (factor EMA, weight write, plain)
   EPI_SPLIT_BF16 = 1,   // Dh <- bf16(acc), Dl <- bf16(acc - Dh)   (Dl optional)
   EPI_SECOND_MOMENT = 2,// D(V~) <- beta*D + alpha*acc^2
-  EPI_SCALE_BF16 = 3    // Dh(X) <- bf16(acc / sqrt(D(V~) + eps))
+  EPI_SCALE_BF16 = 3,   // Dh(X) <- bf16(acc / sqrt(D(V~) + eps))
+  // Alg. 1 lines 4, 10, 11 in rotated coordinates, acc = G~:
+  //   D2(M~) <- beta1 D2 + (1-beta1) acc ; D(V~) <- beta D + alpha acc^2 ; Dh(X) <- bf16(D2 / sqrt(D + eps))
+  EPI_ROTATED_ADAM = 4
 };
 
 struct TcOperand {
@@ -133,8 +139,9 @@ struct TcProblem {
   int32_t epilogue = EPI_AXPBY_F32;
   int32_t tau_max = 0;            // of the layer (delay bookkeeping on the device)
   int32_t dyn_scalars = 0;        // 1: alpha / beta come from the launch arguments
-  float alpha = 1.f, beta = 0.f, eps = 0.f;
+  float alpha = 1.f, beta = 0.f, eps = 0.f, beta1 = 0.f;
   float* D = nullptr; int64_t ldd = 0;                                   // fp32 in/out
+  float* D2 = nullptr;                                                   // second fp32 in/out (same ld)
   __nv_bfloat16* Dh = nullptr; __nv_bfloat16* Dl = nullptr; int64_t ldh = 0;  // bf16 outputs
 };
 

@@ -195,6 +195,26 @@ k_widen_bf16(const __nv_bfloat16* __restrict__ X, float* __restrict__ out, int64
     out[i] = __bfloat162float(X[i]);
 }
 
+// out <- beta1 M + (1-beta1) G, M untouched (M_t for a refresh that reads the momentum)
+template <bool G_BF16>
+__global__ void __launch_bounds__(kThreads)
+k_ema_out(float* __restrict__ out, const float* __restrict__ M, const void* __restrict__ G, int64_t numel,
+          float beta1) {
+  const float omb = 1.0f - beta1;
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  const int64_t nvec = numel >> 2;
+  for (int64_t v = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; v < nvec; v += stride) {
+    const int64_t i = v << 2;
+    const float4 g = load_grad4<G_BF16>(G, i);
+    float4 m = ld4(M + i);
+    m.x = beta1 * m.x + omb * g.x; m.y = beta1 * m.y + omb * g.y;
+    m.z = beta1 * m.z + omb * g.z; m.w = beta1 * m.w + omb * g.w;
+    st4(out + i, m);
+  }
+  for (int64_t i = (nvec << 2) + blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < numel; i += stride)
+    out[i] = beta1 * M[i] + omb * load_grad1<G_BF16>(G, i);
+}
+
 __global__ void __launch_bounds__(kThreads)
 k_f32_to_f64(const float* __restrict__ X, double* __restrict__ out, int64_t numel) {
   const int64_t stride = (int64_t)gridDim.x * blockDim.x;
@@ -251,6 +271,14 @@ cudaError_t split_bf16(const float* X, __nv_bfloat16* hi, __nv_bfloat16* lo, int
 
 cudaError_t widen_bf16(const __nv_bfloat16* X, float* out, int64_t numel, cudaStream_t s) {
   k_widen_bf16<<<grid_for((numel + 3) / 4), kThreads, 0, s>>>(X, out, numel);
+  return cudaGetLastError();
+}
+
+cudaError_t ema_out(float* out, const float* M, const void* G, int g_is_bf16, int64_t numel, float beta1,
+                    cudaStream_t s) {
+  const int grid = grid_for((numel + 3) / 4);
+  if (g_is_bf16) k_ema_out<true><<<grid, kThreads, 0, s>>>(out, M, G, numel, beta1);
+  else k_ema_out<false><<<grid, kThreads, 0, s>>>(out, M, G, numel, beta1);
   return cudaGetLastError();
 }
 

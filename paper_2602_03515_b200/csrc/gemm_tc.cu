@@ -2,7 +2,8 @@
 //   D_tile = sum over operand pairs p and k-blocks of A_p[128 x 64] * B_p[256 x 64]^T
 // TMA (cp.async.bulk.tensor, 128-byte swizzle) stages operand tiles in shared memory, one elected
 // thread issues tcgen05.mma (kind::f16, bf16 operands, fp32 accumulation) into tensor memory,
-// four epilogue warps read the accumulator back with tcgen05.ld and apply a fused epilogue
+// four epilogue warps read the accumulator back with tcgen05.ld, turn it through shared memory so
+// that global memory is accessed along rows, and apply a fused epilogue
 // (factor EMA, bf16 hi/lo split, second-moment update, Adam scaling, weight write).
 //
 // One persistent CTA per SM walks a static tile list that spans every problem of a launch
@@ -37,7 +38,9 @@ constexpr int STAGES = 4;
 constexpr int A_BYTES = BM * BK * 2;             // 16 KiB
 constexpr int B_BYTES = BN * BK * 2;             // 32 KiB
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024;   // + slack to align the tiles to 1 KiB
+constexpr int EPI_LD = 36;                       // padded row of an epilogue tile (floats): 16-byte rows, no bank conflicts
+constexpr int EPI_BYTES = 4 * 32 * EPI_LD * 4;   // one 32 x 32 fp32 tile per epilogue warp
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BYTES + 1024;   // + slack to align the tiles to 1 KiB
 constexpr int TMEM_COLS = 512;
 constexpr int NUM_THREADS = 192;                 // warp 0: TMA, warp 1: MMA, warps 2..5: epilogue
 constexpr int MAX_PAIRS = 3;
@@ -50,13 +53,13 @@ struct alignas(128) DevProblem {
   int32_t a_mn, b_mn, epilogue, tiles_m;
   int32_t tiles_n, tile_begin, tile_count, tau_max;
   int32_t ring_slots, a_ring_mask, b_ring_mask, dyn_scalars;
-  float alpha, beta, eps, pad_;
+  float alpha, beta, eps, beta1;
   float* D;
   long long ldd;
   __nv_bfloat16* Dh;
   __nv_bfloat16* Dl;
   long long ldh;
-  long long pad2_;
+  float* D2;
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -235,6 +238,7 @@ k_tc_gemm(const DevProblem* __restrict__ probs, int n_probs, int total_tiles, lo
   const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   auto sA = [&](int s) { return tiles_base + (uint32_t)s * A_BYTES; };
   auto sB = [&](int s) { return tiles_base + (uint32_t)STAGES * A_BYTES + (uint32_t)s * B_BYTES; };
+  float* epi_tiles = reinterpret_cast<float*>(smem_raw + ((tiles_base - smem_u32(smem_raw)) + (uint32_t)STAGES * STAGE_BYTES));
   const uint32_t bar0 = smem_u32(bars);
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
   auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
@@ -337,90 +341,97 @@ k_tc_gemm(const DevProblem* __restrict__ probs, int n_probs, int total_tiles, lo
     }
   } else {
     // ======================= epilogue warps =======================
+    // A warp may read only its own quadrant of tensor memory, where lane = accumulator row: a
+    // 32 x 32 block arrives with one row per lane.  It is turned through a padded shared-memory
+    // tile so that global memory is accessed along rows: 8 lanes cover 128 contiguous bytes of one
+    // row, a warp instruction four whole rows.
     const int quad = warp & 3;                    // tensor-memory lane quadrant this warp may read
+    float* tile = epi_tiles + quad * (32 * EPI_LD);
+    const int sub_r = lane >> 3, sub_c = (lane & 7) * 4;
     int acc = 0; uint32_t acc_phase = 0;
-    for (int tile = blockIdx.x; tile < total_tiles && !*abort_flag; tile += gridDim.x) {
-      const TileInfo ti = locate_tile(probs, n_probs, tile, calls, tau);
+    for (int tile_i = blockIdx.x; tile_i < total_tiles && !*abort_flag; tile_i += gridDim.x) {
+      const TileInfo ti = locate_tile(probs, n_probs, tile_i, calls, tau);
       if (!ti.active) continue;
       const DevProblem* p = ti.p;
       if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag, status)) break;
       tc_fence_after();
-      const int row = ti.m0 + quad * 32 + lane;
-      const bool row_ok = row < p->Md;
       const float alpha = p->dyn_scalars ? dyn_alpha : p->alpha;
       const float beta = p->dyn_scalars ? dyn_beta : p->beta;
       const float eps = p->eps;
       const int epi = p->epilogue;
+      const int row_base = ti.m0 + quad * 32;
+      const bool quad_ok = row_base < p->Md;      // uniform across the warp
 #pragma unroll 1
       for (int c0 = 0; c0 < BN; c0 += 32) {
         if (ti.n0 + c0 >= p->Nd) break;           // uniform across the warp
         float v[32];
         tmem_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * BN + c0), v);
-        if (!row_ok) continue;
-        const int col0 = ti.n0 + c0;
-        if (epi == EPI_AXPBY_F32) {
-          float* d = p->D + (long long)row * p->ldd + col0;
+        if (!quad_ok) continue;
+        __syncwarp();
 #pragma unroll
-          for (int j = 0; j < 32; j += 4) {
-            if (col0 + j >= p->Nd) break;
-            float4 o = make_float4(alpha * v[j], alpha * v[j + 1], alpha * v[j + 2], alpha * v[j + 3]);
+        for (int q = 0; q < 8; ++q)
+          *reinterpret_cast<float4*>(tile + lane * EPI_LD + 4 * q) = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+        __syncwarp();
+        const int col = ti.n0 + c0 + sub_c;
+        // columns come in multiples of 8: a float4 is all in or all out
+        const int n_it = (col < p->Nd) ? 8 : 0;
+#pragma unroll 2
+        for (int it = 0; it < n_it; ++it) {
+          const int rl = it * 4 + sub_r;
+          const int row = row_base + rl;
+          if (row >= p->Md) break;
+          const float4 a = *reinterpret_cast<const float4*>(tile + rl * EPI_LD + sub_c);
+          if (epi == EPI_AXPBY_F32) {
+            float* d = p->D + (long long)row * p->ldd + col;
+            float4 o = make_float4(alpha * a.x, alpha * a.y, alpha * a.z, alpha * a.w);
             if (beta != 0.0f) {
-              const float4 old = *reinterpret_cast<const float4*>(d + j);
+              const float4 old = *reinterpret_cast<const float4*>(d);
               o.x = fmaf(beta, old.x, o.x); o.y = fmaf(beta, old.y, o.y);
               o.z = fmaf(beta, old.z, o.z); o.w = fmaf(beta, old.w, o.w);
             }
-            *reinterpret_cast<float4*>(d + j) = o;
-          }
-        } else if (epi == EPI_SECOND_MOMENT) {
-          float* d = p->D + (long long)row * p->ldd + col0;
-#pragma unroll
-          for (int j = 0; j < 32; j += 4) {
-            if (col0 + j >= p->Nd) break;
-            float4 s = *reinterpret_cast<const float4*>(d + j);
-            s.x = fmaf(beta, s.x, alpha * v[j] * v[j]);
-            s.y = fmaf(beta, s.y, alpha * v[j + 1] * v[j + 1]);
-            s.z = fmaf(beta, s.z, alpha * v[j + 2] * v[j + 2]);
-            s.w = fmaf(beta, s.w, alpha * v[j + 3] * v[j + 3]);
-            *reinterpret_cast<float4*>(d + j) = s;
-          }
-        } else if (epi == EPI_SCALE_BF16) {
-          const float* d = p->D + (long long)row * p->ldd + col0;
-          __nv_bfloat16* xh = p->Dh + (long long)row * p->ldh + col0;
-#pragma unroll
-          for (int j = 0; j < 32; j += 8) {
-            if (col0 + j >= p->Nd) break;
-            const float4 s0 = *reinterpret_cast<const float4*>(d + j);
-            const float4 s1 = *reinterpret_cast<const float4*>(d + j + 4);
-            uint4 o;
-            o.x = pack2_bf16(v[j] / sqrtf(s0.x + eps), v[j + 1] / sqrtf(s0.y + eps));
-            o.y = pack2_bf16(v[j + 2] / sqrtf(s0.z + eps), v[j + 3] / sqrtf(s0.w + eps));
-            o.z = pack2_bf16(v[j + 4] / sqrtf(s1.x + eps), v[j + 5] / sqrtf(s1.y + eps));
-            o.w = pack2_bf16(v[j + 6] / sqrtf(s1.z + eps), v[j + 7] / sqrtf(s1.w + eps));
-            *reinterpret_cast<uint4*>(xh + j) = o;
-          }
-        } else {  // EPI_SPLIT_BF16
-          __nv_bfloat16* dh = p->Dh + (long long)row * p->ldh + col0;
-          __nv_bfloat16* dl = p->Dl ? p->Dl + (long long)row * p->ldh + col0 : nullptr;
-#pragma unroll
-          for (int j = 0; j < 32; j += 8) {
-            if (col0 + j >= p->Nd) break;
-            float h[8];
-#pragma unroll
-            for (int e = 0; e < 8; ++e) h[e] = __bfloat162float(__float2bfloat16_rn(v[j + e]));
-            uint4 o;
-            o.x = pack2_bf16(h[0], h[1]); o.y = pack2_bf16(h[2], h[3]);
-            o.z = pack2_bf16(h[4], h[5]); o.w = pack2_bf16(h[6], h[7]);
-            *reinterpret_cast<uint4*>(dh + j) = o;
-            if (dl) {
-              uint4 l;
-              l.x = pack2_bf16(v[j] - h[0], v[j + 1] - h[1]);
-              l.y = pack2_bf16(v[j + 2] - h[2], v[j + 3] - h[3]);
-              l.z = pack2_bf16(v[j + 4] - h[4], v[j + 5] - h[5]);
-              l.w = pack2_bf16(v[j + 6] - h[6], v[j + 7] - h[7]);
-              *reinterpret_cast<uint4*>(dl + j) = l;
+            *reinterpret_cast<float4*>(d) = o;
+          } else if (epi == EPI_ROTATED_ADAM) {
+            float* d = p->D + (long long)row * p->ldd + col;      // V~
+            float* m2 = p->D2 + (long long)row * p->ldd + col;    // M~
+            const float b1 = p->beta1, ob1 = 1.0f - p->beta1;
+            float4 mm = *reinterpret_cast<const float4*>(m2);
+            float4 ss = *reinterpret_cast<const float4*>(d);
+            mm.x = b1 * mm.x + ob1 * a.x; mm.y = b1 * mm.y + ob1 * a.y;
+            mm.z = b1 * mm.z + ob1 * a.z; mm.w = b1 * mm.w + ob1 * a.w;
+            ss.x = fmaf(beta, ss.x, alpha * a.x * a.x); ss.y = fmaf(beta, ss.y, alpha * a.y * a.y);
+            ss.z = fmaf(beta, ss.z, alpha * a.z * a.z); ss.w = fmaf(beta, ss.w, alpha * a.w * a.w);
+            *reinterpret_cast<float4*>(m2) = mm;
+            *reinterpret_cast<float4*>(d) = ss;
+            uint2 o;
+            o.x = pack2_bf16(mm.x / sqrtf(ss.x + eps), mm.y / sqrtf(ss.y + eps));
+            o.y = pack2_bf16(mm.z / sqrtf(ss.z + eps), mm.w / sqrtf(ss.w + eps));
+            *reinterpret_cast<uint2*>(p->Dh + (long long)row * p->ldh + col) = o;
+          } else if (epi == EPI_SECOND_MOMENT) {
+            float* d = p->D + (long long)row * p->ldd + col;
+            float4 s4 = *reinterpret_cast<const float4*>(d);
+            s4.x = fmaf(beta, s4.x, alpha * a.x * a.x); s4.y = fmaf(beta, s4.y, alpha * a.y * a.y);
+            s4.z = fmaf(beta, s4.z, alpha * a.z * a.z); s4.w = fmaf(beta, s4.w, alpha * a.w * a.w);
+            *reinterpret_cast<float4*>(d) = s4;
+          } else if (epi == EPI_SCALE_BF16) {
+            const float4 s4 = *reinterpret_cast<const float4*>(p->D + (long long)row * p->ldd + col);
+            uint2 o;
+            o.x = pack2_bf16(a.x / sqrtf(s4.x + eps), a.y / sqrtf(s4.y + eps));
+            o.y = pack2_bf16(a.z / sqrtf(s4.z + eps), a.w / sqrtf(s4.w + eps));
+            *reinterpret_cast<uint2*>(p->Dh + (long long)row * p->ldh + col) = o;
+          } else {  // EPI_SPLIT_BF16
+            const float h0 = __bfloat162float(__float2bfloat16_rn(a.x)), h1 = __bfloat162float(__float2bfloat16_rn(a.y));
+            const float h2 = __bfloat162float(__float2bfloat16_rn(a.z)), h3 = __bfloat162float(__float2bfloat16_rn(a.w));
+            uint2 o;
+            o.x = pack2_bf16(h0, h1); o.y = pack2_bf16(h2, h3);
+            *reinterpret_cast<uint2*>(p->Dh + (long long)row * p->ldh + col) = o;
+            if (p->Dl) {
+              uint2 l;
+              l.x = pack2_bf16(a.x - h0, a.y - h1); l.y = pack2_bf16(a.z - h2, a.w - h3);
+              *reinterpret_cast<uint2*>(p->Dl + (long long)row * p->ldh + col) = l;
             }
           }
         }
+        __syncwarp();                             // the tile is rewritten by the next block
       }
       // all tcgen05.ld of this warp have completed (wait::ld): hand the accumulator back
       tc_fence_before();
@@ -538,10 +549,12 @@ TcPlan* tc_plan_create(const TcProblem* problems, int n, int device, cudaStream_
     tile_begin += d.tile_count;
     d.tau_max = q.tau_max;
     d.dyn_scalars = q.dyn_scalars;
-    d.alpha = q.alpha; d.beta = q.beta; d.eps = q.eps;
-    d.D = q.D; d.ldd = q.ldd; d.Dh = q.Dh; d.Dl = q.Dl; d.ldh = q.ldh;
+    d.alpha = q.alpha; d.beta = q.beta; d.eps = q.eps; d.beta1 = q.beta1;
+    d.D = q.D; d.ldd = q.ldd; d.Dh = q.Dh; d.Dl = q.Dl; d.ldh = q.ldh; d.D2 = q.D2;
     const bool need_D = q.epilogue != EPI_SPLIT_BF16;
-    const bool need_H = q.epilogue == EPI_SPLIT_BF16 || q.epilogue == EPI_SCALE_BF16;
+    const bool need_H = q.epilogue == EPI_SPLIT_BF16 || q.epilogue == EPI_SCALE_BF16 || q.epilogue == EPI_ROTATED_ADAM;
+    if (q.epilogue == EPI_ROTATED_ADAM && (!q.D2 || (reinterpret_cast<uintptr_t>(q.D2) & 15)))
+      return fail("tensor-core problem: second in/out pointer missing or misaligned");
     if ((need_D && (!q.D || (q.ldd % 4) || (reinterpret_cast<uintptr_t>(q.D) & 15))) ||
         (need_H && (!q.Dh || (q.ldh % 8) || (reinterpret_cast<uintptr_t>(q.Dh) & 15))) ||
         (q.Dl && (reinterpret_cast<uintptr_t>(q.Dl) & 15)))

@@ -1,20 +1,28 @@
-// Launch plan of the tensor-core path of one step.  Layers are processed in chunks whose
-// transient bf16 scratch (hi/lo split of M, first-side products, X) fits a byte budget; within a
-// chunk every phase of Algorithm 1 is ONE grouped launch over all layers of the chunk:
+// Launch plan of the tensor-core path of one step.
 //
-//   momentum EMA (+ bf16 hi/lo of M)                       element-wise, per layer
-//   factors   L <- b L + (1-b) G G^T , R <- b R + (1-b) G^T G          (Alg. 2)
-//   [refresh of the layers that are due]                                (Alg. 1 lines 5-6)
-//   fwd1      T_G = U^T G , T_M = U^T M            -> bf16 hi/lo        (Alg. 1 lines 8-9)
-//   v2        V~ <- b2 V~ + (1-b2) (T_G V)^2        fused epilogue      (line 10)
-//   scale     X = (T_M V) / sqrt(V~ + eps)          fused epilogue      (line 11)
+// Between two refreshes the bases U, V are constant, so the rotated momentum obeys
+//   M~_t = U^T M_t V = beta1 M~_{t-1} + (1 - beta1) U^T G_t V
+// exactly (Alg. 1 line 4 is linear).  The tensor-core path therefore keeps M~ as its state instead
+// of M: the momentum is never rotated, which removes one of the four two-sided products of Alg. 1,
+// and its EMA joins the second-moment update and the Adam scaling in one fused epilogue.  Only a
+// refresh needs M itself: the due layers are re-expressed, M = U M~ V^T with the old basis before
+// the refresh (Alg. 2 with S = 1st reads M) and M~ = U^T M V with the new basis after it.
+//
+// Layers are processed in chunks whose transient bf16 scratch fits a byte budget; within a chunk
+// every phase is ONE grouped launch over all layers of the chunk:
+//
+//   factors   L <- b L + (1-b) G G^T , R <- b R + (1-b) G^T G            (Alg. 2)
+//   [refresh of the layers that are due, bracketed by the re-expression]  (Alg. 1 lines 5-6)
+//   fwd1      T = U^T G                               -> bf16 hi/lo       (Alg. 1 line 8, first side)
+//   adam      G~ = T V, fused epilogue: M~ <- b1 M~ + (1-b1) G~ ; V~ <- b2 V~ + (1-b2) G~^2 ;
+//             X = M~ / sqrt(V~ + eps)                                      (lines 4, 8-11)
 //   back1     Y = U X
-//   wwrite    W <- (1 - eta lambda) W - eta Y V^T   fused epilogue
+//   wwrite    W <- (1 - eta lambda) W - eta Y V^T     fused epilogue      (line 11)
 //
-// fp32 operands of the forward rotations (U, V, M, T) enter as a bf16 hi/lo pair and the
-// products hi*hi + lo*hi + hi*lo are accumulated in tensor memory: a single bf16 rounding of
-// the basis leaks the dominant gradient directions into every rotated coordinate at the 1e-3
-// level, which for low-rank-plus-noise gradients is as large as the noise coordinates
+// fp32 operands of the forward rotations (U, V, T, and M / M~ in the re-expression) enter as a
+// bf16 hi/lo pair and the products hi*hi + lo*hi + hi*lo are accumulated in tensor memory: a single
+// bf16 rounding of the basis leaks the dominant gradient directions into every rotated coordinate
+// at the 1e-3 level, which for low-rank-plus-noise gradients is as large as the noise coordinates
 // themselves.  The back rotation acts on X, whose entries are O(1) by construction, and uses
 // single bf16 operands.
 #include <algorithm>
@@ -29,19 +37,26 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 constexpr size_t kDefaultScratch = 4ull << 30;
 
 struct LayerScratch {
-  __nv_bfloat16 *Mh = nullptr, *Ml = nullptr, *TGh = nullptr, *TGl = nullptr, *TMh = nullptr, *TMl = nullptr,
-                *X = nullptr;
+  __nv_bfloat16* B[4] = {nullptr, nullptr, nullptr, nullptr};
 };
 
 size_t layer_scratch_bytes(const Layer& L) {
   const size_t one = align_up((size_t)L.d.m * L.d.n * 2);
-  return (L.left && L.right) ? 7 * one : 3 * one;
+  return (L.left && L.right) ? 4 * one : 2 * one;
 }
+
+// The four phases of a re-expression: M = U M~ V^T (back) and M~ = U^T M V (fwd), each with a
+// first-side product into a bf16 hi/lo pair and a second-side product into the fp32 buffer.
+struct RxPlans {
+  TcPlan *back1 = nullptr, *back2 = nullptr, *fwd1 = nullptr, *fwd2 = nullptr;
+};
 
 struct Chunk {
   std::vector<int> ids;
   std::vector<LayerScratch> scr;
-  TcPlan *factors = nullptr, *fwd1 = nullptr, *v2 = nullptr, *scale = nullptr, *back1 = nullptr, *wwrite = nullptr;
+  TcPlan *factors = nullptr, *fwd1 = nullptr, *adam = nullptr, *back1 = nullptr, *wwrite = nullptr;
+  RxPlans rx;                       // all layers of the chunk
+  std::vector<RxPlans> rx_layer;    // one layer at a time
 };
 
 std::vector<std::vector<int>> make_chunks(const std::vector<Layer>& layers, const br_hparams& hp) {
@@ -67,33 +82,16 @@ TcOperand ring_op(const Layer& L, int mn) {
   return o;
 }
 
-}  // namespace
-
-struct TcStep {
-  std::vector<Chunk> chunks;
-  std::vector<TcPlan*> factor_plan;   // per layer, BR_ACCUM_ON_REFRESH only
-  std::string err;
-};
-
-size_t tc_step_scratch_bytes(const std::vector<Layer>& layers, const br_hparams& hp) {
-  size_t worst = 0;
-  for (const auto& ids : make_chunks(layers, hp)) {
-    size_t b = 0;
-    for (int i : ids) b += layer_scratch_bytes(layers[i]);
-    worst = std::max(worst, b);
-  }
-  return worst;
+// hi*hi + lo*hi + hi*lo for (A, B) given as hi/lo pairs
+void three_pairs(TcProblem& q, const void* Ah, const void* Al, int64_t lda, int a_mn, const void* Bh,
+                 const void* Bl, int64_t ldb, int b_mn) {
+  q.n_pairs = 3;
+  q.A[0] = op(Ah, lda, a_mn); q.B[0] = op(Bh, ldb, b_mn);
+  q.A[1] = op(Al, lda, a_mn); q.B[1] = op(Bh, ldb, b_mn);
+  q.A[2] = op(Ah, lda, a_mn); q.B[2] = op(Bl, ldb, b_mn);
 }
 
-void tc_step_destroy(TcStep* t) {
-  if (!t) return;
-  for (Chunk& c : t->chunks)
-    for (TcPlan* p : {c.factors, c.fwd1, c.v2, c.scale, c.back1, c.wwrite}) tc_plan_destroy(p);
-  for (TcPlan* p : t->factor_plan) tc_plan_destroy(p);
-  delete t;
-}
-
-static void factor_problems(const Layer& L, float beta, std::vector<TcProblem>* out) {
+void factor_problems(const Layer& L, float beta, std::vector<TcProblem>* out) {
   const int64_t m = L.d.m, n = L.d.n;
   if (L.L) {      // L <- beta L + (1-beta) G G^T : both operands K-major views of G
     TcProblem q; q.Md = m; q.Nd = m; q.K = n; q.n_pairs = 1;
@@ -109,6 +107,146 @@ static void factor_problems(const Layer& L, float beta, std::vector<TcProblem>* 
   }
 }
 
+struct StepProblems {
+  std::vector<TcProblem> factors, fwd1, adam, back1, wwrite;
+};
+struct RxProblems {
+  std::vector<TcProblem> back1, back2, fwd1, fwd2;
+};
+
+void rotated_adam_epilogue(TcProblem& q, const Layer& L, const br_hparams& hp, __nv_bfloat16* X) {
+  q.epilogue = EPI_ROTATED_ADAM;
+  q.alpha = 1.f - hp.beta2; q.beta = hp.beta2; q.beta1 = hp.beta1; q.eps = hp.eps;
+  q.D = L.V2; q.D2 = L.M; q.ldd = L.d.n; q.Dh = X; q.ldh = L.d.n;
+}
+
+void step_problems(const Layer& L, const LayerScratch& S, const br_hparams& hp, StepProblems* P) {
+  const int64_t m = L.d.m, n = L.d.n;
+  const int tm = L.d.tau_max;
+  if (L.left && L.right) {
+    {  // T = U^T G : (Uh, G) + (Ul, G); U and G both enter MN-major (contraction over rows)
+      TcProblem q; q.Md = m; q.Nd = n; q.K = m; q.n_pairs = 2; q.tau_max = tm;
+      q.A[0] = op(L.Uh, m, 1); q.B[0] = ring_op(L, 1);
+      q.A[1] = op(L.Ul, m, 1); q.B[1] = ring_op(L, 1);
+      q.epilogue = EPI_SPLIT_BF16; q.Dh = S.B[0]; q.Dl = S.B[1]; q.ldh = n;
+      P->fwd1.push_back(q);
+    }
+    {  // G~ = T V : T K-major, V MN-major
+      TcProblem q; q.Md = m; q.Nd = n; q.K = n; q.tau_max = tm;
+      three_pairs(q, S.B[0], S.B[1], n, 0, L.Vh, L.Vl, n, 1);
+      rotated_adam_epilogue(q, L, hp, S.B[2]);
+      P->adam.push_back(q);
+    }
+    {  // Y = U X : U K-major, X MN-major
+      TcProblem q; q.Md = m; q.Nd = n; q.K = m; q.n_pairs = 1; q.tau_max = tm;
+      q.A[0] = op(L.Uh, m, 0); q.B[0] = op(S.B[2], n, 1);
+      q.epilogue = EPI_SPLIT_BF16; q.Dh = S.B[0]; q.Dl = nullptr; q.ldh = n;
+      P->back1.push_back(q);
+    }
+    {  // W <- decay W - eta Y V^T : both K-major
+      TcProblem q; q.Md = m; q.Nd = n; q.K = n; q.n_pairs = 1; q.tau_max = tm;
+      q.A[0] = op(S.B[0], n, 0); q.B[0] = op(L.Vh, n, 0);
+      q.epilogue = EPI_AXPBY_F32; q.dyn_scalars = 1; q.D = L.d.weight; q.ldd = n;
+      P->wwrite.push_back(q);
+    }
+  } else if (L.left) {
+    {  // G~ = U^T G
+      TcProblem q; q.Md = m; q.Nd = n; q.K = m; q.n_pairs = 2; q.tau_max = tm;
+      q.A[0] = op(L.Uh, m, 1); q.B[0] = ring_op(L, 1);
+      q.A[1] = op(L.Ul, m, 1); q.B[1] = ring_op(L, 1);
+      rotated_adam_epilogue(q, L, hp, S.B[0]);
+      P->adam.push_back(q);
+    }
+    {  // W <- decay W - eta U X
+      TcProblem q; q.Md = m; q.Nd = n; q.K = m; q.n_pairs = 1; q.tau_max = tm;
+      q.A[0] = op(L.Uh, m, 0); q.B[0] = op(S.B[0], n, 1);
+      q.epilogue = EPI_AXPBY_F32; q.dyn_scalars = 1; q.D = L.d.weight; q.ldd = n;
+      P->wwrite.push_back(q);
+    }
+  } else {
+    {  // G~ = G V
+      TcProblem q; q.Md = m; q.Nd = n; q.K = n; q.n_pairs = 2; q.tau_max = tm;
+      q.A[0] = ring_op(L, 0); q.B[0] = op(L.Vh, n, 1);
+      q.A[1] = ring_op(L, 0); q.B[1] = op(L.Vl, n, 1);
+      rotated_adam_epilogue(q, L, hp, S.B[0]);
+      P->adam.push_back(q);
+    }
+    {  // W <- decay W - eta X V^T
+      TcProblem q; q.Md = m; q.Nd = n; q.K = n; q.n_pairs = 1; q.tau_max = tm;
+      q.A[0] = op(S.B[0], n, 0); q.B[0] = op(L.Vh, n, 0);
+      q.epilogue = EPI_AXPBY_F32; q.dyn_scalars = 1; q.D = L.d.weight; q.ldd = n;
+      P->wwrite.push_back(q);
+    }
+  }
+}
+
+// Re-expression problems.  The fp32 buffer L.M is split into the bf16 pair (B0, B1) by the caller
+// before either direction; the first-side product of a bilateral layer goes to (B2, B3).
+void rx_problems(const Layer& L, const LayerScratch& S, RxProblems* P) {
+  const int64_t m = L.d.m, n = L.d.n;
+  auto store_f32 = [&](TcProblem& q) {
+    q.epilogue = EPI_AXPBY_F32; q.alpha = 1.f; q.beta = 0.f; q.D = L.M; q.ldd = n;
+  };
+  auto store_pair = [&](TcProblem& q) {
+    q.epilogue = EPI_SPLIT_BF16; q.Dh = S.B[2]; q.Dl = S.B[3]; q.ldh = n;
+  };
+  if (L.left && L.right) {
+    { TcProblem q; q.Md = m; q.Nd = n; q.K = m;      // Y = U M~ : U K-major, M~ MN-major
+      three_pairs(q, L.Uh, L.Ul, m, 0, S.B[0], S.B[1], n, 1); store_pair(q); P->back1.push_back(q); }
+    { TcProblem q; q.Md = m; q.Nd = n; q.K = n;      // M = Y V^T : both K-major
+      three_pairs(q, S.B[2], S.B[3], n, 0, L.Vh, L.Vl, n, 0); store_f32(q); P->back2.push_back(q); }
+    { TcProblem q; q.Md = m; q.Nd = n; q.K = m;      // T = U^T M : both MN-major
+      three_pairs(q, L.Uh, L.Ul, m, 1, S.B[0], S.B[1], n, 1); store_pair(q); P->fwd1.push_back(q); }
+    { TcProblem q; q.Md = m; q.Nd = n; q.K = n;      // M~ = T V : T K-major, V MN-major
+      three_pairs(q, S.B[2], S.B[3], n, 0, L.Vh, L.Vl, n, 1); store_f32(q); P->fwd2.push_back(q); }
+  } else if (L.left) {
+    { TcProblem q; q.Md = m; q.Nd = n; q.K = m;      // M = U M~
+      three_pairs(q, L.Uh, L.Ul, m, 0, S.B[0], S.B[1], n, 1); store_f32(q); P->back2.push_back(q); }
+    { TcProblem q; q.Md = m; q.Nd = n; q.K = m;      // M~ = U^T M
+      three_pairs(q, L.Uh, L.Ul, m, 1, S.B[0], S.B[1], n, 1); store_f32(q); P->fwd2.push_back(q); }
+  } else {
+    { TcProblem q; q.Md = m; q.Nd = n; q.K = n;      // M = M~ V^T
+      three_pairs(q, S.B[0], S.B[1], n, 0, L.Vh, L.Vl, n, 0); store_f32(q); P->back2.push_back(q); }
+    { TcProblem q; q.Md = m; q.Nd = n; q.K = n;      // M~ = M V
+      three_pairs(q, S.B[0], S.B[1], n, 0, L.Vh, L.Vl, n, 1); store_f32(q); P->fwd2.push_back(q); }
+  }
+}
+
+void destroy(RxPlans& r) {
+  for (TcPlan* p : {r.back1, r.back2, r.fwd1, r.fwd2}) tc_plan_destroy(p);
+  r = RxPlans{};
+}
+
+}  // namespace
+
+struct TcStep {
+  std::vector<Chunk> chunks;
+  std::vector<TcPlan*> factor_plan;   // per layer, BR_ACCUM_ON_REFRESH only
+  std::vector<int> chunk_of, slot_of; // per layer: its chunk and its position in the chunk
+  std::string err;
+};
+
+size_t tc_step_scratch_bytes(const std::vector<Layer>& layers, const br_hparams& hp) {
+  size_t worst = 0;
+  for (const auto& ids : make_chunks(layers, hp)) {
+    size_t b = 0;
+    for (int i : ids) b += layer_scratch_bytes(layers[i]);
+    worst = std::max(worst, b);
+  }
+  return worst;
+}
+
+void tc_step_destroy(TcStep* t) {
+  if (!t) return;
+  for (Chunk& c : t->chunks) {
+    for (TcPlan* p : {c.factors, c.fwd1, c.adam, c.back1, c.wwrite}) tc_plan_destroy(p);
+    destroy(c.rx);
+    for (RxPlans& r : c.rx_layer) destroy(r);
+  }
+  for (TcPlan* p : t->factor_plan) tc_plan_destroy(p);
+  delete t;
+}
+
 TcStep* tc_step_create(std::vector<Layer>& layers, const br_hparams& hp, char* scratch, size_t bytes,
                        int device, cudaStream_t s, const char** err) {
   static thread_local std::string last;
@@ -121,9 +259,18 @@ TcStep* tc_step_create(std::vector<Layer>& layers, const br_hparams& hp, char* s
   if (!tc_supported(device)) { last = "tensor-core path needs an sm_100 device and cuTensorMapEncodeTiled"; if (err) *err = last.c_str(); return nullptr; }
   TcStep* t = new TcStep();
   t->factor_plan.assign(layers.size(), nullptr);
+  t->chunk_of.assign(layers.size(), -1);
+  t->slot_of.assign(layers.size(), -1);
   const float beta_f = hp.beta_factor < 0.f ? hp.beta2 : hp.beta_factor;
+  const char* perr = nullptr;
+  auto build = [&](std::vector<TcProblem>& v, TcPlan** dst) -> bool {
+    if (v.empty()) return true;
+    *dst = tc_plan_create(v.data(), (int)v.size(), device, s, &perr);
+    return *dst != nullptr;
+  };
   for (const auto& ids : chunk_ids) {
-    Chunk c;
+    t->chunks.emplace_back();
+    Chunk& c = t->chunks.back();
     c.ids = ids;
     size_t off = 0;
     auto take = [&](size_t numel) {
@@ -131,112 +278,32 @@ TcStep* tc_step_create(std::vector<Layer>& layers, const br_hparams& hp, char* s
       off += align_up(numel * 2);
       return p;
     };
-    std::vector<TcProblem> factors, fwd1, v2, scale, back1, wwrite;
-    for (int i : ids) {
-      const Layer& L = layers[i];
-      const int64_t m = L.d.m, n = L.d.n, mn = m * n;
+    StepProblems P;
+    RxProblems R;
+    c.rx_layer.resize(ids.size());
+    for (size_t j = 0; j < ids.size(); ++j) {
+      const Layer& L = layers[ids[j]];
+      t->chunk_of[ids[j]] = (int)t->chunks.size() - 1;
+      t->slot_of[ids[j]] = (int)j;
+      const int64_t mn = L.d.m * L.d.n;
       LayerScratch S;
-      S.Mh = take(mn); S.Ml = take(mn); S.X = take(mn);
-      if (L.left && L.right) { S.TGh = take(mn); S.TGl = take(mn); S.TMh = take(mn); S.TMl = take(mn); }
+      const int nb = (L.left && L.right) ? 4 : 2;
+      for (int b = 0; b < nb; ++b) S.B[b] = take(mn);
       c.scr.push_back(S);
-      const int tm = L.d.tau_max;
-      if (L.d.src == BR_SRC_SECOND && hp.accum == BR_ACCUM_EVERY_STEP) factor_problems(L, beta_f, &factors);
-      if (L.left && L.right) {
-        {  // T_G = U^T G : (Uh, G) + (Ul, G); U and G both enter MN-major (contraction over rows)
-          TcProblem q; q.Md = m; q.Nd = n; q.K = m; q.n_pairs = 2; q.tau_max = tm;
-          q.A[0] = op(L.Uh, m, 1); q.B[0] = ring_op(L, 1);
-          q.A[1] = op(L.Ul, m, 1); q.B[1] = ring_op(L, 1);
-          q.epilogue = EPI_SPLIT_BF16; q.Dh = S.TGh; q.Dl = S.TGl; q.ldh = n;
-          fwd1.push_back(q);
-        }
-        {  // T_M = U^T M : (Uh, Mh) + (Ul, Mh) + (Uh, Ml)
-          TcProblem q; q.Md = m; q.Nd = n; q.K = m; q.n_pairs = 3; q.tau_max = tm;
-          q.A[0] = op(L.Uh, m, 1); q.B[0] = op(S.Mh, n, 1);
-          q.A[1] = op(L.Ul, m, 1); q.B[1] = op(S.Mh, n, 1);
-          q.A[2] = op(L.Uh, m, 1); q.B[2] = op(S.Ml, n, 1);
-          q.epilogue = EPI_SPLIT_BF16; q.Dh = S.TMh; q.Dl = S.TMl; q.ldh = n;
-          fwd1.push_back(q);
-        }
-        for (int which = 0; which < 2; ++which) {   // (T V): T K-major, V MN-major
-          TcProblem q; q.Md = m; q.Nd = n; q.K = n; q.n_pairs = 3; q.tau_max = tm;
-          const __nv_bfloat16* Th = which ? S.TMh : S.TGh;
-          const __nv_bfloat16* Tl = which ? S.TMl : S.TGl;
-          q.A[0] = op(Th, n, 0); q.B[0] = op(L.Vh, n, 1);
-          q.A[1] = op(Tl, n, 0); q.B[1] = op(L.Vh, n, 1);
-          q.A[2] = op(Th, n, 0); q.B[2] = op(L.Vl, n, 1);
-          q.D = L.V2; q.ldd = n;
-          if (!which) { q.epilogue = EPI_SECOND_MOMENT; q.alpha = 1.f - hp.beta2; q.beta = hp.beta2; v2.push_back(q); }
-          else { q.epilogue = EPI_SCALE_BF16; q.eps = hp.eps; q.Dh = S.X; q.ldh = n; scale.push_back(q); }
-        }
-        {  // Y = U X : U K-major, X MN-major; Y reuses the T_G buffer
-          TcProblem q; q.Md = m; q.Nd = n; q.K = m; q.n_pairs = 1; q.tau_max = tm;
-          q.A[0] = op(L.Uh, m, 0); q.B[0] = op(S.X, n, 1);
-          q.epilogue = EPI_SPLIT_BF16; q.Dh = S.TGh; q.Dl = nullptr; q.ldh = n;
-          back1.push_back(q);
-        }
-        {  // W <- decay W - eta Y V^T : both K-major
-          TcProblem q; q.Md = m; q.Nd = n; q.K = n; q.n_pairs = 1; q.tau_max = tm;
-          q.A[0] = op(S.TGh, n, 0); q.B[0] = op(L.Vh, n, 0);
-          q.epilogue = EPI_AXPBY_F32; q.dyn_scalars = 1; q.D = L.d.weight; q.ldd = n;
-          wwrite.push_back(q);
-        }
-      } else if (L.left) {
-        {  // V~ from U^T G
-          TcProblem q; q.Md = m; q.Nd = n; q.K = m; q.n_pairs = 2; q.tau_max = tm;
-          q.A[0] = op(L.Uh, m, 1); q.B[0] = ring_op(L, 1);
-          q.A[1] = op(L.Ul, m, 1); q.B[1] = ring_op(L, 1);
-          q.epilogue = EPI_SECOND_MOMENT; q.alpha = 1.f - hp.beta2; q.beta = hp.beta2; q.D = L.V2; q.ldd = n;
-          v2.push_back(q);
-        }
-        {  // X from U^T M
-          TcProblem q; q.Md = m; q.Nd = n; q.K = m; q.n_pairs = 3; q.tau_max = tm;
-          q.A[0] = op(L.Uh, m, 1); q.B[0] = op(S.Mh, n, 1);
-          q.A[1] = op(L.Ul, m, 1); q.B[1] = op(S.Mh, n, 1);
-          q.A[2] = op(L.Uh, m, 1); q.B[2] = op(S.Ml, n, 1);
-          q.epilogue = EPI_SCALE_BF16; q.eps = hp.eps; q.D = L.V2; q.ldd = n; q.Dh = S.X; q.ldh = n;
-          scale.push_back(q);
-        }
-        {  // W <- decay W - eta U X
-          TcProblem q; q.Md = m; q.Nd = n; q.K = m; q.n_pairs = 1; q.tau_max = tm;
-          q.A[0] = op(L.Uh, m, 0); q.B[0] = op(S.X, n, 1);
-          q.epilogue = EPI_AXPBY_F32; q.dyn_scalars = 1; q.D = L.d.weight; q.ldd = n;
-          wwrite.push_back(q);
-        }
-      } else {
-        {  // V~ from G V
-          TcProblem q; q.Md = m; q.Nd = n; q.K = n; q.n_pairs = 2; q.tau_max = tm;
-          q.A[0] = ring_op(L, 0); q.B[0] = op(L.Vh, n, 1);
-          q.A[1] = ring_op(L, 0); q.B[1] = op(L.Vl, n, 1);
-          q.epilogue = EPI_SECOND_MOMENT; q.alpha = 1.f - hp.beta2; q.beta = hp.beta2; q.D = L.V2; q.ldd = n;
-          v2.push_back(q);
-        }
-        {  // X from M V
-          TcProblem q; q.Md = m; q.Nd = n; q.K = n; q.n_pairs = 3; q.tau_max = tm;
-          q.A[0] = op(S.Mh, n, 0); q.B[0] = op(L.Vh, n, 1);
-          q.A[1] = op(S.Ml, n, 0); q.B[1] = op(L.Vh, n, 1);
-          q.A[2] = op(S.Mh, n, 0); q.B[2] = op(L.Vl, n, 1);
-          q.epilogue = EPI_SCALE_BF16; q.eps = hp.eps; q.D = L.V2; q.ldd = n; q.Dh = S.X; q.ldh = n;
-          scale.push_back(q);
-        }
-        {  // W <- decay W - eta X V^T
-          TcProblem q; q.Md = m; q.Nd = n; q.K = n; q.n_pairs = 1; q.tau_max = tm;
-          q.A[0] = op(S.X, n, 0); q.B[0] = op(L.Vh, n, 0);
-          q.epilogue = EPI_AXPBY_F32; q.dyn_scalars = 1; q.D = L.d.weight; q.ldd = n;
-          wwrite.push_back(q);
-        }
-      }
+      if (off > bytes) return fail(t, "tensor-core scratch is smaller than the plan needs");
+      if (L.d.src == BR_SRC_SECOND && hp.accum == BR_ACCUM_EVERY_STEP) factor_problems(L, beta_f, &P.factors);
+      step_problems(L, S, hp, &P);
+      rx_problems(L, S, &R);
+      RxProblems one;
+      rx_problems(L, S, &one);
+      RxPlans& r = c.rx_layer[j];
+      if (!build(one.back1, &r.back1) || !build(one.back2, &r.back2) || !build(one.fwd1, &r.fwd1) ||
+          !build(one.fwd2, &r.fwd2))
+        return fail(t, perr ? perr : "plan creation failed");
     }
-    if (off > bytes) return fail(t, "tensor-core scratch is smaller than the plan needs");
-    const char* perr = nullptr;
-    auto build = [&](std::vector<TcProblem>& v, TcPlan** dst) -> bool {
-      if (v.empty()) return true;
-      *dst = tc_plan_create(v.data(), (int)v.size(), device, s, &perr);
-      return *dst != nullptr;
-    };
-    t->chunks.push_back(c);
-    Chunk& cc = t->chunks.back();
-    if (!build(factors, &cc.factors) || !build(fwd1, &cc.fwd1) || !build(v2, &cc.v2) || !build(scale, &cc.scale) ||
-        !build(back1, &cc.back1) || !build(wwrite, &cc.wwrite))
+    if (!build(P.factors, &c.factors) || !build(P.fwd1, &c.fwd1) || !build(P.adam, &c.adam) ||
+        !build(P.back1, &c.back1) || !build(P.wwrite, &c.wwrite) || !build(R.back1, &c.rx.back1) ||
+        !build(R.back2, &c.rx.back2) || !build(R.fwd1, &c.rx.fwd1) || !build(R.fwd2, &c.rx.fwd2))
       return fail(t, perr ? perr : "plan creation failed");
   }
   if (hp.accum == BR_ACCUM_ON_REFRESH) {
@@ -245,7 +312,6 @@ TcStep* tc_step_create(std::vector<Layer>& layers, const br_hparams& hp, char* s
       if (!L.use_tc || L.d.src != BR_SRC_SECOND) continue;
       std::vector<TcProblem> f;
       factor_problems(L, beta_f, &f);
-      const char* perr = nullptr;
       if (!f.empty() && !(t->factor_plan[i] = tc_plan_create(f.data(), (int)f.size(), device, s, &perr)))
         return fail(t, perr ? perr : "plan creation failed");
     }
@@ -253,59 +319,110 @@ TcStep* tc_step_create(std::vector<Layer>& layers, const br_hparams& hp, char* s
   return t;
 }
 
-int tc_step_run(TcStep* t, std::vector<Layer>& layers, const std::vector<const void*>& G, long long calls,
-                int tau, const br_hparams& hp, int* d_status, cudaStream_t s, LaunchStats* stats,
-                const TcStepCallbacks& cb, const char** err) {
-  static thread_local std::string last;
-  auto cuda_fail = [&](const char* what, cudaError_t e) {
+namespace {
+
+struct Launcher {
+  int* d_status; cudaStream_t s; LaunchStats* stats; const char** err;
+  int fail(const char* what, cudaError_t e) {
+    static thread_local std::string last;
     last = std::string(what) + ": " + cudaGetErrorString(e);
     if (err) *err = last.c_str();
     return (int)BR_ERR_CUDA;
-  };
+  }
+  int run(TcPlan* p, const char* what, long long calls, int tau, float a, float b) {
+    if (!p) return 0;
+    const int span = stats->prof.begin(PROF_TC, s);
+    cudaError_t e = tc_plan_launch(p, calls, tau, a, b, d_status, s);
+    stats->prof.end(span, s, tc_plan_flops(p));
+    if (e != cudaSuccess) return fail(what, e);
+    stats->launches += 1;
+    stats->gemm_flops += tc_plan_flops(p);
+    return 0;
+  }
+  // re-expression plans read no ring and skip no layer: calls = 1, tau = 0 makes every problem active
+  int run_rx(TcPlan* p, const char* what) { return run(p, what, 1, 0, 1.f, 0.f); }
+};
+
+// One direction of the re-expression for the layers at the given positions of chunk c.
+int reexpress_chunk(Chunk& c, std::vector<Layer>& layers, const std::vector<int>& slots, bool forward,
+                    Launcher& lz) {
+  for (int j : slots) {
+    const Layer& L = layers[c.ids[j]];
+    cudaError_t e = split_bf16(L.M, c.scr[j].B[0], c.scr[j].B[1], L.d.m * L.d.n, lz.s);
+    if (e != cudaSuccess) return lz.fail("split_bf16", e);
+    lz.stats->launches += 1;
+  }
+  int rc;
+  if (slots.size() == c.ids.size()) {
+    if ((rc = lz.run_rx(forward ? c.rx.fwd1 : c.rx.back1, "re-expression, first side"))) return rc;
+    if ((rc = lz.run_rx(forward ? c.rx.fwd2 : c.rx.back2, "re-expression, second side"))) return rc;
+  } else {
+    for (int j : slots) {
+      RxPlans& r = c.rx_layer[j];
+      if ((rc = lz.run_rx(forward ? r.fwd1 : r.back1, "re-expression, first side"))) return rc;
+      if ((rc = lz.run_rx(forward ? r.fwd2 : r.back2, "re-expression, second side"))) return rc;
+    }
+  }
+  return 0;
+}
+
+}  // namespace
+
+int tc_step_reexpress(TcStep* t, std::vector<Layer>& layers, const int* ids, int n, int forward, int* d_status,
+                      cudaStream_t s, LaunchStats* stats, const char** err) {
+  if (!t) return 0;
+  Launcher lz{d_status, s, stats, err};
+  for (size_t ci = 0; ci < t->chunks.size(); ++ci) {
+    std::vector<int> slots;
+    for (int k = 0; k < n; ++k)
+      if (ids[k] >= 0 && ids[k] < (int)layers.size() && t->chunk_of[ids[k]] == (int)ci) slots.push_back(t->slot_of[ids[k]]);
+    if (slots.empty()) continue;
+    std::sort(slots.begin(), slots.end());
+    int rc = reexpress_chunk(t->chunks[ci], layers, slots, forward != 0, lz);
+    if (rc) return rc;
+  }
+  return 0;
+}
+
+int tc_step_run(TcStep* t, std::vector<Layer>& layers, const std::vector<const void*>& G, long long calls,
+                int tau, const br_hparams& hp, int* d_status, cudaStream_t s, LaunchStats* stats,
+                const TcStepCallbacks& cb, const char** err) {
+  Launcher lz{d_status, s, stats, err};
   const float dyn_alpha = -hp.lr, dyn_beta = 1.0f - hp.lr * hp.weight_decay;
   for (Chunk& c : t->chunks) {
     bool any = false;
-    for (size_t j = 0; j < c.ids.size(); ++j) {
-      Layer& L = layers[c.ids[j]];
-      const void* g = G[c.ids[j]];
-      if (!g) continue;
-      any = true;
-      // Alg. 1 line 4, with the bf16 hi/lo pair of the new M for the rotation
-      const int span = stats->prof.begin(PROF_EMA, s);
-      cudaError_t e = ema_momentum(L.M, g, 1, L.d.m * L.d.n, hp.beta1, nullptr, c.scr[j].Mh, c.scr[j].Ml, s);
-      stats->prof.end(span, s, 14.0 * (double)L.d.m * (double)L.d.n);
-      if (e != cudaSuccess) return cuda_fail("ema_momentum", e);
-      stats->launches += 1;
-    }
+    for (int i : c.ids) any = any || G[i] != nullptr;
     if (!any) continue;
-    auto launch = [&](TcPlan* p, const char* what) -> int {
-      if (!p) return 0;
-      const int span = stats->prof.begin(PROF_TC, s);
-      cudaError_t e = tc_plan_launch(p, calls, tau, dyn_alpha, dyn_beta, d_status, s);
-      stats->prof.end(span, s, tc_plan_flops(p));
-      if (e != cudaSuccess) return cuda_fail(what, e);
-      stats->launches += 1;
-      stats->gemm_flops += tc_plan_flops(p);
-      return 0;
-    };
     int rc;
-    if ((rc = launch(c.factors, "factor launch"))) return rc;
-    std::vector<int> due;
-    for (int i : c.ids) {
+    if ((rc = lz.run(c.factors, "factor launch", calls, tau, dyn_alpha, dyn_beta))) return rc;
+    std::vector<int> due, due_slots;
+    for (size_t j = 0; j < c.ids.size(); ++j) {
+      const int i = c.ids[j];
       Layer& L = layers[i];
       if (!G[i] || L.t % L.freq != 0) continue;
-      if (t->factor_plan[i] && (rc = launch(t->factor_plan[i], "factor launch"))) return rc;
+      if (t->factor_plan[i] && (rc = lz.run(t->factor_plan[i], "factor launch", calls, tau, dyn_alpha, dyn_beta))) return rc;
       due.push_back(i);
+      due_slots.push_back((int)j);
     }
     if (!due.empty()) {
+      // M_{t-1} = U M~_{t-1} V^T with the old basis; S = 1st refreshes from M_t = b1 M_{t-1} + (1-b1) G
+      if ((rc = reexpress_chunk(c, layers, due_slots, false, lz))) return rc;
+      for (int i : due) {
+        Layer& L = layers[i];
+        if (L.d.src != BR_SRC_FIRST) continue;
+        cudaError_t e = ema_out(L.Morig, L.M, G[i], L.d.grad_dtype == BR_BF16, L.d.m * L.d.n, hp.beta1, s);
+        if (e != cudaSuccess) return lz.fail("ema_out", e);
+        stats->launches += 1;
+      }
       rc = cb.refresh(cb.ctx, due.data(), (int)due.size());
       if (rc != 0) { if (err) *err = nullptr; return rc; }
+      // M~_{t-1} = U^T M_{t-1} V with the new basis
+      if ((rc = reexpress_chunk(c, layers, due_slots, true, lz))) return rc;
     }
-    if ((rc = launch(c.fwd1, "first-side rotation launch"))) return rc;
-    if ((rc = launch(c.v2, "second-moment launch"))) return rc;
-    if ((rc = launch(c.scale, "scaling launch"))) return rc;
-    if ((rc = launch(c.back1, "back-rotation launch"))) return rc;
-    if ((rc = launch(c.wwrite, "weight-write launch"))) return rc;
+    if ((rc = lz.run(c.fwd1, "first-side rotation launch", calls, tau, dyn_alpha, dyn_beta))) return rc;
+    if ((rc = lz.run(c.adam, "rotated-Adam launch", calls, tau, dyn_alpha, dyn_beta))) return rc;
+    if ((rc = lz.run(c.back1, "back-rotation launch", calls, tau, dyn_alpha, dyn_beta))) return rc;
+    if ((rc = lz.run(c.wwrite, "weight-write launch", calls, tau, dyn_alpha, dyn_beta))) return rc;
   }
   return 0;
 }

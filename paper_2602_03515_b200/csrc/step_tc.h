@@ -12,7 +12,10 @@ struct Layer {
   bool left = false, right = false;   // which sides carry a rotation
   bool use_tc = false;                // contractions run on the tcgen05 tile kernel
   int freq = 1;
+  // M holds the momentum of Alg. 1 line 4: in the original space on the fp32 path, in ROTATED
+  // coordinates (M~ = U^T M V) on the tensor-core path (see step_tc.cu)
   float *M = nullptr, *V2 = nullptr, *U = nullptr, *V = nullptr, *L = nullptr, *R = nullptr;
+  float* Morig = nullptr;             // tensor-core layers with S = 1st: M_t in the original space for a refresh
   __nv_bfloat16 *Uh = nullptr, *Ul = nullptr, *Vh = nullptr, *Vl = nullptr;  // bf16 hi/lo of U, V
   char* ring = nullptr;
   int ring_slots = 0;                 // physical slots: tau_max, or 1 for a tensor-core layer without delay
@@ -45,6 +48,10 @@ TcStep* tc_step_create(std::vector<Layer>& layers, const br_hparams& hp, char* s
 int tc_step_run(TcStep* t, std::vector<Layer>& layers, const std::vector<const void*>& G, long long calls,
                 int tau, const br_hparams& hp, int* d_status, cudaStream_t s, LaunchStats* stats,
                 const TcStepCallbacks& cb, const char** err);
+// Re-express the momentum buffer of the given tensor-core layers in place: forward = 0 turns M~ into
+// M = U M~ V^T, forward = 1 turns M into M~ = U^T M V, with the bases as they are at that point.
+int tc_step_reexpress(TcStep* t, std::vector<Layer>& layers, const int* ids, int n, int forward, int* d_status,
+                      cudaStream_t s, LaunchStats* stats, const char** err);
 void tc_step_destroy(TcStep* t);
 
 }  // namespace br

@@ -139,6 +139,8 @@ struct TcProblem {
   int32_t epilogue = EPI_AXPBY_F32;
   int32_t tau_max = 0;            // of the layer (delay bookkeeping on the device)
   int32_t dyn_scalars = 0;        // 1: alpha / beta come from the launch arguments
+  int32_t symmetric = 0;          // 1: A_p = B_p and D is square: only tiles touching the upper triangle are
+                                  // computed, the rest of D is written as their mirror image (EPI_AXPBY_F32 only)
   float alpha = 1.f, beta = 0.f, eps = 0.f, beta1 = 0.f;
   float* D = nullptr; int64_t ldd = 0;                                   // fp32 in/out
   float* D2 = nullptr;                                                   // second fp32 in/out (same ld)

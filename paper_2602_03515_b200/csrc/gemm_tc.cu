@@ -38,7 +38,7 @@ constexpr int STAGES = 4;
 constexpr int A_BYTES = BM * BK * 2;             // 16 KiB
 constexpr int B_BYTES = BN * BK * 2;             // 32 KiB
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-constexpr int EPI_LD = 36;                       // padded row of an epilogue tile (floats): 16-byte rows, no bank conflicts
+constexpr int EPI_LD = 33;                       // padded row of an epilogue tile (floats): rows and columns both conflict-free
 constexpr int EPI_BYTES = 4 * 32 * EPI_LD * 4;   // one 32 x 32 fp32 tile per epilogue warp
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BYTES + 1024;   // + slack to align the tiles to 1 KiB
 constexpr int TMEM_COLS = 512;
@@ -60,6 +60,7 @@ struct alignas(128) DevProblem {
   __nv_bfloat16* Dl;
   long long ldh;
   float* D2;
+  int32_t symmetric, pad0_, pad1_, pad2_;
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -215,6 +216,8 @@ __device__ __forceinline__ TileInfo locate_tile(const DevProblem* probs, int n_p
   // apply sits in ring slot (calls - 1 - tau) mod slots
   const int tl = tau < 0 ? p->tau_max : tau;
   ti.active = (calls - tl >= 1);
+  // a symmetric product is computed on the tiles that touch the upper triangle only
+  if (p->symmetric && ti.m0 >= ti.n0 + BN) ti.active = false;
   ti.z = 0;
   if (p->ring_slots > 0 && ti.active) ti.z = (int)((calls - 1 - tl) % p->ring_slots);
   return ti;
@@ -344,7 +347,10 @@ k_tc_gemm(const DevProblem* __restrict__ probs, int n_probs, int total_tiles, lo
     // A warp may read only its own quadrant of tensor memory, where lane = accumulator row: a
     // 32 x 32 block arrives with one row per lane.  It is turned through a padded shared-memory
     // tile so that global memory is accessed along rows: 8 lanes cover 128 contiguous bytes of one
-    // row, a warp instruction four whole rows.
+    // row, a warp instruction four whole rows.  The values a read-modify-write epilogue needs are
+    // prefetched into L2 while the main loop of the tile is still running and then loaded eight
+    // rows deep before the first one is used.  A symmetric product (the factor EMAs) writes its
+    // strictly-upper blocks a second time, transposed, instead of computing the lower triangle.
     const int quad = warp & 3;                    // tensor-memory lane quadrant this warp may read
     float* tile = epi_tiles + quad * (32 * EPI_LD);
     const int sub_r = lane >> 3, sub_c = (lane & 7) * 4;
@@ -353,83 +359,170 @@ k_tc_gemm(const DevProblem* __restrict__ probs, int n_probs, int total_tiles, lo
       const TileInfo ti = locate_tile(probs, n_probs, tile_i, calls, tau);
       if (!ti.active) continue;
       const DevProblem* p = ti.p;
-      if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag, status)) break;
-      tc_fence_after();
       const float alpha = p->dyn_scalars ? dyn_alpha : p->alpha;
       const float beta = p->dyn_scalars ? dyn_beta : p->beta;
       const float eps = p->eps;
       const int epi = p->epilogue;
       const int row_base = ti.m0 + quad * 32;
       const bool quad_ok = row_base < p->Md;      // uniform across the warp
+      const bool reads_d = (epi == EPI_AXPBY_F32 && beta != 0.0f) || epi == EPI_ROTATED_ADAM ||
+                           epi == EPI_SECOND_MOMENT || epi == EPI_SCALE_BF16;
+      if (reads_d && row_base + lane < p->Md) {
+        const float* d = p->D + (long long)(row_base + lane) * p->ldd + ti.n0;
+#pragma unroll
+        for (int q = 0; q < BN / 32; ++q)
+          if (ti.n0 + 32 * q < p->Nd) {
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(d + 32 * q));
+            if (epi == EPI_ROTATED_ADAM)
+              asm volatile("prefetch.global.L2 [%0];" ::"l"(p->D2 + (long long)(row_base + lane) * p->ldd + ti.n0 + 32 * q));
+          }
+      }
+      if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag, status)) break;
+      tc_fence_after();
 #pragma unroll 1
       for (int c0 = 0; c0 < BN; c0 += 32) {
-        if (ti.n0 + c0 >= p->Nd) break;           // uniform across the warp
+        const int col0 = ti.n0 + c0;
+        if (col0 >= p->Nd) break;                 // uniform across the warp
         float v[32];
         tmem_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * BN + c0), v);
-        if (!quad_ok) continue;
+        // nothing to write: rows beyond the matrix, or a block strictly below the diagonal of a
+        // symmetric product (its mirror image is written by the block above the diagonal)
+        if (!quad_ok || (p->symmetric && row_base >= col0 + 32)) continue;
         __syncwarp();
 #pragma unroll
-        for (int q = 0; q < 8; ++q)
-          *reinterpret_cast<float4*>(tile + lane * EPI_LD + 4 * q) = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+        for (int j = 0; j < 32; ++j) tile[lane * EPI_LD + j] = v[j];
         __syncwarp();
-        const int col = ti.n0 + c0 + sub_c;
-        // columns come in multiples of 8: a float4 is all in or all out
-        const int n_it = (col < p->Nd) ? 8 : 0;
-#pragma unroll 2
-        for (int it = 0; it < n_it; ++it) {
-          const int rl = it * 4 + sub_r;
-          const int row = row_base + rl;
-          if (row >= p->Md) break;
-          const float4 a = *reinterpret_cast<const float4*>(tile + rl * EPI_LD + sub_c);
-          if (epi == EPI_AXPBY_F32) {
-            float* d = p->D + (long long)row * p->ldd + col;
-            float4 o = make_float4(alpha * a.x, alpha * a.y, alpha * a.z, alpha * a.w);
-            if (beta != 0.0f) {
-              const float4 old = *reinterpret_cast<const float4*>(d);
-              o.x = fmaf(beta, old.x, o.x); o.y = fmaf(beta, old.y, o.y);
-              o.z = fmaf(beta, old.z, o.z); o.w = fmaf(beta, old.w, o.w);
+        const int col = col0 + sub_c;
+        // columns come in multiples of 8: a group of four is all in or all out
+        int n_it = 0;
+        if (col < p->Nd) { n_it = (p->Md - row_base - sub_r + 3) >> 2; n_it = n_it > 8 ? 8 : n_it; }
+        float4 a[8];
+#pragma unroll
+        for (int it = 0; it < 8; ++it) {
+          const float* t4 = tile + (it * 4 + sub_r) * EPI_LD + sub_c;
+          a[it] = make_float4(t4[0], t4[1], t4[2], t4[3]);
+        }
+        if (epi == EPI_AXPBY_F32) {
+          float* d = p->D + (long long)(row_base + sub_r) * p->ldd + col;
+          const long long step = 4 * p->ldd;
+          float4 old[8];
+          if (beta != 0.0f) {
+#pragma unroll
+            for (int it = 0; it < 8; ++it)
+              if (it < n_it) old[it] = *reinterpret_cast<const float4*>(d + it * step);
+          }
+#pragma unroll
+          for (int it = 0; it < 8; ++it) {
+            float4 o = make_float4(alpha * a[it].x, alpha * a[it].y, alpha * a[it].z, alpha * a[it].w);
+            if (beta != 0.0f && it < n_it) {
+              o.x = fmaf(beta, old[it].x, o.x); o.y = fmaf(beta, old[it].y, o.y);
+              o.z = fmaf(beta, old[it].z, o.z); o.w = fmaf(beta, old[it].w, o.w);
             }
-            *reinterpret_cast<float4*>(d) = o;
-          } else if (epi == EPI_ROTATED_ADAM) {
-            float* d = p->D + (long long)row * p->ldd + col;      // V~
-            float* m2 = p->D2 + (long long)row * p->ldd + col;    // M~
-            const float b1 = p->beta1, ob1 = 1.0f - p->beta1;
-            float4 mm = *reinterpret_cast<const float4*>(m2);
-            float4 ss = *reinterpret_cast<const float4*>(d);
-            mm.x = b1 * mm.x + ob1 * a.x; mm.y = b1 * mm.y + ob1 * a.y;
-            mm.z = b1 * mm.z + ob1 * a.z; mm.w = b1 * mm.w + ob1 * a.w;
-            ss.x = fmaf(beta, ss.x, alpha * a.x * a.x); ss.y = fmaf(beta, ss.y, alpha * a.y * a.y);
-            ss.z = fmaf(beta, ss.z, alpha * a.z * a.z); ss.w = fmaf(beta, ss.w, alpha * a.w * a.w);
-            *reinterpret_cast<float4*>(m2) = mm;
-            *reinterpret_cast<float4*>(d) = ss;
-            uint2 o;
-            o.x = pack2_bf16(mm.x / sqrtf(ss.x + eps), mm.y / sqrtf(ss.y + eps));
-            o.y = pack2_bf16(mm.z / sqrtf(ss.z + eps), mm.w / sqrtf(ss.w + eps));
-            *reinterpret_cast<uint2*>(p->Dh + (long long)row * p->ldh + col) = o;
-          } else if (epi == EPI_SECOND_MOMENT) {
-            float* d = p->D + (long long)row * p->ldd + col;
-            float4 s4 = *reinterpret_cast<const float4*>(d);
-            s4.x = fmaf(beta, s4.x, alpha * a.x * a.x); s4.y = fmaf(beta, s4.y, alpha * a.y * a.y);
-            s4.z = fmaf(beta, s4.z, alpha * a.z * a.z); s4.w = fmaf(beta, s4.w, alpha * a.w * a.w);
-            *reinterpret_cast<float4*>(d) = s4;
-          } else if (epi == EPI_SCALE_BF16) {
-            const float4 s4 = *reinterpret_cast<const float4*>(p->D + (long long)row * p->ldd + col);
-            uint2 o;
-            o.x = pack2_bf16(a.x / sqrtf(s4.x + eps), a.y / sqrtf(s4.y + eps));
-            o.y = pack2_bf16(a.z / sqrtf(s4.z + eps), a.w / sqrtf(s4.w + eps));
-            *reinterpret_cast<uint2*>(p->Dh + (long long)row * p->ldh + col) = o;
-          } else {  // EPI_SPLIT_BF16
-            const float h0 = __bfloat162float(__float2bfloat16_rn(a.x)), h1 = __bfloat162float(__float2bfloat16_rn(a.y));
-            const float h2 = __bfloat162float(__float2bfloat16_rn(a.z)), h3 = __bfloat162float(__float2bfloat16_rn(a.w));
-            uint2 o;
-            o.x = pack2_bf16(h0, h1); o.y = pack2_bf16(h2, h3);
-            *reinterpret_cast<uint2*>(p->Dh + (long long)row * p->ldh + col) = o;
-            if (p->Dl) {
-              uint2 l;
-              l.x = pack2_bf16(a.x - h0, a.y - h1); l.y = pack2_bf16(a.z - h2, a.w - h3);
-              *reinterpret_cast<uint2*>(p->Dl + (long long)row * p->ldh + col) = l;
+            if (it < n_it) *reinterpret_cast<float4*>(d + it * step) = o;
+            a[it] = o;
+          }
+          if (p->symmetric && col0 >= row_base + 32) {
+            // mirror image: element (r, c) of this block also is element (c, r) of the result
+            __syncwarp();
+#pragma unroll
+            for (int it = 0; it < 8; ++it) {
+              float* t4 = tile + (it * 4 + sub_r) * EPI_LD + sub_c;
+              t4[0] = a[it].x; t4[1] = a[it].y; t4[2] = a[it].z; t4[3] = a[it].w;
+            }
+            __syncwarp();
+            const int mrow0 = col0 + sub_r, mcol = row_base + sub_c;   // transposed block: rows col0.., columns row_base..
+            if (mcol < p->Nd) {
+#pragma unroll
+              for (int it = 0; it < 8; ++it) {
+                const int mrow = mrow0 + it * 4;
+                if (mrow >= p->Md) break;
+                const float* t1 = tile + sub_c * EPI_LD + (it * 4 + sub_r);
+                *reinterpret_cast<float4*>(p->D + (long long)mrow * p->ldd + mcol) =
+                    make_float4(t1[0], t1[EPI_LD], t1[2 * EPI_LD], t1[3 * EPI_LD]);
+              }
             }
           }
+        } else if (epi == EPI_ROTATED_ADAM) {
+          float* d = p->D + (long long)(row_base + sub_r) * p->ldd + col;      // V~
+          float* m2 = p->D2 + (long long)(row_base + sub_r) * p->ldd + col;    // M~
+          __nv_bfloat16* xh = p->Dh + (long long)(row_base + sub_r) * p->ldh + col;
+          const long long step = 4 * p->ldd, steph = 4 * p->ldh;
+          const float b1 = p->beta1, ob1 = 1.0f - p->beta1;
+          float4 mm[8], ss[8];
+#pragma unroll
+          for (int it = 0; it < 8; ++it)
+            if (it < n_it) {
+              mm[it] = *reinterpret_cast<const float4*>(m2 + it * step);
+              ss[it] = *reinterpret_cast<const float4*>(d + it * step);
+            }
+#pragma unroll
+          for (int it = 0; it < 8; ++it)
+            if (it < n_it) {
+              const float4 g = a[it];
+              float4 m = mm[it], q = ss[it];
+              m.x = b1 * m.x + ob1 * g.x; m.y = b1 * m.y + ob1 * g.y;
+              m.z = b1 * m.z + ob1 * g.z; m.w = b1 * m.w + ob1 * g.w;
+              q.x = fmaf(beta, q.x, alpha * g.x * g.x); q.y = fmaf(beta, q.y, alpha * g.y * g.y);
+              q.z = fmaf(beta, q.z, alpha * g.z * g.z); q.w = fmaf(beta, q.w, alpha * g.w * g.w);
+              *reinterpret_cast<float4*>(m2 + it * step) = m;
+              *reinterpret_cast<float4*>(d + it * step) = q;
+              uint2 o;
+              o.x = pack2_bf16(m.x / sqrtf(q.x + eps), m.y / sqrtf(q.y + eps));
+              o.y = pack2_bf16(m.z / sqrtf(q.z + eps), m.w / sqrtf(q.w + eps));
+              *reinterpret_cast<uint2*>(xh + it * steph) = o;
+            }
+        } else if (epi == EPI_SECOND_MOMENT) {
+          float* d = p->D + (long long)(row_base + sub_r) * p->ldd + col;
+          const long long step = 4 * p->ldd;
+          float4 ss[8];
+#pragma unroll
+          for (int it = 0; it < 8; ++it)
+            if (it < n_it) ss[it] = *reinterpret_cast<const float4*>(d + it * step);
+#pragma unroll
+          for (int it = 0; it < 8; ++it)
+            if (it < n_it) {
+              const float4 g = a[it];
+              float4 q = ss[it];
+              q.x = fmaf(beta, q.x, alpha * g.x * g.x); q.y = fmaf(beta, q.y, alpha * g.y * g.y);
+              q.z = fmaf(beta, q.z, alpha * g.z * g.z); q.w = fmaf(beta, q.w, alpha * g.w * g.w);
+              *reinterpret_cast<float4*>(d + it * step) = q;
+            }
+        } else if (epi == EPI_SCALE_BF16) {
+          const float* d = p->D + (long long)(row_base + sub_r) * p->ldd + col;
+          __nv_bfloat16* xh = p->Dh + (long long)(row_base + sub_r) * p->ldh + col;
+          const long long step = 4 * p->ldd, steph = 4 * p->ldh;
+          float4 ss[8];
+#pragma unroll
+          for (int it = 0; it < 8; ++it)
+            if (it < n_it) ss[it] = *reinterpret_cast<const float4*>(d + it * step);
+#pragma unroll
+          for (int it = 0; it < 8; ++it)
+            if (it < n_it) {
+              const float4 g = a[it], q = ss[it];
+              uint2 o;
+              o.x = pack2_bf16(g.x / sqrtf(q.x + eps), g.y / sqrtf(q.y + eps));
+              o.y = pack2_bf16(g.z / sqrtf(q.z + eps), g.w / sqrtf(q.w + eps));
+              *reinterpret_cast<uint2*>(xh + it * steph) = o;
+            }
+        } else {  // EPI_SPLIT_BF16
+          __nv_bfloat16* dh = p->Dh + (long long)(row_base + sub_r) * p->ldh + col;
+          __nv_bfloat16* dl = p->Dl ? p->Dl + (long long)(row_base + sub_r) * p->ldh + col : nullptr;
+          const long long steph = 4 * p->ldh;
+#pragma unroll
+          for (int it = 0; it < 8; ++it)
+            if (it < n_it) {
+              const float4 g = a[it];
+              const float h0 = __bfloat162float(__float2bfloat16_rn(g.x)), h1 = __bfloat162float(__float2bfloat16_rn(g.y));
+              const float h2 = __bfloat162float(__float2bfloat16_rn(g.z)), h3 = __bfloat162float(__float2bfloat16_rn(g.w));
+              uint2 o;
+              o.x = pack2_bf16(h0, h1); o.y = pack2_bf16(h2, h3);
+              *reinterpret_cast<uint2*>(dh + it * steph) = o;
+              if (dl) {
+                uint2 l;
+                l.x = pack2_bf16(g.x - h0, g.y - h1); l.y = pack2_bf16(g.z - h2, g.w - h3);
+                *reinterpret_cast<uint2*>(dl + it * steph) = l;
+              }
+            }
         }
         __syncwarp();                             // the tile is rewritten by the next block
       }
@@ -550,6 +643,9 @@ TcPlan* tc_plan_create(const TcProblem* problems, int n, int device, cudaStream_
     d.tau_max = q.tau_max;
     d.dyn_scalars = q.dyn_scalars;
     d.alpha = q.alpha; d.beta = q.beta; d.eps = q.eps; d.beta1 = q.beta1;
+    d.symmetric = q.symmetric ? 1 : 0;
+    if (q.symmetric && (q.Md != q.Nd || q.epilogue != EPI_AXPBY_F32))
+      return fail("tensor-core problem: a symmetric product needs a square fp32 result");
     d.D = q.D; d.ldd = q.ldd; d.Dh = q.Dh; d.Dl = q.Dl; d.ldh = q.ldh; d.D2 = q.D2;
     const bool need_D = q.epilogue != EPI_SPLIT_BF16;
     const bool need_H = q.epilogue == EPI_SPLIT_BF16 || q.epilogue == EPI_SCALE_BF16 || q.epilogue == EPI_ROTATED_ADAM;
@@ -559,7 +655,16 @@ TcPlan* tc_plan_create(const TcProblem* problems, int n, int device, cudaStream_
         (need_H && (!q.Dh || (q.ldh % 8) || (reinterpret_cast<uintptr_t>(q.Dh) & 15))) ||
         (q.Dl && (reinterpret_cast<uintptr_t>(q.Dl) & 15)))
       return fail("tensor-core problem: output pointer missing or misaligned");
-    flops += 2.0 * (double)q.Md * (double)q.Nd * (double)q.K * q.n_pairs;
+    if (q.symmetric) {
+      // executed work: the tiles that touch the upper triangle
+      int64_t computed = 0;
+      for (int64_t rb = 0; rb < d.tiles_m; ++rb)
+        for (int64_t cb = 0; cb < d.tiles_n; ++cb)
+          if (rb * BM < cb * BN + BN) ++computed;
+      flops += 2.0 * (double)computed * BM * BN * (double)q.K * q.n_pairs;
+    } else {
+      flops += 2.0 * (double)q.Md * (double)q.Nd * (double)q.K * q.n_pairs;
+    }
   }
   TcPlan* plan = new TcPlan();
   plan->n = n;

@@ -97,12 +97,14 @@ void factor_problems(const Layer& L, float beta, std::vector<TcProblem>* out) {
     TcProblem q; q.Md = m; q.Nd = m; q.K = n; q.n_pairs = 1;
     q.A[0] = ring_op(L, 0); q.B[0] = ring_op(L, 0);
     q.epilogue = EPI_AXPBY_F32; q.alpha = 1.f - beta; q.beta = beta; q.D = L.L; q.ldd = m; q.tau_max = L.d.tau_max;
+    q.symmetric = 1;
     out->push_back(q);
   }
   if (L.R) {      // R <- beta R + (1-beta) G^T G : both operands MN-major views of G
     TcProblem q; q.Md = n; q.Nd = n; q.K = m; q.n_pairs = 1;
     q.A[0] = ring_op(L, 1); q.B[0] = ring_op(L, 1);
     q.epilogue = EPI_AXPBY_F32; q.alpha = 1.f - beta; q.beta = beta; q.D = L.R; q.ldd = n; q.tau_max = L.d.tau_max;
+    q.symmetric = 1;
     out->push_back(q);
   }
 }

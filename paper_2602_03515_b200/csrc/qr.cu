@@ -21,7 +21,9 @@
 // on its own output ("twice is enough"), which restores orthogonality to the rounding level.  The
 // second sweep is decided on the device: the first sweep compares the squared norm each column has
 // left when its panel is reached with the squared norm it started with, and clears a flag when the
-// ratio falls below 1e-4; every launch of the second sweep returns at once while the flag is set.
+// ratio falls below 1e-8 (a column that kept less than 1e-4 of its length: one sweep then leaves an
+// orthogonality error of up to ~1e-16 * 1e4^2); every launch of the second sweep returns at once
+// while the flag is set.
 // All reductions are done in a fixed order, so the result is bit-reproducible from run to run.
 #include <algorithm>
 
@@ -37,7 +39,7 @@ inline int64_t cdiv(int64_t a, int64_t b) { return (a + b - 1) / b; }
 inline int panel_width(int64_t k) { return k >= 1024 ? 128 : 64; }
 inline int gram_splits(int64_t k) { return (int)std::min<int64_t>(64, std::max<int64_t>(1, cdiv(k, 128))); }
 inline int proj_splits_max(int64_t k) { return k >= 1024 ? 64 : 1; }
-constexpr double kIllRatio = 1e-4;   // squared-norm ratio below which the second sweep runs
+constexpr double kIllRatio = 1e-8;   // squared-norm ratio below which the second sweep runs
 // sub-buffers of the work area start on 256-byte boundaries
 inline int64_t pad32(int64_t doubles) { return (doubles + 31) / 32 * 32; }
 

@@ -6,6 +6,12 @@
 // that global memory is accessed along rows, and apply a fused epilogue
 // (factor EMA, bf16 hi/lo split, second-moment update, Adam scaling, weight write).
 //
+// A problem may sum several operand pairs into one tile (the bf16 hi/lo products of an fp32
+// operand).  When the pairs are combinations of at most two distinct A and two distinct B operands
+// (hi*hi + lo*hi + hi*lo), the kernel runs in its shared-operand form: a stage holds one k-block of
+// every distinct operand (2 x 16 KiB + 2 x 32 KiB) and all combinations are issued from it, so each
+// operand tile is fetched from L2 once per k-block instead of once per pair.
+//
 // One persistent CTA per SM walks a static tile list that spans every problem of a launch
 // (all layers of one phase of the step), so small and large matrices share one launch.
 // Two 256-column accumulators in tensor memory let the epilogue of a tile overlap the main
@@ -38,6 +44,9 @@ constexpr int STAGES = 4;
 constexpr int A_BYTES = BM * BK * 2;             // 16 KiB
 constexpr int B_BYTES = BN * BK * 2;             // 32 KiB
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int SH_STAGES = 2;                     // shared-operand form: two stages of 2 A tiles + 2 B tiles
+constexpr int SH_STAGE_BYTES = 2 * A_BYTES + 2 * B_BYTES;
+static_assert(SH_STAGES * SH_STAGE_BYTES == STAGES * STAGE_BYTES, "both forms use the same operand area");
 constexpr int EPI_LD = 33;                       // padded row of an epilogue tile (floats): rows and columns both conflict-free
 constexpr int EPI_BYTES = 4 * 32 * EPI_LD * 4;   // one 32 x 32 fp32 tile per epilogue warp
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BYTES + 1024;   // + slack to align the tiles to 1 KiB
@@ -60,7 +69,9 @@ struct alignas(128) DevProblem {
   __nv_bfloat16* Dl;
   long long ldh;
   float* D2;
-  int32_t symmetric, pad0_, pad1_, pad2_;
+  // shared-operand form: mapA[0..nA) / mapB[0..nB) are the distinct operands, `combos` lists the
+  // products to issue per k-block: bits 8.. = count, bits 2c, 2c+1 = (A index, B index) of product c
+  int32_t symmetric, nA, nB, combos;
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -226,9 +237,11 @@ __device__ __forceinline__ TileInfo locate_tile(const DevProblem* probs, int n_p
 // ---------------------------------------------------------------------------------------------
 // The kernel
 // ---------------------------------------------------------------------------------------------
+template <bool SHARED>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 k_tc_gemm(const DevProblem* __restrict__ probs, int n_probs, int total_tiles, long long calls,
           int tau, float dyn_alpha, float dyn_beta, int* status) {
+  constexpr int NST = SHARED ? SH_STAGES : STAGES;
   extern __shared__ uint8_t smem_raw[];
   __shared__ alignas(8) uint64_t bars[2 * STAGES + 4];
   __shared__ uint32_t tmem_slot;
@@ -239,8 +252,15 @@ k_tc_gemm(const DevProblem* __restrict__ probs, int n_probs, int total_tiles, lo
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  auto sA = [&](int s) { return tiles_base + (uint32_t)s * A_BYTES; };
-  auto sB = [&](int s) { return tiles_base + (uint32_t)STAGES * A_BYTES + (uint32_t)s * B_BYTES; };
+  // operand slot i of stage s
+  auto sA = [&](int s, int i) {
+    return SHARED ? tiles_base + (uint32_t)s * SH_STAGE_BYTES + (uint32_t)i * A_BYTES
+                  : tiles_base + (uint32_t)s * A_BYTES;
+  };
+  auto sB = [&](int s, int i) {
+    return SHARED ? tiles_base + (uint32_t)s * SH_STAGE_BYTES + 2u * A_BYTES + (uint32_t)i * B_BYTES
+                  : tiles_base + (uint32_t)STAGES * A_BYTES + (uint32_t)s * B_BYTES;
+  };
   float* epi_tiles = reinterpret_cast<float*>(smem_raw + ((tiles_base - smem_u32(smem_raw)) + (uint32_t)STAGES * STAGE_BYTES));
   const uint32_t bar0 = smem_u32(bars);
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
@@ -249,7 +269,7 @@ k_tc_gemm(const DevProblem* __restrict__ probs, int n_probs, int total_tiles, lo
   auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + 2 + a); };
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int s = 0; s < NST; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
     abort_word = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -273,30 +293,43 @@ k_tc_gemm(const DevProblem* __restrict__ probs, int n_probs, int total_tiles, lo
         const DevProblem* p = ti.p;
         const int nkb = (p->K + BK - 1) / BK;
         bool ok = true;
-        for (int pr = 0; pr < p->n_pairs && ok; ++pr) {
-          const CUtensorMap* ma = &p->mapA[pr];
-          const CUtensorMap* mb = &p->mapB[pr];
-          const int za = ((p->a_ring_mask >> pr) & 1) ? ti.z : 0;
-          const int zb = ((p->b_ring_mask >> pr) & 1) ? ti.z : 0;
+        auto load_a = [&](uint32_t dst, const CUtensorMap* ma, int k0, int za, uint32_t bar) {
+          if (p->a_mn) {
+#pragma unroll
+            for (int j = 0; j < BM / 64; ++j) tma_load_3d(dst + j * (BK * 128), ma, bar, ti.m0 + 64 * j, k0, za);
+          } else {
+            tma_load_3d(dst, ma, bar, k0, ti.m0, za);
+          }
+        };
+        auto load_b = [&](uint32_t dst, const CUtensorMap* mb, int k0, int zb, uint32_t bar) {
+          if (p->b_mn) {
+#pragma unroll
+            for (int j = 0; j < BN / 64; ++j) tma_load_3d(dst + j * (BK * 128), mb, bar, ti.n0 + 64 * j, k0, zb);
+          } else {
+            tma_load_3d(dst, mb, bar, k0, ti.n0, zb);
+          }
+        };
+        if (SHARED) {
           for (int kb = 0; kb < nkb; ++kb) {
             if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, status)) { ok = false; break; }
-            mbar_expect_tx(full_bar(stage), STAGE_BYTES);
-            const int k0 = kb * BK;
-            if (p->a_mn) {
-#pragma unroll
-              for (int j = 0; j < BM / 64; ++j)
-                tma_load_3d(sA(stage) + j * (BK * 128), ma, full_bar(stage), ti.m0 + 64 * j, k0, za);
-            } else {
-              tma_load_3d(sA(stage), ma, full_bar(stage), k0, ti.m0, za);
+            mbar_expect_tx(full_bar(stage), (uint32_t)(p->nA * A_BYTES + p->nB * B_BYTES));
+            for (int i = 0; i < p->nA; ++i)
+              load_a(sA(stage, i), &p->mapA[i], kb * BK, ((p->a_ring_mask >> i) & 1) ? ti.z : 0, full_bar(stage));
+            for (int i = 0; i < p->nB; ++i)
+              load_b(sB(stage, i), &p->mapB[i], kb * BK, ((p->b_ring_mask >> i) & 1) ? ti.z : 0, full_bar(stage));
+            if (++stage == NST) { stage = 0; phase ^= 1u; }
+          }
+        } else {
+          for (int pr = 0; pr < p->n_pairs && ok; ++pr) {
+            const int za = ((p->a_ring_mask >> pr) & 1) ? ti.z : 0;
+            const int zb = ((p->b_ring_mask >> pr) & 1) ? ti.z : 0;
+            for (int kb = 0; kb < nkb; ++kb) {
+              if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, status)) { ok = false; break; }
+              mbar_expect_tx(full_bar(stage), STAGE_BYTES);
+              load_a(sA(stage, 0), &p->mapA[pr], kb * BK, za, full_bar(stage));
+              load_b(sB(stage, 0), &p->mapB[pr], kb * BK, zb, full_bar(stage));
+              if (++stage == NST) { stage = 0; phase ^= 1u; }
             }
-            if (p->b_mn) {
-#pragma unroll
-              for (int j = 0; j < BN / 64; ++j)
-                tma_load_3d(sB(stage) + j * (BK * 128), mb, full_bar(stage), ti.n0 + 64 * j, k0, zb);
-            } else {
-              tma_load_3d(sB(stage), mb, full_bar(stage), k0, ti.n0, zb);
-            }
-            if (++stage == STAGES) { stage = 0; phase ^= 1u; }
           }
         }
         if (!ok) break;
@@ -322,19 +355,25 @@ k_tc_gemm(const DevProblem* __restrict__ probs, int n_probs, int total_tiles, lo
         const uint32_t d_tmem = tmem_base + (uint32_t)acc * BN;
         uint32_t accumulate = 0;
         bool ok = true;
-        for (int it = 0; it < p->n_pairs * nkb; ++it) {
+        const int n_steps = SHARED ? nkb : p->n_pairs * nkb;
+        const int n_combo = SHARED ? (p->combos >> 8) : 1;
+        for (int it = 0; it < n_steps; ++it) {
           if (!mbar_wait(full_bar(stage), phase, abort_flag, status)) { ok = false; break; }
           tc_fence_after();
-          const uint64_t adesc = make_smem_desc(sA(stage), a_lbo, 1024);
-          const uint64_t bdesc = make_smem_desc(sB(stage), b_lbo, 1024);
+          for (int c = 0; c < n_combo; ++c) {
+            const int ai = SHARED ? ((p->combos >> (2 * c)) & 1) : 0;
+            const int bi = SHARED ? ((p->combos >> (2 * c + 1)) & 1) : 0;
+            const uint64_t adesc = make_smem_desc(sA(stage, ai), a_lbo, 1024);
+            const uint64_t bdesc = make_smem_desc(sB(stage, bi), b_lbo, 1024);
 #pragma unroll
-          for (int k = 0; k < BK / UMMA_K; ++k) {
-            umma_bf16(d_tmem, adesc + (uint64_t)((k * a_adv) >> 4), bdesc + (uint64_t)((k * b_adv) >> 4),
-                      idesc, accumulate);
-            accumulate = 1;
+            for (int k = 0; k < BK / UMMA_K; ++k) {
+              umma_bf16(d_tmem, adesc + (uint64_t)((k * a_adv) >> 4), bdesc + (uint64_t)((k * b_adv) >> 4),
+                        idesc, accumulate);
+              accumulate = 1;
+            }
           }
           umma_commit(empty_bar(stage));          // frees the stage once these MMAs have read it
-          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+          if (++stage == NST) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
         umma_commit(tfull_bar(acc));              // accumulator complete
@@ -596,6 +635,7 @@ bool encode_operand(CUtensorMap* map, const TcOperand& op, int64_t rows, int64_t
 }  // namespace
 
 struct TcPlan {
+  bool shared = false;          // launches the shared-operand form of the kernel
   DevProblem* d_probs = nullptr;
   int n = 0;
   int total_tiles = 0;
@@ -614,6 +654,29 @@ TcPlan* tc_plan_create(const TcProblem* problems, int n, int device, cudaStream_
   static thread_local std::string last;
   auto fail = [&](const std::string& m) -> TcPlan* { last = m; if (err) *err = last.c_str(); return nullptr; };
   if (n <= 0) return fail("empty plan");
+  // The shared-operand form pays off when some problem sums several pairs, and applies when every
+  // problem combines at most two distinct A and two distinct B operands.
+  auto same_operand = [](const TcOperand& x, const TcOperand& y) {
+    return x.ptr == y.ptr && x.ld == y.ld && x.mn_major == y.mn_major && x.ring_slots == y.ring_slots &&
+           x.slot_stride_bytes == y.slot_stride_bytes;
+  };
+  bool shared = false, eligible = true;
+  for (int i = 0; i < n; ++i) {
+    const TcProblem& q = problems[i];
+    if (q.n_pairs < 1 || q.n_pairs > MAX_PAIRS) return fail("tensor-core problem: 1 to 3 operand pairs");
+    if (q.n_pairs > 1) shared = true;
+    int nA = 0, nB = 0;
+    for (int p = 0; p < q.n_pairs; ++p) {
+      bool newa = true, newb = true;
+      for (int u = 0; u < p; ++u) {
+        if (same_operand(q.A[u], q.A[p])) newa = false;
+        if (same_operand(q.B[u], q.B[p])) newb = false;
+      }
+      nA += newa; nB += newb;
+    }
+    if (nA > 2 || nB > 2) eligible = false;
+  }
+  shared = shared && eligible;
   std::vector<DevProblem> host(n);
   int tile_begin = 0;
   double flops = 0.0;
@@ -625,13 +688,36 @@ TcPlan* tc_plan_create(const TcProblem* problems, int n, int device, cudaStream_
         (q.Md % 8) || (q.Nd % 8) || (q.K % 8) || q.Md > (1ll << 30) || q.Nd > (1ll << 30) || q.K > (1ll << 30))
       return fail("tensor-core problem: dimensions must be positive multiples of 8");
     std::string e;
-    for (int p = 0; p < q.n_pairs; ++p) {
+    for (int p = 0; p < q.n_pairs; ++p)
       if (q.A[p].mn_major != q.A[0].mn_major || q.B[p].mn_major != q.B[0].mn_major)
         return fail("tensor-core problem: all pairs must share operand majors");
-      if (!encode_operand(&d.mapA[p], q.A[p], q.Md, q.K, BM, &e)) return fail(e);
-      if (!encode_operand(&d.mapB[p], q.B[p], q.Nd, q.K, BN, &e)) return fail(e);
-      if (q.A[p].ring_slots > 0) { d.a_ring_mask |= 1 << p; d.ring_slots = q.A[p].ring_slots; }
-      if (q.B[p].ring_slots > 0) { d.b_ring_mask |= 1 << p; d.ring_slots = q.B[p].ring_slots; }
+    if (shared) {
+      // distinct operands and the list of products
+      int ua[MAX_PAIRS], ub[MAX_PAIRS], nA = 0, nB = 0, combos = 0;
+      for (int p = 0; p < q.n_pairs; ++p) {
+        int ia = -1, ib = -1;
+        for (int u = 0; u < nA; ++u) if (same_operand(q.A[ua[u]], q.A[p])) ia = u;
+        for (int u = 0; u < nB; ++u) if (same_operand(q.B[ub[u]], q.B[p])) ib = u;
+        if (ia < 0) { ia = nA; ua[nA++] = p; }
+        if (ib < 0) { ib = nB; ub[nB++] = p; }
+        combos |= (ia | (ib << 1)) << (2 * p);
+      }
+      for (int u = 0; u < nA; ++u) {
+        if (!encode_operand(&d.mapA[u], q.A[ua[u]], q.Md, q.K, BM, &e)) return fail(e);
+        if (q.A[ua[u]].ring_slots > 0) { d.a_ring_mask |= 1 << u; d.ring_slots = q.A[ua[u]].ring_slots; }
+      }
+      for (int u = 0; u < nB; ++u) {
+        if (!encode_operand(&d.mapB[u], q.B[ub[u]], q.Nd, q.K, BN, &e)) return fail(e);
+        if (q.B[ub[u]].ring_slots > 0) { d.b_ring_mask |= 1 << u; d.ring_slots = q.B[ub[u]].ring_slots; }
+      }
+      d.nA = nA; d.nB = nB; d.combos = combos | (q.n_pairs << 8);
+    } else {
+      for (int p = 0; p < q.n_pairs; ++p) {
+        if (!encode_operand(&d.mapA[p], q.A[p], q.Md, q.K, BM, &e)) return fail(e);
+        if (!encode_operand(&d.mapB[p], q.B[p], q.Nd, q.K, BN, &e)) return fail(e);
+        if (q.A[p].ring_slots > 0) { d.a_ring_mask |= 1 << p; d.ring_slots = q.A[p].ring_slots; }
+        if (q.B[p].ring_slots > 0) { d.b_ring_mask |= 1 << p; d.ring_slots = q.B[p].ring_slots; }
+      }
     }
     d.Md = (int32_t)q.Md; d.Nd = (int32_t)q.Nd; d.K = (int32_t)q.K; d.n_pairs = q.n_pairs;
     d.a_mn = q.A[0].mn_major; d.b_mn = q.B[0].mn_major; d.epilogue = q.epilogue;
@@ -667,6 +753,7 @@ TcPlan* tc_plan_create(const TcProblem* problems, int n, int device, cudaStream_
     }
   }
   TcPlan* plan = new TcPlan();
+  plan->shared = shared;
   plan->n = n;
   plan->total_tiles = tile_begin;
   plan->flops = flops;
@@ -683,7 +770,8 @@ TcPlan* tc_plan_create(const TcProblem* problems, int n, int device, cudaStream_
   }
   static std::once_flag attr_once;
   std::call_once(attr_once, [] {
-    cudaFuncSetAttribute(k_tc_gemm, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    cudaFuncSetAttribute(k_tc_gemm<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    cudaFuncSetAttribute(k_tc_gemm<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
   });
   return plan;
 }
@@ -700,9 +788,15 @@ cudaError_t tc_plan_launch(TcPlan* p, long long calls, int tau, float dyn_alpha,
                            int* status_word, cudaStream_t s) {
   const int grid = p->total_tiles < p->sm_count ? p->total_tiles : p->sm_count;
   // per-device attribute: set again when another device is current (cheap, idempotent)
-  cudaFuncSetAttribute(k_tc_gemm, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
-  k_tc_gemm<<<grid, NUM_THREADS, SMEM_BYTES, s>>>(p->d_probs, p->n, p->total_tiles, calls, tau, dyn_alpha,
-                                                  dyn_beta, status_word);
+  if (p->shared) {
+    cudaFuncSetAttribute(k_tc_gemm<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    k_tc_gemm<true><<<grid, NUM_THREADS, SMEM_BYTES, s>>>(p->d_probs, p->n, p->total_tiles, calls, tau, dyn_alpha,
+                                                          dyn_beta, status_word);
+  } else {
+    cudaFuncSetAttribute(k_tc_gemm<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    k_tc_gemm<false><<<grid, NUM_THREADS, SMEM_BYTES, s>>>(p->d_probs, p->n, p->total_tiles, calls, tau, dyn_alpha,
+                                                           dyn_beta, status_word);
+  }
   return cudaGetLastError();
 }
 

@@ -112,6 +112,12 @@ typedef struct {
   int64_t ring_slot;      /* ring slot the next call writes: calls mod tau_max (0 if no ring) */
   int64_t refresh_count;  /* refreshes done for this layer, scheduled and forced             */
   int64_t next_refresh_t; /* next t with t mod freq == 0                                     */
+  /* Not part of the method's integer state: what the library remembers about the conditioning of
+   * the last refresh of this layer's bases (bit 0: left, bit 1: right; set = no column of F Q shrank
+   * below 1e-3 of its length under orthonormalisation).  The next refresh of a tensor-core layer
+   * runs its block projections on the tensor cores only for a basis whose bit is set.  Saved and
+   * restored with the other counters so that a resumed run takes the same decisions. */
+  int64_t basis_flags;
 } br_counters;
 
 typedef enum {

@@ -11,7 +11,7 @@ from .binding import (  # noqa: F401
     BR_BUF_W, BR_BUF_M, BR_BUF_V2, BR_BUF_U, BR_BUF_V, BR_BUF_L, BR_BUF_R, BR_BUF_RING, BR_BUF_MROT,
     BrError, BrLayerDesc, BrHparams, BrCounters, load_library, library_path,
     br_state_bytes, br_create, br_step, br_set_lr, br_refresh_basis, br_sync_status,
-    br_get_counters, br_set_counters, br_get_state, br_set_state, br_get_launch_stats,
+    br_get_counters, br_get_basis_flags, br_set_counters, br_get_state, br_set_state, br_get_launch_stats,
     br_profile, br_get_profile, br_destroy, br_strerror, br_last_error, br_gemm_bf16, br_power_static,
     BasisRotation,
 )

@@ -41,10 +41,12 @@ class BrHparams(C.Structure):
 
 class BrCounters(C.Structure):
     _fields_ = [("calls", C.c_int64), ("t", C.c_int64), ("ring_slot", C.c_int64),
-                ("refresh_count", C.c_int64), ("next_refresh_t", C.c_int64)]
+                ("refresh_count", C.c_int64), ("next_refresh_t", C.c_int64), ("basis_flags", C.c_int64)]
 
     def as_dict(self):
-        return {k: int(getattr(self, k)) for k, _ in self._fields_}
+        """The integer state of the method (what the oracle also keeps); `basis_flags` is the library's own
+        note on conditioning and is read with br_get_basis_flags."""
+        return {k: int(getattr(self, k)) for k, _ in self._fields_ if k != "basis_flags"}
 
 
 class BrProfileStats(C.Structure):
@@ -166,8 +168,15 @@ def br_get_counters(handle, layer: int) -> dict:
     return c.as_dict()
 
 
-def br_set_counters(handle, layer: int, calls: int, t: int, refresh_count: int) -> int:
-    c = BrCounters(calls=calls, t=t, ring_slot=0, refresh_count=refresh_count, next_refresh_t=0)
+def br_get_basis_flags(handle, layer: int) -> int:
+    c = BrCounters()
+    _check(load_library().br_get_counters(handle, int(layer), C.byref(c)), handle)
+    return int(c.basis_flags)
+
+
+def br_set_counters(handle, layer: int, calls: int, t: int, refresh_count: int, basis_flags: int = 0) -> int:
+    c = BrCounters(calls=calls, t=t, ring_slot=0, refresh_count=refresh_count, next_refresh_t=0,
+                   basis_flags=basis_flags)
     return _check(load_library().br_set_counters(handle, int(layer), C.byref(c)), handle)
 
 

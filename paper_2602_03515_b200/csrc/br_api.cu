@@ -101,11 +101,22 @@ struct br_handle {
     cudaStream_t stream = nullptr;
     cudaEvent_t done = nullptr;
     double *rA = nullptr, *rF = nullptr, *rQ = nullptr, *rZ = nullptr, *rWork = nullptr;
+    char* tcq_scratch = nullptr;          // scratch of the tensor-core projections (largest eligible order)
+    std::vector<QrTc*> tcq;               // their plans, one per distinct eligible order
   };
   static constexpr int kMaxLanes = 3;
   Lane lanes[kMaxLanes];
   int n_lanes = 1;
   cudaEvent_t ev_begin = nullptr;
+  // Conditioning notes of the last refresh, per layer and side (index 2 * layer + (right side)):
+  // written on the device by the refresh, copied to pinned host memory after every batch, read by
+  // the host before the next one (which then decides where the block projections run).
+  int* d_cond = nullptr;
+  int* h_cond = nullptr;
+  std::vector<int> cond_known;
+  cudaEvent_t ev_cond = nullptr;
+  bool cond_pending = false;
+  size_t tcq_bytes = 0;
   // tensor-core path
   TcStep* tc = nullptr;
   LaunchStats stats;
@@ -163,6 +174,12 @@ void layout(br_handle* h, Bump& b, Sizes* sz) {
     h->sGt = b.take<float>(max_numel);
     h->sMt = b.take<float>(max_numel);
   }
+  h->tcq_bytes = 0;
+  for (const Layer& L : h->layers) {
+    if (!L.use_tc) continue;
+    if (L.left) h->tcq_bytes = std::max(h->tcq_bytes, qr_tc_scratch_bytes(L.d.m));
+    if (L.right) h->tcq_bytes = std::max(h->tcq_bytes, qr_tc_scratch_bytes(L.d.n));
+  }
   if (max_k) {
     h->n_lanes = (int)std::min<size_t>(br_handle::kMaxLanes, std::max<size_t>(1, n_sides));
     // tuning aid: BR_REFRESH_LANES=1..3 caps the number of concurrent refresh lanes
@@ -177,8 +194,10 @@ void layout(br_handle* h, Bump& b, Sizes* sz) {
       ln.rQ = b.take<double>(max_k * max_k);
       ln.rWork = b.take<double>(qr_work_doubles((int64_t)max_k));
       if (max_z) ln.rZ = b.take<double>(max_z);
+      if (h->tcq_bytes) ln.tcq_scratch = b.take<char>(h->tcq_bytes);
     }
   }
+  h->d_cond = b.take<int>(2 * h->layers.size() + 2);
   h->d_status = b.take<int>(64);
   (void)hp;
   sz->total = b.off;
@@ -240,7 +259,12 @@ br_status refresh_side(br_handle* h, Layer& L, bool left_side, br_handle::Lane& 
       BR_CUDA(h, fdgemm(1, 0, n, n, m, 1.0, Mo, n, ln.rZ, n, 0.0, ln.rA, n, s));
       count(h, 2); h->stats.gemm_flops += 4.0 * n * n * m;
     }
-    BR_CUDA(h, qr_pos_inplace(ln.rA, k, ln.rWork, h->d_status, s, &h->stats.launches, &h->stats.gemm_flops));
+    const int ci = 2 * (int)(&L - h->layers.data()) + (left_side ? 0 : 1);
+    QrTc* tcq = nullptr;
+    if (L.use_tc && h->cond_known[ci])
+      for (QrTc* t : ln.tcq) if (qr_tc_order(t) == k) tcq = t;
+    BR_CUDA(h, qr_pos_inplace(ln.rA, k, ln.rWork, h->d_status, s, &h->stats.launches, &h->stats.gemm_flops, tcq,
+                              h->d_cond + ci));
     BR_CUDA(h, f64_to_f32(ln.rA, Q, k * k, s));
     count(h);
   }
@@ -262,6 +286,12 @@ br_status refresh_layers(br_handle* h, const int* ids, int n_ids) {
     if (L.right) jobs.push_back({ids[j], false, (double)L.d.n * L.d.n * L.d.n});
   }
   if (jobs.empty()) return BR_OK;
+  if (h->cond_pending) {
+    // the notes of the previous batch: long since on the host unless the two refreshes are back to back
+    BR_CUDA(h, cudaEventSynchronize(h->ev_cond));
+    for (size_t i = 0; i < h->cond_known.size(); ++i) h->cond_known[i] = h->h_cond[i];
+    h->cond_pending = false;
+  }
   std::stable_sort(jobs.begin(), jobs.end(), [](const Job& a, const Job& b) { return a.cost > b.cost; });
   const int nl = (int)std::min<size_t>((size_t)h->n_lanes, jobs.size());
   std::vector<std::vector<Job>> per_lane(nl);
@@ -293,6 +323,9 @@ br_status refresh_layers(br_handle* h, const int* ids, int n_ids) {
     BR_CUDA(h, cudaStreamWaitEvent(h->stream, h->lanes[i].done, 0));
   }
   h->stats.prof.end(span, h->stream, h->stats.gemm_flops - f0);
+  BR_CUDA(h, cudaMemcpyAsync(h->h_cond, h->d_cond, sizeof(int) * h->cond_known.size(), cudaMemcpyDeviceToHost, h->stream));
+  BR_CUDA(h, cudaEventRecord(h->ev_cond, h->stream));
+  h->cond_pending = true;
   for (int j = 0; j < n_ids; ++j) {
     Layer& L = h->layers[ids[j]];
     if (L.left || L.right) L.refresh_count += 1;
@@ -531,6 +564,30 @@ br_status br_create(br_handle** out, const br_layer_desc* layers, int n_layers, 
     if ((e = cudaEventCreateWithFlags(&h->lanes[i].done, cudaEventDisableTiming)) != cudaSuccess) return fail("cudaEventCreate", e);
   }
   if ((e = cudaEventCreateWithFlags(&h->ev_begin, cudaEventDisableTiming)) != cudaSuccess) return fail("cudaEventCreate", e);
+  if ((e = cudaEventCreateWithFlags(&h->ev_cond, cudaEventDisableTiming)) != cudaSuccess) return fail("cudaEventCreate", e);
+  h->cond_known.assign(2 * h->layers.size(), 0);
+  if ((e = cudaMallocHost(reinterpret_cast<void**>(&h->h_cond), sizeof(int) * (h->cond_known.size() + 2))) != cudaSuccess)
+    return fail("cudaMallocHost", e);
+  if (h->tcq_bytes) {
+    std::vector<int64_t> orders;
+    for (const Layer& L : h->layers) {
+      if (!L.use_tc) continue;
+      for (int64_t k : {L.left ? L.d.m : (int64_t)0, L.right ? L.d.n : (int64_t)0})
+        if (k && qr_tc_eligible(k) && std::find(orders.begin(), orders.end(), k) == orders.end()) orders.push_back(k);
+    }
+    for (int i = 0; i < h->n_lanes; ++i)
+      for (int64_t k : orders) {
+        const char* qerr = nullptr;
+        QrTc* t = qr_tc_create(k, h->lanes[i].tcq_scratch, device, s, &qerr);
+        if (!t) {
+          g_create_error = qerr ? qerr : "tensor-core projection plans could not be created";
+          if (h->alloc.alloc) h->alloc.free(h->slab, h->alloc.ctx); else cudaFree(h->slab);
+          delete h;
+          return BR_ERR_CUDA;
+        }
+        h->lanes[i].tcq.push_back(t);
+      }
+  }
   const char* tc_err = nullptr;
   h->tc = tc_step_create(h->layers, h->hp, h->slab + sz.total, tc_bytes, device, s, &tc_err);
   if (!h->tc && tc_err) {
@@ -683,6 +740,14 @@ br_status br_get_counters(br_handle* h, int layer, br_counters* out) {
   out->ring_slot = L.d.tau_max > 0 ? h->calls % L.d.tau_max : 0;
   out->refresh_count = L.refresh_count;
   out->next_refresh_t = (L.t / L.freq + 1) * L.freq;
+  if (h->cond_pending) {
+    if (cudaSetDevice(h->device) != cudaSuccess || cudaEventSynchronize(h->ev_cond) != cudaSuccess) {
+      h->err = "could not read the conditioning notes of the last refresh"; return BR_ERR_CUDA;
+    }
+    for (size_t i = 0; i < h->cond_known.size(); ++i) h->cond_known[i] = h->h_cond[i];
+    h->cond_pending = false;
+  }
+  out->basis_flags = (h->cond_known[2 * layer] ? 1 : 0) | (h->cond_known[2 * layer + 1] ? 2 : 0);
   return BR_OK;
 }
 
@@ -694,6 +759,19 @@ br_status br_set_counters(br_handle* h, int layer, const br_counters* in) {
   h->calls = in->calls;
   L.t = in->t;
   L.refresh_count = in->refresh_count;
+  {
+    br_status st = check_handle(h);
+    if (st != BR_OK) return st;
+    BR_CUDA(h, cudaStreamSynchronize(h->stream));
+    if (h->cond_pending) {
+      for (size_t i = 0; i < h->cond_known.size(); ++i) h->cond_known[i] = h->h_cond[i];
+      h->cond_pending = false;
+    }
+    const int v[2] = {(int)(in->basis_flags & 1), (int)((in->basis_flags >> 1) & 1)};
+    h->cond_known[2 * layer] = v[0];
+    h->cond_known[2 * layer + 1] = v[1];
+    BR_CUDA(h, cudaMemcpy(h->d_cond + 2 * layer, v, sizeof v, cudaMemcpyHostToDevice));
+  }
   return BR_OK;
 }
 
@@ -827,6 +905,10 @@ br_status br_destroy(br_handle* h) {
     if (h->lanes[i].done) cudaEventDestroy(h->lanes[i].done);
   }
   if (h->ev_begin) cudaEventDestroy(h->ev_begin);
+  if (h->ev_cond) cudaEventDestroy(h->ev_cond);
+  if (h->h_cond) cudaFreeHost(h->h_cond);
+  for (int i = 0; i < br_handle::kMaxLanes; ++i)
+    for (QrTc* t : h->lanes[i].tcq) qr_tc_destroy(t);
   for (auto& sp : h->stats.prof.spans) { cudaEventDestroy(sp.a); cudaEventDestroy(sp.b); }
   for (auto e : h->stats.prof.free_events) cudaEventDestroy(e);
   if (h->slab) {

@@ -77,6 +77,13 @@ cudaError_t widen_bf16(const __nv_bfloat16* X, float* out, int64_t numel, cudaSt
 // out(double) <- in(float) ; out(float) <- in(double)
 cudaError_t f64_to_f32(const double* X, float* out, int64_t numel, cudaStream_t s);
 cudaError_t f32_to_f64(const float* X, double* out, int64_t numel, cudaStream_t s);
+// Three-term bf16 split (all 24 bits of the fp32 rounding of x) of a rows x cols block of a strided
+// fp64 matrix, or of a contiguous fp32 array, into compact planes; A (fp64, strided) -= D (fp32, compact).
+cudaError_t split3_f64(const double* X, int64_t ld, int64_t rows, int64_t cols, __nv_bfloat16* p1,
+                       __nv_bfloat16* p2, __nv_bfloat16* p3, cudaStream_t s);
+cudaError_t split3_f32(const float* X, int64_t numel, __nv_bfloat16* p1, __nv_bfloat16* p2, __nv_bfloat16* p3,
+                       cudaStream_t s);
+cudaError_t sub_f32_from_f64(double* A, int64_t ld, int64_t rows, int64_t cols, const float* D, cudaStream_t s);
 // out <- beta1 M + (1-beta1) G (out-of-place form of Alg. 1 line 4)
 cudaError_t ema_out(float* out, const float* M, const void* G, int g_is_bf16, int64_t numel, float beta1,
                     cudaStream_t s);
@@ -108,8 +115,21 @@ cudaError_t dgemm_ex(int ta, int tb, int64_t M, int64_t N, int64_t K, double alp
 // BR_WARN_RANK_DEFICIENT when a pivot underflows.  Returns the number of launches in *launches.
 // ---------------------------------------------------------------------------------------------
 size_t qr_work_doubles(int64_t k);
+// Optional tensor-core form of the block projections (see qr.cu): plans and scratch for one order
+// k, created once.  qr_tc_scratch_bytes is 0 when the order is not eligible.
+struct QrTc;
+bool qr_tc_eligible(int64_t k);
+size_t qr_tc_scratch_bytes(int64_t k);
+QrTc* qr_tc_create(int64_t k, char* scratch, int device, cudaStream_t s, const char** err);
+void qr_tc_destroy(QrTc* t);
+int64_t qr_tc_order(const QrTc* t);
+cudaError_t qr_tc_project(QrTc* t, int node, double* A, int64_t k, int64_t jp, int64_t wp, int64_t jt,
+                          int64_t wt, int* status, cudaStream_t s);
+// tc: null, or the plans for this order: the first sweep then projects on the tensor cores (ask for it
+// only when the previous refresh of this basis left *cond_out == 1).  cond_out: DEVICE int that
+// receives 1 when no column shrank below 1e-3 of its length during this factorisation, else 0.
 cudaError_t qr_pos_inplace(double* A, int64_t k, double* work, int* status, cudaStream_t s,
-                           int64_t* launches, double* flops);
+                           int64_t* launches, double* flops, QrTc* tc = nullptr, int* cond_out = nullptr);
 
 // ---------------------------------------------------------------------------------------------
 // tcgen05 grouped contraction (gemm_tc.cu)
@@ -158,6 +178,11 @@ void tc_plan_destroy(TcPlan* p);
 cudaError_t tc_plan_launch(TcPlan* p, long long calls, int tau, float dyn_alpha, float dyn_beta,
                            int* status_word, cudaStream_t s);
 double tc_plan_flops(const TcPlan* p);
+// Launch only the problems [first, first + count) of a plan (e.g. one node of a recursion whose
+// problems all live in one plan), and the flop count of that range.
+cudaError_t tc_plan_launch_range(TcPlan* p, int first, int count, long long calls, int tau, float dyn_alpha,
+                                 float dyn_beta, int* status_word, cudaStream_t s);
+double tc_plan_flops_range(const TcPlan* p, int first, int count);
 int tc_supported(int device);
 
 }  // namespace br

@@ -215,6 +215,44 @@ k_ema_out(float* __restrict__ out, const float* __restrict__ M, const void* __re
     out[i] = beta1 * M[i] + omb * load_grad1<G_BF16>(G, i);
 }
 
+// x (rounded to fp32) = p1 + p2 + p3 with three bf16 terms: all 24 significant bits survive.
+__device__ __forceinline__ void split3(float f, __nv_bfloat16& p1, __nv_bfloat16& p2, __nv_bfloat16& p3) {
+  const float h1 = bf16_round(f);
+  const float r1 = f - h1;
+  const float h2 = bf16_round(r1);
+  const float r2 = r1 - h2;
+  p1 = __float2bfloat16_rn(h1); p2 = __float2bfloat16_rn(h2); p3 = __float2bfloat16_rn(r2);
+}
+
+// X: rows x cols block of a row-major fp64 matrix with leading dimension ld -> three compact
+// (ld = cols) bf16 planes
+__global__ void __launch_bounds__(kThreads)
+k_split3_f64(const double* __restrict__ X, int64_t ld, int64_t rows, int64_t cols, __nv_bfloat16* __restrict__ p1,
+             __nv_bfloat16* __restrict__ p2, __nv_bfloat16* __restrict__ p3) {
+  const int64_t total = rows * cols;
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t r = i / cols, c = i - r * cols;
+    split3((float)X[r * ld + c], p1[i], p2[i], p3[i]);
+  }
+}
+
+__global__ void __launch_bounds__(kThreads)
+k_split3_f32(const float* __restrict__ X, int64_t numel, __nv_bfloat16* __restrict__ p1,
+             __nv_bfloat16* __restrict__ p2, __nv_bfloat16* __restrict__ p3) {
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < numel; i += (int64_t)gridDim.x * blockDim.x)
+    split3(X[i], p1[i], p2[i], p3[i]);
+}
+
+// A (fp64, leading dimension ld) -= D (fp32, compact rows x cols)
+__global__ void __launch_bounds__(kThreads)
+k_sub_f32_from_f64(double* __restrict__ A, int64_t ld, int64_t rows, int64_t cols, const float* __restrict__ D) {
+  const int64_t total = rows * cols;
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t r = i / cols, c = i - r * cols;
+    A[r * ld + c] -= (double)D[i];
+  }
+}
+
 __global__ void __launch_bounds__(kThreads)
 k_f32_to_f64(const float* __restrict__ X, double* __restrict__ out, int64_t numel) {
   const int64_t stride = (int64_t)gridDim.x * blockDim.x;
@@ -279,6 +317,23 @@ cudaError_t ema_out(float* out, const float* M, const void* G, int g_is_bf16, in
   const int grid = grid_for((numel + 3) / 4);
   if (g_is_bf16) k_ema_out<true><<<grid, kThreads, 0, s>>>(out, M, G, numel, beta1);
   else k_ema_out<false><<<grid, kThreads, 0, s>>>(out, M, G, numel, beta1);
+  return cudaGetLastError();
+}
+
+cudaError_t split3_f64(const double* X, int64_t ld, int64_t rows, int64_t cols, __nv_bfloat16* p1,
+                       __nv_bfloat16* p2, __nv_bfloat16* p3, cudaStream_t s) {
+  k_split3_f64<<<grid_for(rows * cols), kThreads, 0, s>>>(X, ld, rows, cols, p1, p2, p3);
+  return cudaGetLastError();
+}
+
+cudaError_t split3_f32(const float* X, int64_t numel, __nv_bfloat16* p1, __nv_bfloat16* p2, __nv_bfloat16* p3,
+                       cudaStream_t s) {
+  k_split3_f32<<<grid_for(numel), kThreads, 0, s>>>(X, numel, p1, p2, p3);
+  return cudaGetLastError();
+}
+
+cudaError_t sub_f32_from_f64(double* A, int64_t ld, int64_t rows, int64_t cols, const float* D, cudaStream_t s) {
+  k_sub_f32_from_f64<<<grid_for(rows * cols), kThreads, 0, s>>>(A, ld, rows, cols, D);
   return cudaGetLastError();
 }
 

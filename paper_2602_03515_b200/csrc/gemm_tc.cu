@@ -239,7 +239,7 @@ __device__ __forceinline__ TileInfo locate_tile(const DevProblem* probs, int n_p
 // ---------------------------------------------------------------------------------------------
 template <bool SHARED>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-k_tc_gemm(const DevProblem* __restrict__ probs, int n_probs, int total_tiles, long long calls,
+k_tc_gemm(const DevProblem* __restrict__ probs, int n_probs, int first_tile, int total_tiles, long long calls,
           int tau, float dyn_alpha, float dyn_beta, int* status) {
   constexpr int NST = SHARED ? SH_STAGES : STAGES;
   extern __shared__ uint8_t smem_raw[];
@@ -287,7 +287,7 @@ k_tc_gemm(const DevProblem* __restrict__ probs, int n_probs, int total_tiles, lo
     // ======================= TMA producer =======================
     if (lane == 0) {
       int stage = 0; uint32_t phase = 0;
-      for (int tile = blockIdx.x; tile < total_tiles && !*abort_flag; tile += gridDim.x) {
+      for (int tile = first_tile + blockIdx.x; tile < total_tiles && !*abort_flag; tile += gridDim.x) {
         const TileInfo ti = locate_tile(probs, n_probs, tile, calls, tau);
         if (!ti.active) continue;
         const DevProblem* p = ti.p;
@@ -340,7 +340,7 @@ k_tc_gemm(const DevProblem* __restrict__ probs, int n_probs, int total_tiles, lo
     if (lane == 0) {
       int stage = 0; uint32_t phase = 0;
       int acc = 0; uint32_t acc_phase = 0;
-      for (int tile = blockIdx.x; tile < total_tiles && !*abort_flag; tile += gridDim.x) {
+      for (int tile = first_tile + blockIdx.x; tile < total_tiles && !*abort_flag; tile += gridDim.x) {
         const TileInfo ti = locate_tile(probs, n_probs, tile, calls, tau);
         if (!ti.active) continue;
         const DevProblem* p = ti.p;
@@ -394,7 +394,7 @@ k_tc_gemm(const DevProblem* __restrict__ probs, int n_probs, int total_tiles, lo
     float* tile = epi_tiles + quad * (32 * EPI_LD);
     const int sub_r = lane >> 3, sub_c = (lane & 7) * 4;
     int acc = 0; uint32_t acc_phase = 0;
-    for (int tile_i = blockIdx.x; tile_i < total_tiles && !*abort_flag; tile_i += gridDim.x) {
+    for (int tile_i = first_tile + blockIdx.x; tile_i < total_tiles && !*abort_flag; tile_i += gridDim.x) {
       const TileInfo ti = locate_tile(probs, n_probs, tile_i, calls, tau);
       if (!ti.active) continue;
       const DevProblem* p = ti.p;
@@ -636,6 +636,8 @@ bool encode_operand(CUtensorMap* map, const TcOperand& op, int64_t rows, int64_t
 
 struct TcPlan {
   bool shared = false;          // launches the shared-operand form of the kernel
+  std::vector<int> tile_begin;  // per problem, plus the total at the end
+  std::vector<double> prob_flops;
   DevProblem* d_probs = nullptr;
   int n = 0;
   int total_tiles = 0;
@@ -678,6 +680,8 @@ TcPlan* tc_plan_create(const TcProblem* problems, int n, int device, cudaStream_
   }
   shared = shared && eligible;
   std::vector<DevProblem> host(n);
+  std::vector<int> tile_starts;
+  std::vector<double> prob_flops;
   int tile_begin = 0;
   double flops = 0.0;
   for (int i = 0; i < n; ++i) {
@@ -725,6 +729,7 @@ TcPlan* tc_plan_create(const TcProblem* problems, int n, int device, cudaStream_
     d.tiles_n = (int32_t)((q.Nd + BN - 1) / BN);
     d.tile_begin = tile_begin;
     d.tile_count = d.tiles_m * d.tiles_n;
+    tile_starts.push_back(tile_begin);
     tile_begin += d.tile_count;
     d.tau_max = q.tau_max;
     d.dyn_scalars = q.dyn_scalars;
@@ -741,6 +746,7 @@ TcPlan* tc_plan_create(const TcProblem* problems, int n, int device, cudaStream_
         (need_H && (!q.Dh || (q.ldh % 8) || (reinterpret_cast<uintptr_t>(q.Dh) & 15))) ||
         (q.Dl && (reinterpret_cast<uintptr_t>(q.Dl) & 15)))
       return fail("tensor-core problem: output pointer missing or misaligned");
+    const double flops_before = flops;
     if (q.symmetric) {
       // executed work: the tiles that touch the upper triangle
       int64_t computed = 0;
@@ -751,9 +757,13 @@ TcPlan* tc_plan_create(const TcProblem* problems, int n, int device, cudaStream_
     } else {
       flops += 2.0 * (double)q.Md * (double)q.Nd * (double)q.K * q.n_pairs;
     }
+    prob_flops.push_back(flops - flops_before);
   }
   TcPlan* plan = new TcPlan();
   plan->shared = shared;
+  tile_starts.push_back(tile_begin);
+  plan->tile_begin = tile_starts;
+  plan->prob_flops = prob_flops;
   plan->n = n;
   plan->total_tiles = tile_begin;
   plan->flops = flops;
@@ -784,20 +794,34 @@ void tc_plan_destroy(TcPlan* p) {
 
 double tc_plan_flops(const TcPlan* p) { return p ? p->flops : 0.0; }
 
-cudaError_t tc_plan_launch(TcPlan* p, long long calls, int tau, float dyn_alpha, float dyn_beta,
-                           int* status_word, cudaStream_t s) {
-  const int grid = p->total_tiles < p->sm_count ? p->total_tiles : p->sm_count;
+cudaError_t tc_plan_launch_range(TcPlan* p, int first, int count, long long calls, int tau, float dyn_alpha,
+                                 float dyn_beta, int* status_word, cudaStream_t s) {
+  if (first < 0 || count < 1 || first + count > p->n) return cudaErrorInvalidValue;
+  const int t0 = p->tile_begin[first], t1 = p->tile_begin[first + count];
+  const int tiles = t1 - t0;
+  const int grid = tiles < p->sm_count ? tiles : p->sm_count;
   // per-device attribute: set again when another device is current (cheap, idempotent)
   if (p->shared) {
     cudaFuncSetAttribute(k_tc_gemm<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
-    k_tc_gemm<true><<<grid, NUM_THREADS, SMEM_BYTES, s>>>(p->d_probs, p->n, p->total_tiles, calls, tau, dyn_alpha,
+    k_tc_gemm<true><<<grid, NUM_THREADS, SMEM_BYTES, s>>>(p->d_probs, p->n, t0, t1, calls, tau, dyn_alpha,
                                                           dyn_beta, status_word);
   } else {
     cudaFuncSetAttribute(k_tc_gemm<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
-    k_tc_gemm<false><<<grid, NUM_THREADS, SMEM_BYTES, s>>>(p->d_probs, p->n, p->total_tiles, calls, tau, dyn_alpha,
+    k_tc_gemm<false><<<grid, NUM_THREADS, SMEM_BYTES, s>>>(p->d_probs, p->n, t0, t1, calls, tau, dyn_alpha,
                                                            dyn_beta, status_word);
   }
   return cudaGetLastError();
+}
+
+cudaError_t tc_plan_launch(TcPlan* p, long long calls, int tau, float dyn_alpha, float dyn_beta,
+                           int* status_word, cudaStream_t s) {
+  return tc_plan_launch_range(p, 0, p->n, calls, tau, dyn_alpha, dyn_beta, status_word, s);
+}
+
+double tc_plan_flops_range(const TcPlan* p, int first, int count) {
+  double f = 0.0;
+  for (int i = first; i < first + count && i < p->n; ++i) f += p->prob_flops[i];
+  return f;
 }
 
 }  // namespace br

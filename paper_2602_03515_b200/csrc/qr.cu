@@ -25,7 +25,21 @@
 // orthogonality error of up to ~1e-16 * 1e4^2); every launch of the second sweep returns at once
 // while the flag is set.
 // All reductions are done in a fixed order, so the result is bit-reproducible from run to run.
+//
+// Tensor-core projections.  Once the basis tracks the factor, the two products of a block
+// projection no longer need fp64: Q_l, A_r and the coefficients C are split into three bf16 terms
+// each (all 24 bits of their fp32 rounding) and the six leading products are accumulated in fp32 on
+// the tcgen05 kernel, C = Q_l^T A_r and D = Q_l C, then A_r -= D in fp64, and the whole projection is
+// applied twice so that what is left of span(Q_l) is ~1e-7 of the column's length after the
+// projection, not before it.  The rounding of D (fp32) remains: ~6e-8 of the column's original
+// length in an arbitrary direction, i.e. 6e-8 / s of the projected column when it shrinks to the
+// fraction s of its length.  The caller therefore asks for this form only for a basis whose
+// previous refresh saw no column shrink below 1e-3 (cond_out), the sweep still measures the
+// shrinkage, and it runs the second (fp64) sweep already when a column keeps less than 1e-3 instead
+// of 1e-4.  The leaves (Cholesky-QR) and the power product stay in fp64.
 #include <algorithm>
+#include <string>
+#include <vector>
 
 #include "br_internal.h"
 
@@ -40,6 +54,8 @@ inline int panel_width(int64_t k) { return k >= 1024 ? 128 : 64; }
 inline int gram_splits(int64_t k) { return (int)std::min<int64_t>(64, std::max<int64_t>(1, cdiv(k, 128))); }
 inline int proj_splits_max(int64_t k) { return k >= 1024 ? 64 : 1; }
 constexpr double kIllRatio = 1e-8;   // squared-norm ratio below which the second sweep runs
+constexpr double kTcRatio = 1e-6;    // the same, when the projections ran on the tensor cores; also
+                                     // the ratio below which the next refresh must not use them
 // sub-buffers of the work area start on 256-byte boundaries
 inline int64_t pad32(int64_t doubles) { return (doubles + 31) / 32 * 32; }
 
@@ -66,15 +82,20 @@ inline int64_t pad32(int64_t doubles) { return (doubles + 31) / 32 * 32; }
 __global__ void __launch_bounds__(512)
 k_chol_inverse(const double* __restrict__ S, int bw, double* __restrict__ Rinv, int* __restrict__ status,
                int* __restrict__ skip_next, const int* __restrict__ skip_self,
-               const double* __restrict__ norm0, int* __restrict__ ill_clear) {
+               const double* __restrict__ norm0, int* __restrict__ ill_clear, double ill_ratio,
+               int* __restrict__ tc_ok_clear) {
   if (skip_self && *skip_self) {
     if (skip_next && threadIdx.x == 0) *skip_next = 1;
     return;
   }
   __shared__ double rowS[2][kB];
-  __shared__ double diag0[kB], diag0_inv[kB], nrm_floor[kB];
+  __shared__ double diag0[kB], diag0_inv[kB], nrm_floor[kB], tc_floor[kB];
   const int t = threadIdx.x, ty = t >> 4, tx = t & 15;
-  if (t < kB) nrm_floor[t] = (norm0 && t < bw) ? kIllRatio * norm0[t] : 0.0;
+  if (t < kB) {
+    const double n0 = (norm0 && t < bw) ? norm0[t] : 0.0;
+    nrm_floor[t] = ill_ratio * n0;
+    tc_floor[t] = kTcRatio * n0;
+  }
   double Z[4][8];
 #pragma unroll
   for (int a = 0; a < 4; ++a) {
@@ -93,7 +114,7 @@ k_chol_inverse(const double* __restrict__ S, int bw, double* __restrict__ Rinv, 
   }
   __syncthreads();
   double defect = 0.0;       // accumulated by thread 0 (every thread sees every pivot)
-  bool ill = false;
+  bool ill = false, tc_bad = false;
 
   for (int c = 0; c < bw; ++c) {
     const int buf = c & 1;
@@ -107,6 +128,7 @@ k_chol_inverse(const double* __restrict__ S, int bw, double* __restrict__ Rinv, 
       if (clamped) atomicMax(status, (int)BR_WARN_RANK_DEFICIENT);
       defect += fmax(0.0, 1.0 - piv * diag0_inv[c]);
       if (orig < nrm_floor[c]) ill = true;
+      if (orig < tc_floor[c]) tc_bad = true;
     }
     const double inv_d = rsqrt(piv);
     double rj[8];
@@ -158,8 +180,13 @@ k_chol_inverse(const double* __restrict__ S, int bw, double* __restrict__ Rinv, 
   if (t == 0) {
     if (skip_next) *skip_next = (defect <= kDefectLimit) ? 1 : 0;
     if (ill && ill_clear) *ill_clear = 0;
+    if (tc_bad && tc_ok_clear) *tc_ok_clear = 0;
   }
 }
+
+// flags at the start of a QR: second sweep cancelled, basis well enough conditioned for the
+// tensor-core projections next time; and the copy of the latter to its long-lived home at the end
+__global__ void k_store_flag(int* dst, const int* src) { *dst = *src; }
 
 // part[z][j] = sum over the row chunk z of A[i][j]^2 (rows in order)
 constexpr int kNormChunks = 32;
@@ -183,17 +210,147 @@ __global__ void __launch_bounds__(256)
 k_column_norms_sum(const double* __restrict__ part, int64_t k, int nchunks, double* __restrict__ norm0,
                    int* __restrict__ flag) {
   const int64_t j = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
-  if (j == 0) *flag = 1;
+  if (j == 0) { flag[0] = 1; flag[1] = 1; }   // sweep-2 cancelled, tensor-core projections allowed next time
   if (j >= k) return;
   double s = 0.0;
   for (int z = 0; z < nchunks; ++z) s += part[(int64_t)z * k + j];
   norm0[j] = s;
 }
 
+struct ProjNode { int64_t jp, wp, jt, wt; };
+
+// projections of orth(0, k) in the order in which the recursion runs them
+// A projection goes to the tensor cores only when it is large: the grouped kernel has no split over
+// K, so a product with a handful of output tiles would leave most SMs idle.
+inline bool tc_node(int64_t wp, int64_t wt) { return wp * wt >= (int64_t)1 << 21; }
+
+void enumerate_nodes(int64_t j0, int64_t w, int64_t b, std::vector<ProjNode>* out) {
+  if (w <= b) return;
+  const int64_t h = cdiv(w, 2 * b) * b;
+  enumerate_nodes(j0, h, b, out);
+  if (tc_node(h, w - h)) out->push_back({j0, h, j0 + h, w - h});
+  enumerate_nodes(j0 + h, w - h, b, out);
+}
+
+}  // namespace
+
+// Plans and scratch of the tensor-core projections for one order k.  Problem 2 i of either plan is
+// the coefficient product of node i, problem 2 i + 1 its update product; plan `lead` holds the
+// products of the two leading bf16 terms (hi*hi + mid*hi + hi*mid), plan `tail` the next three.
+struct QrTc {
+  int64_t k = 0;
+  std::vector<ProjNode> nodes;
+  TcPlan *lead = nullptr, *tail = nullptr;
+  __nv_bfloat16 *Q[3] = {}, *A[3] = {}, *C[3] = {};
+  float *Cf = nullptr, *Df = nullptr;
+};
+
+namespace {
+inline int64_t tc_hmax(int64_t k) { return cdiv(k, 2 * 128) * 128; }
+inline size_t al256(size_t x) { return (x + 255) / 256 * 256; }
+}  // namespace
+
+int64_t qr_tc_order(const QrTc* t) { return t ? t->k : 0; }
+bool qr_tc_eligible(int64_t k) { return k >= 4096 && (k % 8) == 0; }
+
+size_t qr_tc_scratch_bytes(int64_t k) {
+  if (!qr_tc_eligible(k)) return 0;
+  const size_t h = (size_t)tc_hmax(k), kk = (size_t)k;
+  return 6 * al256(kk * h * 2) + al256(h * h * 4) + 3 * al256(h * h * 2) + al256(kk * h * 4);
+}
+
+void qr_tc_destroy(QrTc* t) {
+  if (!t) return;
+  tc_plan_destroy(t->lead);
+  tc_plan_destroy(t->tail);
+  delete t;
+}
+
+QrTc* qr_tc_create(int64_t k, char* scratch, int device, cudaStream_t s, const char** err) {
+  static thread_local std::string last;
+  if (err) *err = nullptr;
+  if (!qr_tc_eligible(k) || !tc_supported(device)) return nullptr;
+  QrTc* t = new QrTc();
+  t->k = k;
+  const size_t h = (size_t)tc_hmax(k), kk = (size_t)k;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { char* p = scratch + off; off += al256(bytes); return p; };
+  for (int i = 0; i < 3; ++i) t->Q[i] = reinterpret_cast<__nv_bfloat16*>(take(kk * h * 2));
+  for (int i = 0; i < 3; ++i) t->A[i] = reinterpret_cast<__nv_bfloat16*>(take(kk * h * 2));
+  t->Cf = reinterpret_cast<float*>(take(h * h * 4));
+  for (int i = 0; i < 3; ++i) t->C[i] = reinterpret_cast<__nv_bfloat16*>(take(h * h * 2));
+  t->Df = reinterpret_cast<float*>(take(kk * h * 4));
+  enumerate_nodes(0, k, 128, &t->nodes);
+  std::vector<TcProblem> lead, tail;
+  auto opnd = [](const void* p, int64_t ld, int mn) { TcOperand o; o.ptr = p; o.ld = ld; o.mn_major = mn; return o; };
+  for (const ProjNode& nd : t->nodes) {
+    // coefficients C = Q^T A_r (contraction over the k rows: both operands MN-major)
+    TcProblem c; c.Md = nd.wp; c.Nd = nd.wt; c.K = k; c.n_pairs = 3;
+    c.epilogue = EPI_AXPBY_F32; c.alpha = 1.f; c.D = t->Cf; c.ldd = nd.wt;
+    TcProblem c2 = c;
+    const int ia[6] = {0, 1, 0, 2, 0, 1}, ib[6] = {0, 0, 1, 0, 2, 1};      // term pairs, leading three first
+    for (int p = 0; p < 3; ++p) {
+      c.A[p] = opnd(t->Q[ia[p]], nd.wp, 1); c.B[p] = opnd(t->A[ib[p]], nd.wt, 1);
+      c2.A[p] = opnd(t->Q[ia[3 + p]], nd.wp, 1); c2.B[p] = opnd(t->A[ib[3 + p]], nd.wt, 1);
+    }
+    c.beta = 0.f; c2.beta = 1.f;
+    // update D = Q C (Q K-major, C MN-major)
+    TcProblem d; d.Md = k; d.Nd = nd.wt; d.K = nd.wp; d.n_pairs = 3;
+    d.epilogue = EPI_AXPBY_F32; d.alpha = 1.f; d.D = t->Df; d.ldd = nd.wt;
+    TcProblem d2 = d;
+    for (int p = 0; p < 3; ++p) {
+      d.A[p] = opnd(t->Q[ia[p]], nd.wp, 0); d.B[p] = opnd(t->C[ib[p]], nd.wt, 1);
+      d2.A[p] = opnd(t->Q[ia[3 + p]], nd.wp, 0); d2.B[p] = opnd(t->C[ib[3 + p]], nd.wt, 1);
+    }
+    d.beta = 0.f; d2.beta = 1.f;
+    lead.push_back(c); lead.push_back(d);
+    tail.push_back(c2); tail.push_back(d2);
+  }
+  const char* perr = nullptr;
+  if (!lead.empty()) {
+    t->lead = tc_plan_create(lead.data(), (int)lead.size(), device, s, &perr);
+    if (t->lead) t->tail = tc_plan_create(tail.data(), (int)tail.size(), device, s, &perr);
+    if (!t->lead || !t->tail) {
+      last = perr ? perr : "plan creation failed";
+      if (err) *err = last.c_str();
+      qr_tc_destroy(t);
+      return nullptr;
+    }
+  }
+  return t;
+}
+
+cudaError_t qr_tc_project(QrTc* t, int node, double* A, int64_t k, int64_t jp, int64_t wp, int64_t jt,
+                          int64_t wt, int* status, cudaStream_t s) {
+  if (node < 0 || node >= (int)t->nodes.size()) return cudaErrorInvalidValue;
+  const ProjNode& nd = t->nodes[node];
+  if (nd.jp != jp || nd.wp != wp || nd.jt != jt || nd.wt != wt || t->k != k) return cudaErrorInvalidValue;
+  cudaError_t e;
+  if ((e = split3_f64(A + jp, k, k, wp, t->Q[0], t->Q[1], t->Q[2], s)) != cudaSuccess) return e;
+  // Twice: the coefficients of the first pass are wrong by ~1e-7 of the column's length BEFORE the
+  // projection, which leaves that much of span(Q_l) in the column; the second pass sees the
+  // shrunken column and leaves ~1e-7 of its length AFTER the projection.
+  for (int pass = 0; pass < 2; ++pass) {
+    if ((e = split3_f64(A + jt, k, k, wt, t->A[0], t->A[1], t->A[2], s)) != cudaSuccess) return e;
+    if ((e = tc_plan_launch_range(t->lead, 2 * node, 1, 1, 0, 1.f, 0.f, status, s)) != cudaSuccess) return e;
+    if ((e = tc_plan_launch_range(t->tail, 2 * node, 1, 1, 0, 1.f, 0.f, status, s)) != cudaSuccess) return e;
+    if ((e = split3_f32(t->Cf, wp * wt, t->C[0], t->C[1], t->C[2], s)) != cudaSuccess) return e;
+    if ((e = tc_plan_launch_range(t->lead, 2 * node + 1, 1, 1, 0, 1.f, 0.f, status, s)) != cudaSuccess) return e;
+    if ((e = tc_plan_launch_range(t->tail, 2 * node + 1, 1, 1, 0, 1.f, 0.f, status, s)) != cudaSuccess) return e;
+    if ((e = sub_f32_from_f64(A + jt, k, k, wt, t->Df, s)) != cudaSuccess) return e;
+  }
+  return cudaSuccess;
+}
+
+namespace {
+
 struct Sweep {
   double* A; int64_t k; int b, sg, sp_max;
   double *gram_part, *S, *Rinv, *norm0, *C, *proj_part;
-  int *skip2, *sweep2_skip;
+  int *skip2, *sweep2_skip;   // sweep2_skip[1] is the "tensor cores allowed next time" flag
+  QrTc* tc = nullptr;         // non-null: block projections of the first sweep on the tensor cores
+  int node = 0;               // running index of the projection in recursion order
+  double ill_ratio = kIllRatio;
   int* status;
   cudaStream_t s;
   const int* skip;        // non-null: every launch of this sweep returns while *skip != 0
@@ -212,7 +369,8 @@ void leaf(Sweep& q, int64_t j0, int bw) {
     cudaError_t e = dgemm_ex(1, 0, bw, bw, k, 1.0, P, k, P, k, 0.0, q.S, bw, q.sg, q.gram_part, skip, q.s);
     if (e != cudaSuccess) { q.err = e; return; }
     k_chol_inverse<<<1, 512, 0, q.s>>>(q.S, bw, q.Rinv, q.status, pass ? nullptr : q.skip2, skip,
-                                       (q.first && !pass) ? q.norm0 + j0 : nullptr, q.sweep2_skip);
+                                       (q.first && !pass) ? q.norm0 + j0 : nullptr, q.sweep2_skip, q.ill_ratio,
+                                       q.sweep2_skip + 1);
     // P <- P R^-1 (in place: a CTA reads only the rows it writes, and writes after its last read)
     e = dgemm_ex(0, 0, k, bw, bw, 1.0, P, k, q.Rinv, bw, 0.0, P, k, 1, nullptr, skip, q.s);
     if (e != cudaSuccess) { q.err = e; return; }
@@ -225,6 +383,11 @@ void leaf(Sweep& q, int64_t j0, int bw) {
 void project(Sweep& q, int64_t jp, int64_t wp, int64_t jt, int64_t wt) {
   if (q.err != cudaSuccess) return;
   const int64_t k = q.k;
+  if (q.tc && q.first && tc_node(wp, wt)) {
+    q.err = qr_tc_project(q.tc, q.node++, q.A, k, jp, wp, jt, wt, q.status, q.s);
+    q.launches += 15;
+    return;
+  }
   const int64_t tiles = cdiv(wp, 128) * cdiv(wt, 128);
   int sp = 1;
   if (tiles < 148) sp = (int)std::max<int64_t>(1, std::min<int64_t>(std::min<int64_t>(cdiv(296, tiles), q.sp_max), k / 128));
@@ -261,8 +424,9 @@ size_t qr_work_doubles(int64_t k) {
 }
 
 cudaError_t qr_pos_inplace(double* A, int64_t k, double* work, int* status, cudaStream_t s,
-                           int64_t* launches, double* flops) {
+                           int64_t* launches, double* flops, QrTc* tc, int* cond_out) {
   Sweep q;
+  if (tc && tc->k == k) { q.tc = tc; q.ill_ratio = kTcRatio; }
   q.A = A; q.k = k; q.s = s; q.status = status;
   q.b = (int)std::min<int64_t>(panel_width(k), k);
   q.sg = gram_splits(k);
@@ -294,9 +458,10 @@ cudaError_t qr_pos_inplace(double* A, int64_t k, double* work, int* status, cuda
   q.skip = q.sweep2_skip; q.first = false;
   orth(q, 0, k);
   if (q.err != cudaSuccess) return q.err;
+  if (cond_out) k_store_flag<<<1, 1, 0, s>>>(cond_out, q.sweep2_skip + 1);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  if (launches) *launches += q.launches + 2;
+  if (launches) *launches += q.launches + 2 + (cond_out ? 1 : 0);
   if (flops) *flops += q.flops;
   return cudaSuccess;
 }

@@ -133,6 +133,41 @@ def test_refresh_order_1024_against_oracle_power():
     assert np.max(np.abs(U.T @ U - np.eye(k))) < 1e-5
 
 
+def test_refresh_tensor_core_projections_order_4224():
+    """Third refresh of a basis of order 4224 in one handle (orders from 4096 use the tensor-core
+    projections).  The first (from U = I) is ill-conditioned, the second runs in fp64 and notes that
+    no column shrank much, so the third runs its large block projections on the tensor cores
+    (three-term bf16 splits, applied twice).  The result is unique (QR with a positive diagonal), so
+    it is compared with LAPACK's QR of the float64 product F U2 after fixing the signs -- the
+    routine the oracle's own Householder QR is pinned against at small orders, where the oracle
+    itself (interpreted loops, minutes at this order) is affordable."""
+    import torch
+    import paper_2602_03515_b200 as br
+    from tests.parity_util import basis_err
+    k = 4224
+    F = _lowrank_noise_factor(k, 16, 33, samples=1)
+    w = torch.zeros(k, 8, device="cuda")
+    opt = br.BasisRotation([LayerSpec("W", k, 8, GEOM_BI, SRC_SECOND, 0)], [w], grad_dtype="bf16",
+                           gemm_prec=br.BR_GEMM_BF16, freq=10 ** 6)
+    try:
+        assert opt.step([(torch.randn(k, 8, device="cuda") * 0.01).to(torch.bfloat16)], 0) == br.BR_OK
+        opt.set_state(0, br.BR_BUF_L, torch.from_numpy(F))
+        opt.refresh_basis(0)
+        assert br.br_get_basis_flags(opt.handle, 0) & 1 == 0       # from the identity: columns shrink by 1e4
+        opt.refresh_basis(0)
+        assert br.br_get_basis_flags(opt.handle, 0) & 1 == 1       # tracking
+        U2 = opt.get_state(0, br.BR_BUF_U).numpy()
+        opt.refresh_basis(0)                                        # large block projections on the tensor cores
+        assert opt.sync_status() == br.BR_OK
+        U3 = opt.get_state(0, br.BR_BUF_U).numpy().astype(np.float64)
+        q, r = np.linalg.qr(F.astype(np.float64) @ U2.astype(np.float64))
+        ref = q * np.sign(np.diag(r))
+        assert basis_err(U3, ref) < 1e-5
+        assert np.max(np.abs(U3.T @ U3 - np.eye(k))) < 1e-5
+    finally:
+        opt.close()
+
+
 def test_refresh_order_6912_properties():
     k = 6912
     F = _lowrank_noise_factor(k, 32, 32, samples=1)

@@ -229,7 +229,7 @@ def main():
     ap.add_argument("--impl", default="ours")
     ap.add_argument("--layers", type=int, default=None, help="decoder depth override (c4/c5)")
     ap.add_argument("--tau", type=int, default=None, help="ring depth override")
-    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--e2e-steps", type=int, default=6)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--scratch-gib", type=float, default=0.0)
     ap.add_argument("--no-refresh", action="store_true",
@@ -262,7 +262,8 @@ def main():
     free0, total_mem = torch.cuda.mem_get_info(dev)
     n_params0 = w0.n_params
     gbytes = 2 if w0.grad_dtype == "bf16" else 4
-    reserve = n_params0 * (4 + gbytes) + (6 << 30)       # caller's weights and gradient buffers + headroom
+    # caller's weights, two gradient sets (the end-to-end leg double-buffers its uploads) + headroom
+    reserve = n_params0 * (4 + 2 * gbytes) + (6 << 30)
     if args.workload in ("c4", "c5"):
         tau, state_bytes = fit_tau(args.workload, args.layers, tau_req, gemm_prec, free0, reserve, br)
         w = get_workload(args.workload, n_layers=args.layers, tau=tau)
@@ -363,13 +364,35 @@ def main():
         w_host = torch.empty(weights[0].shape, dtype=torch.float32, pin_memory=True)
         h2d = sum(h_.numel() * h_.element_size() for h_ in host)
         d2h = w_host.numel() * 4 + 4
-        sync_all()
-        t0 = time.perf_counter()
-        with torch.cuda.stream(stream):
-            for _ in range(args.e2e_steps):
-                for h_, g in zip(host, grads):
+        # Every step uploads its gradients from pinned host memory and reads a weight matrix and the
+        # status word back.  The upload of step i + 1 runs on a copy stream, into the other of two device
+        # gradient sets, while step i computes (the library has copied a call's gradients into its ring
+        # by the time the stream passes that call's work, so a set is free again two steps later).
+        grads2 = [torch.empty_like(g) for g in grads]
+        sets = [grads, grads2]
+        copy_stream = torch.cuda.Stream(device=dev)
+        up = [torch.cuda.Event(), torch.cuda.Event()]          # upload of a set finished
+        used = [torch.cuda.Event(), torch.cuda.Event()]        # the step that read a set has been passed
+
+        def upload(i):
+            with torch.cuda.stream(copy_stream):
+                copy_stream.wait_event(used[i % 2])
+                for h_, g in zip(host, sets[i % 2]):
                     g.copy_(h_, non_blocking=True)
-                opt.step(grads, tau)
+                up[i % 2].record(copy_stream)
+
+        sync_all()
+        for ev in used:
+            ev.record(stream)
+        t0 = time.perf_counter()
+        upload(0)
+        with torch.cuda.stream(stream):
+            for i in range(args.e2e_steps):
+                if i + 1 < args.e2e_steps:
+                    upload(i + 1)
+                stream.wait_event(up[i % 2])
+                opt.step(sets[i % 2], tau)
+                used[i % 2].record(stream)
                 w_host.copy_(weights[0], non_blocking=True)
                 st = opt.sync_status()          # waits for the stream and reads the status word back
                 assert st >= 0
@@ -380,7 +403,7 @@ def main():
             dist.all_reduce(t, op=dist.ReduceOp.MAX)
         e2e = {"value": world * n_params / (float(t.item()) / 1e3), "unit": UNIT, "ms_per_step": float(t.item()),
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": args.e2e_steps}
-        del host
+        del host, grads2
 
     # ---- rooflines -------------------------------------------------------------------------------
     alg_flops = algorithmic_flops_per_step(w)

@@ -204,6 +204,26 @@ BR_API br_status br_get_profile(br_handle* h, br_profile_stats* out);
 /* Free everything the handle allocated.  NULL is accepted.  Synchronises the stream. */
 BR_API br_status br_destroy(br_handle* h);
 
+/*
+ * Stage-aware refresh period (App. I of the paper, "Stage-aware basis rotation implementation").
+ * For a pipeline of P stages, a stage whose gradients are tau updates old and a base period f0:
+ *   mid = floor(P / 2) - 1;  n = mid - tau if tau > mid, else mid + 1 - tau;
+ *   f = floor(f0 / (1 - n / mid)),
+ * evaluated in exact integer arithmetic as floor(f0 * mid / (mid - n)).  The printed rule is undefined
+ * where mid - n <= 0 (for P = 32: tau <= 1) or mid <= 0 (P < 4): those arguments return BR_ERR_INVALID
+ * and leave *out_freq alone, as do P < 1, tau < 0 or f0 < 1.  A result below 1 is raised to 1.
+ * Host only.  The period is what br_layer_desc.freq takes, per layer.
+ */
+BR_API br_status br_stage_aware_freq(int P, int tau, int f0, int* out_freq);
+
+/*
+ * Effective delay of stage-dependent delays (Sec. 2.3, Eq. (effective-delay)):
+ *   tau' = sqrt( sum_i C_i^2 tau_i^2 / sum_i C_i^2 )
+ * for n groups of coordinates with smoothness constants C_i (HOST array, not all zero) and delays
+ * tau_i >= 0 (HOST array).  Host only.
+ */
+BR_API br_status br_effective_delay(const double* C, const int* tau, int n, double* out);
+
 BR_API const char* br_strerror(int status);
 /* Message of the last error on this handle (or of the last failed br_create when h is NULL). */
 BR_API const char* br_last_error(const br_handle* h);

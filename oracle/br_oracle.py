@@ -334,6 +334,33 @@ class Oracle:
                     next_refresh_t=(lay.t // freq + 1) * freq)
 
 
+def stage_aware_freq(P: int, tau: int, f0: int) -> int:
+    """Stage-aware refresh period, App. I ("Stage-aware basis rotation implementation"):
+    mid = floor(P/2) - 1; n = mid - tau if tau > mid else mid + 1 - tau; f = floor(f0 / (1 - n/mid)),
+    written out in exact rational arithmetic.  The printed rule is undefined where 1 - n/mid <= 0
+    (or mid <= 0): ValueError there.  A period below 1 is raised to 1."""
+    from fractions import Fraction
+    from math import floor
+    if P < 1 or tau < 0 or f0 < 1:
+        raise ValueError("bad argument")
+    mid = P // 2 - 1
+    if mid <= 0:
+        raise ValueError("the rule needs floor(P/2) - 1 > 0")
+    n = mid - tau if tau > mid else mid + 1 - tau
+    den = 1 - Fraction(n, mid)
+    if den <= 0:
+        raise ValueError("the rule divides by zero or goes negative at this delay")
+    return max(1, floor(Fraction(f0) / den))
+
+
+def effective_delay(consts, taus) -> float:
+    """Effective delay of stage-dependent delays, Sec. 2.3, Eq. (effective-delay):
+    tau' = sqrt(sum_i C_i^2 tau_i^2 / sum_i C_i^2)."""
+    c2 = np.asarray(consts, dtype=np.float64) ** 2
+    t = np.asarray(taus, dtype=np.float64)
+    return float(np.sqrt(np.sum(c2 * t * t) / np.sum(c2)))
+
+
 def make_oracle(workload, weights: Sequence[np.ndarray], **hp_over) -> Oracle:
     """Build an Oracle for a `workloads.Workload` (shapes and hyper-parameters only)."""
     hp = Hyper(lr=workload.lr, beta1=workload.beta1, beta2=workload.beta2, eps=workload.eps,

@@ -95,6 +95,8 @@ def load_library():
         "br_get_launch_stats": ([H, C.POINTER(C.c_int64), C.POINTER(C.c_double)], C.c_int),
         "br_profile": ([H, C.c_int], C.c_int),
         "br_get_profile": ([H, C.POINTER(BrProfileStats)], C.c_int),
+        "br_stage_aware_freq": ([C.c_int, C.c_int, C.c_int, C.POINTER(C.c_int)], C.c_int),
+        "br_effective_delay": ([C.POINTER(C.c_double), C.POINTER(C.c_int), C.c_int, C.POINTER(C.c_double)], C.c_int),
         "br_destroy": ([H], C.c_int),
         "br_power_static": ([C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p], C.c_int),
         "br_strerror": ([C.c_int], C.c_char_p),
@@ -202,6 +204,22 @@ def br_get_profile(handle) -> dict:
     st = BrProfileStats()
     _check(load_library().br_get_profile(handle, C.byref(st)), handle)
     return st.as_dict()
+
+
+def br_stage_aware_freq(P: int, tau: int, f0: int) -> int:
+    out = C.c_int(0)
+    _check(load_library().br_stage_aware_freq(int(P), int(tau), int(f0), C.byref(out)))
+    return int(out.value)
+
+
+def br_effective_delay(consts, taus) -> float:
+    n = len(consts)
+    assert n == len(taus)
+    cs = (C.c_double * n)(*[float(x) for x in consts])
+    ts = (C.c_int * n)(*[int(x) for x in taus])
+    out = C.c_double(0.0)
+    _check(load_library().br_effective_delay(cs, ts, n, C.byref(out)))
+    return float(out.value)
 
 
 def br_destroy(handle) -> int:

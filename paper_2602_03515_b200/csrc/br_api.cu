@@ -918,6 +918,34 @@ br_status br_destroy(br_handle* h) {
   return BR_OK;
 }
 
+br_status br_stage_aware_freq(int P, int tau, int f0, int* out_freq) {
+  if (!out_freq || P < 1 || tau < 0 || f0 < 1) return BR_ERR_INVALID;
+  const long long mid = P / 2 - 1;
+  if (mid <= 0) return BR_ERR_INVALID;
+  const long long n = tau > mid ? mid - tau : mid + 1 - tau;
+  const long long den = mid - n;                 // (1 - n / mid) * mid
+  if (den <= 0) return BR_ERR_INVALID;
+  long long f = ((long long)f0 * mid) / den;     // both positive: truncation is the floor
+  if (f < 1) f = 1;
+  if (f > 0x7fffffffLL) f = 0x7fffffffLL;
+  *out_freq = (int)f;
+  return BR_OK;
+}
+
+br_status br_effective_delay(const double* C, const int* tau, int n, double* out) {
+  if (!C || !tau || !out || n < 1) return BR_ERR_INVALID;
+  double num = 0.0, den = 0.0;
+  for (int i = 0; i < n; ++i) {
+    if (tau[i] < 0 || !std::isfinite(C[i])) return BR_ERR_INVALID;
+    const double c2 = C[i] * C[i];
+    num += c2 * (double)tau[i] * (double)tau[i];
+    den += c2;
+  }
+  if (!(den > 0.0)) return BR_ERR_INVALID;
+  *out = std::sqrt(num / den);
+  return BR_OK;
+}
+
 const char* br_strerror(int status) {
   switch (status) {
     case BR_OK: return "ok";

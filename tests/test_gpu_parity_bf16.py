@@ -141,3 +141,16 @@ def test_momentum_accessor_round_trip_tensor_core():
             assert rel_l2(dg[0], do[0]) <= TOL_DW
     finally:
         sbs.close()
+
+
+def test_stage_aware_delays_and_refresh_periods():
+    """Stage-dependent delays tau = K - k (Sec. 2.3) with the refresh period of each stage taken from
+    the App. I rule (P = 8, f0 = 3: periods 1, 2, 4, 9 for delays 5, 4, 3, 2), one handle, tensor-core
+    path: every layer follows its own delay and schedule."""
+    import paper_2602_03515_b200 as br
+    taus = [5, 4, 3, 2]
+    freqs = [br.br_stage_aware_freq(8, t, 3) for t in taus]
+    assert freqs == [1, 2, 4, 9]
+    layers = [LayerSpec(f"stage{i}", 128, 136, GEOM_BI, SRC_SECOND, t, f) for i, (t, f) in enumerate(zip(taus, freqs))]
+    w = Workload("stages", layers, "bf16", "iid_normal", 0.02, tau=5, freq=3, calls=16, seed=12)
+    _run(w, 16, tau=-1)

@@ -82,3 +82,28 @@ def test_ring_total_grows_with_tau(br):
     t0, _ = br.br_state_bytes([_desc(br, 64, 32, 2, 2, tau=0)], _hp(br))
     t4, _ = br.br_state_bytes([_desc(br, 64, 32, 2, 2, tau=4)], _hp(br))
     assert t4 - t0 == 4 * 64 * 32 * 4
+
+
+def test_stage_aware_helpers_match_the_oracle(br):
+    """Host-only helpers of the stage-aware operation (App. I rule, Eq. (effective-delay)) against
+    the oracle's rational-arithmetic / numpy statements of the same formulas."""
+    import numpy as np
+    from oracle import br_oracle as O
+    for P in (4, 8, 9, 32, 33):
+        for f0 in (1, 10, 14, 50):
+            for tau in range(0, P + 3):
+                try:
+                    want = O.stage_aware_freq(P, tau, f0)
+                except ValueError:
+                    with pytest.raises(br.BrError) as e:
+                        br.br_stage_aware_freq(P, tau, f0)
+                    assert e.value.status == br.BR_ERR_INVALID
+                    continue
+                assert br.br_stage_aware_freq(P, tau, f0) == want, (P, tau, f0)
+    rng = np.random.default_rng(0)
+    for n in (1, 5, 32):
+        c = rng.uniform(0.1, 3.0, n)
+        t = rng.integers(0, 32, n)
+        assert abs(br.br_effective_delay(c, t) - O.effective_delay(c, t)) < 1e-12
+    with pytest.raises(br.BrError):
+        br.br_effective_delay([0.0, 0.0], [1, 2])

@@ -394,3 +394,30 @@ def test_forced_refresh_matches_scheduled_and_rejects_t0():
     q, r_ = np.linalg.qr(lay.L)       # U was I: Power(L, I) = qr(L)
     assert np.allclose(lay.U, q * np.sign(np.diag(r_))[None, :], atol=1e-12)
     assert lay.t == t and lay.refresh_count == 1
+
+
+def test_stage_aware_frequency_rule_hand_values():
+    """App. I with P = 32 (mid = 15) and f0 = 10, worked by hand from the printed rule:
+    tau = 31: n = -16, 1 - n/mid = 31/15, f = floor(150/31) = 4;   tau = 16: n = -1, f = floor(150/16) = 9;
+    tau = 15: n = 1, f = floor(150/14) = 10;   tau = 8: n = 8, f = floor(150/7) = 21;   tau = 2: n = 14, f = 150.
+    tau = 1 divides by zero and tau = 0 goes negative: undefined.  The period shrinks as the delay grows."""
+    for tau, want in ((31, 4), (16, 9), (15, 10), (8, 21), (2, 150)):
+        assert O.stage_aware_freq(32, tau, 10) == want
+    for tau in (0, 1):
+        with pytest.raises(ValueError):
+            O.stage_aware_freq(32, tau, 10)
+    with pytest.raises(ValueError):
+        O.stage_aware_freq(3, 1, 10)
+    fs = [O.stage_aware_freq(32, tau, 10) for tau in range(2, 32)]
+    assert all(a >= b for a, b in zip(fs, fs[1:]))
+    assert O.stage_aware_freq(32, 15, 14) == 15          # exactly 14 / (14/15): no floating-point floor slip
+
+
+def test_effective_delay_closed_forms():
+    """Eq. (effective-delay): one group gives its own delay; equal constants give the root mean square;
+    a group with a zero constant does not count; scaling all constants changes nothing."""
+    assert O.effective_delay([3.0], [7]) == pytest.approx(7.0)
+    assert O.effective_delay([1, 1, 1, 1], [0, 1, 2, 3]) == pytest.approx(np.sqrt(14 / 4))
+    assert O.effective_delay([2.0, 0.0], [5, 100]) == pytest.approx(5.0)
+    assert O.effective_delay([1, 2, 3], [3, 2, 1]) == pytest.approx(O.effective_delay([10, 20, 30], [3, 2, 1]))
+    assert O.effective_delay([1, 2, 3], [3, 2, 1]) == pytest.approx(np.sqrt((9 + 16 + 9) / 14))

@@ -92,11 +92,29 @@ def qr_pos(A: np.ndarray):
     return Q, R, deficient
 
 
+COMPLETION = 1e-6
+
+
+def qr_completed(A: np.ndarray, Qprev: np.ndarray):
+    """Q factor of A with a positive diagonal of R.  The paper does not say what Power() returns
+    when F Q is rank-deficient (S = 1st on the larger side of a bilateral layer: M M^T has rank
+    <= min(m, n)).  Reading taken here: whenever the plain factorisation meets a negligible pivot,
+    the directions outside the range of A are completed from the current basis, by factorising
+    A with COMPLETION * ||A_j|| * Qprev_j added to every column j (a zero column becomes Qprev_j),
+    which has full rank when Qprev has.  The rule is invariant to a rescaling of A or of its columns."""
+    Q, R, d = qr_pos(A)
+    if d:
+        cn = np.linalg.norm(A, axis=0)
+        w = np.where(cn > 0.0, COMPLETION * cn, 1.0)
+        Q, R, _ = qr_pos(A + Qprev * w[None, :])
+    return Q, R, d
+
+
 def power(F: np.ndarray, Q: np.ndarray, iters: int = 1):
     """Power(F, Q): `iters` times Q <- qr(F Q).Q (Sec. 3.2; the paper uses 1)."""
     deficient = False
     for _ in range(iters):
-        Q, _, d = qr_pos(F @ Q)
+        Q, _, d = qr_completed(F @ Q, Q)
         deficient |= d
     return Q, deficient
 
@@ -233,7 +251,7 @@ def _power_with_pivot(F, Q, iters):
     deficient, piv = False, np.inf
     for _ in range(iters):
         A = F @ Q
-        Q, R, d = qr_pos(A)
+        Q, R, d = qr_completed(A, Q)
         deficient |= d
         cn = np.linalg.norm(A, axis=0)
         cn[cn == 0] = 1.0

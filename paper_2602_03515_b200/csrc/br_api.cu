@@ -192,7 +192,7 @@ void layout(br_handle* h, Bump& b, Sizes* sz) {
       ln.rA = b.take<double>(max_k * max_k);
       ln.rF = b.take<double>(max_k * max_k);
       ln.rQ = b.take<double>(max_k * max_k);
-      ln.rWork = b.take<double>(qr_work_doubles((int64_t)max_k));
+      ln.rWork = b.take<double>(std::max<size_t>(qr_work_doubles((int64_t)max_k), 1056));   // also 1025 doubles of norm scratch
       if (max_z) ln.rZ = b.take<double>(max_z);
       if (h->tcq_bytes) ln.tcq_scratch = b.take<char>(h->tcq_bytes);
     }
@@ -258,6 +258,18 @@ br_status refresh_side(br_handle* h, Layer& L, bool left_side, br_handle::Lane& 
       BR_CUDA(h, sdgemm(0, 0, m, n, n, 1.0, Mo, n, Q, n, 0.0, ln.rZ, n, s));
       BR_CUDA(h, fdgemm(1, 0, n, n, m, 1.0, Mo, n, ln.rZ, n, 0.0, ln.rA, n, s));
       count(h, 2); h->stats.gemm_flops += 4.0 * n * n * m;
+    }
+    // A rank-deficient product has no unique Q factor.  Which products are is known on the host: with
+    // S = 1st, M M^T (M^T M) has rank <= min(m, n), short of the larger side; with S = 2nd, a factor that
+    // has accumulated a gradients has rank <= a * (the other dimension).  The directions outside the
+    // range of F Q are then completed from the current basis: what is orthonormalised is F Q with
+    // 1e-6 ||(F Q)_j|| Q_j added to every column j (full rank whenever Q is).
+    const int64_t other = left_side ? n : m;
+    const bool short_of_rank = (L.d.src == BR_SRC_FIRST) ? (k > other)
+                                                         : (L.n_accum < (k + other - 1) / other);
+    if (short_of_rank) {
+      BR_CUDA(h, qr_complete_columns(ln.rA, Q, k, ln.rWork, h->d_status, s));
+      count(h, 3);
     }
     const int ci = 2 * (int)(&L - h->layers.data()) + (left_side ? 0 : 1);
     QrTc* tcq = nullptr;
@@ -350,6 +362,7 @@ br_status accumulate_factors_simt(br_handle* h, Layer& L, const float* G) {
     BR_CUDA(h, sgemm(1, 0, n, n, m, 1.0f - beta, G, n, G, n, beta, L.R, n, h->stream));
     count(h); h->stats.gemm_flops += 2.0 * n * n * m;
   }
+  L.n_accum += 1;
   return BR_OK;
 }
 
@@ -759,6 +772,7 @@ br_status br_set_counters(br_handle* h, int layer, const br_counters* in) {
   h->calls = in->calls;
   L.t = in->t;
   L.refresh_count = in->refresh_count;
+  L.n_accum = std::max(L.n_accum, h->hp.accum == BR_ACCUM_EVERY_STEP ? in->t : in->refresh_count);
   {
     br_status st = check_handle(h);
     if (st != BR_OK) return st;
@@ -852,6 +866,7 @@ br_status br_set_state(br_handle* h, int layer, int which, const void* host_src,
   } else {
     BR_CUDA(h, cudaMemcpy(p, host_src, bytes, cudaMemcpyHostToDevice));
   }
+  if (which == BR_BUF_L || which == BR_BUF_R) L.n_accum = (int64_t)1 << 40;   // a factor given by the caller: taken as full rank
   if (L.use_tc && which == BR_BUF_U) { BR_CUDA(h, split_bf16(L.U, L.Uh, L.Ul, L.d.m * L.d.m, h->stream)); count(h); }
   if (L.use_tc && which == BR_BUF_V) { BR_CUDA(h, split_bf16(L.V, L.Vh, L.Vl, L.d.n * L.d.n, h->stream)); count(h); }
   BR_CUDA(h, cudaStreamSynchronize(h->stream));

@@ -123,6 +123,10 @@ size_t qr_tc_scratch_bytes(int64_t k);
 QrTc* qr_tc_create(int64_t k, char* scratch, int device, cudaStream_t s, const char** err);
 void qr_tc_destroy(QrTc* t);
 int64_t qr_tc_order(const QrTc* t);
+// Completion of a product that is short of rank: A[:, j] += 1e-6 * ||A[:, j]|| * Q[:, j] (Q fp32, the
+// current basis; a zero column becomes Q[:, j]), and BR_WARN_RANK_DEFICIENT is raised in *status.
+// work: the QR work area of this order (used for the column norms).
+cudaError_t qr_complete_columns(double* A, const float* Q, int64_t k, double* work, int* status, cudaStream_t s);
 cudaError_t qr_tc_project(QrTc* t, int node, double* A, int64_t k, int64_t jp, int64_t wp, int64_t jt,
                           int64_t wt, int* status, cudaStream_t s);
 // tc: null, or the plans for this order: the first sweep then projects on the tensor cores (ask for it

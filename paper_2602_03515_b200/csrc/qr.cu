@@ -417,6 +417,38 @@ inline int64_t proj_part_doubles(int64_t k) {
 
 }  // namespace
 
+namespace {
+constexpr double kCompletion = 1e-6;
+__global__ void __launch_bounds__(256)
+k_complete_columns(double* __restrict__ A, const float* __restrict__ Q, int64_t k, const double* __restrict__ norm2,
+                   int* __restrict__ status) {
+  const int64_t total = k * k;
+  if (blockIdx.x == 0 && threadIdx.x == 0) atomicMax(status, (int)BR_WARN_RANK_DEFICIENT);
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t c = i % k;
+    const double n2 = norm2[c];
+    const double d = n2 > 0.0 ? kCompletion * sqrt(n2) : 1.0;
+    A[i] = fma(d, (double)Q[i], A[i]);
+  }
+}
+}  // namespace
+
+cudaError_t qr_complete_columns(double* A, const float* Q, int64_t k, double* work, int* status, cudaStream_t s) {
+  // column norms exactly as the factorisation computes them (same kernels, same order)
+  double* part = work;                                   // kNormChunks * k doubles at most (see qr_work_doubles)
+  const int nchunks = (int)std::min<int64_t>(kNormChunks, std::max<int64_t>(1, k / 4));
+  const int64_t rows_per_chunk = cdiv(k, nchunks);
+  const int used = (int)cdiv(k, rows_per_chunk);
+  double* norm2 = part + (int64_t)used * k;
+  int* dummy = reinterpret_cast<int*>(norm2 + k);
+  dim3 grid((unsigned)cdiv(k, 256), (unsigned)used);
+  k_column_norms_partial<<<grid, 256, 0, s>>>(A, k, rows_per_chunk, part);
+  k_column_norms_sum<<<(unsigned)cdiv(k, 256), 256, 0, s>>>(part, k, used, norm2, dummy);
+  const int64_t blocks = cdiv(k * k, 256);
+  k_complete_columns<<<(unsigned)(blocks < 1184 ? blocks : 1184), 256, 0, s>>>(A, Q, k, norm2, status);
+  return cudaGetLastError();
+}
+
 size_t qr_work_doubles(int64_t k) {
   const int64_t b = std::min<int64_t>(panel_width(k), k);
   return (size_t)(pad32((int64_t)gram_splits(k) * b * b) + 2 * pad32(b * b) + 64 + pad32(k) +

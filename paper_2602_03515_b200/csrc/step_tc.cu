@@ -397,12 +397,17 @@ int tc_step_run(TcStep* t, std::vector<Layer>& layers, const std::vector<const v
     if (!any) continue;
     int rc;
     if ((rc = lz.run(c.factors, "factor launch", calls, tau, dyn_alpha, dyn_beta))) return rc;
+    if (c.factors)
+      for (int i : c.ids) if (G[i]) layers[i].n_accum += 1;
     std::vector<int> due, due_slots;
     for (size_t j = 0; j < c.ids.size(); ++j) {
       const int i = c.ids[j];
       Layer& L = layers[i];
       if (!G[i] || L.t % L.freq != 0) continue;
-      if (t->factor_plan[i] && (rc = lz.run(t->factor_plan[i], "factor launch", calls, tau, dyn_alpha, dyn_beta))) return rc;
+      if (t->factor_plan[i]) {
+        if ((rc = lz.run(t->factor_plan[i], "factor launch", calls, tau, dyn_alpha, dyn_beta))) return rc;
+        L.n_accum += 1;
+      }
       due.push_back(i);
       due_slots.push_back((int)j);
     }

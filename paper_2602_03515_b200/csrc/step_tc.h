@@ -21,6 +21,7 @@ struct Layer {
   int ring_slots = 0;                 // physical slots: tau_max, or 1 for a tensor-core layer without delay
   size_t slot_stride = 0;             // bytes between ring slots
   int64_t t = 0, refresh_count = 0;
+  int64_t n_accum = 0;                // gradients accumulated into L / R so far (bounds their rank)
 };
 
 std::string format(const char* fmt, ...);

@@ -145,7 +145,7 @@ def test_refresh_tensor_core_projections_order_4224():
     import paper_2602_03515_b200 as br
     from tests.parity_util import basis_err
     k = 4224
-    F = _lowrank_noise_factor(k, 16, 33, samples=1)
+    F = _lowrank_noise_factor(k, 16, 33, samples=3)      # 13,000 noise samples: the noise part is well conditioned
     w = torch.zeros(k, 8, device="cuda")
     opt = br.BasisRotation([LayerSpec("W", k, 8, GEOM_BI, SRC_SECOND, 0)], [w], grad_dtype="bf16",
                            gemm_prec=br.BR_GEMM_BF16, freq=10 ** 6)
@@ -170,7 +170,7 @@ def test_refresh_tensor_core_projections_order_4224():
 
 def test_refresh_order_6912_properties():
     k = 6912
-    F = _lowrank_noise_factor(k, 32, 32, samples=1)
+    F = _lowrank_noise_factor(k, 32, 32, samples=2)      # 14,000 noise samples for order 6912: full rank with margin
     Q0 = np.eye(k, dtype=np.float32)
     U1 = _forced_refresh(k, F, Q0)                      # ill-conditioned first refresh
     U1f = U1.astype(np.float32)

@@ -20,10 +20,14 @@ def _run(w, calls, tau=-1, tol=TOL_DW, **kw):
     import paper_2602_03515_b200 as br
     sbs = SideBySide(w, gemm_prec=br.BR_GEMM_BF16, **kw)
     worst = 0.0
+    deficient = False
     try:
         for c in range(calls):
             st_g, st_o, dg, do = sbs.step(tau)
-            assert st_g == st_o, (c, st_g, st_o)
+            # (a rank-deficient refresh is reported by the oracle's step at once, by the library through
+            # the status word that br_sync_status reads)
+            assert st_g == st_o or (st_g == br.BR_OK and st_o == 2), (c, st_g, st_o)
+            deficient = deficient or st_o == 2
             for li, (a, b) in enumerate(zip(dg, do)):
                 if b is None:
                     assert not np.any(a)
@@ -33,7 +37,7 @@ def _run(w, calls, tau=-1, tol=TOL_DW, **kw):
                 assert e <= tol, (c, li, e)
             for li in range(len(w.layers)):
                 assert sbs.opt.counters(li) == sbs.oracle.counters(li)
-        assert sbs.opt.sync_status() == br.BR_OK
+        assert sbs.opt.sync_status() == (br.BR_WARN_RANK_DEFICIENT if deficient else br.BR_OK)
         for li, lay in enumerate(sbs.oracle.layers):
             # the tensor-core path keeps M~ = U^T M V (accumulated from bf16-pair products); M is U M~ V^T
             assert rel_l2(sbs.state(li, br.BR_BUF_M), lay.M) < 1e-4
@@ -145,12 +149,21 @@ def test_momentum_accessor_round_trip_tensor_core():
 
 def test_stage_aware_delays_and_refresh_periods():
     """Stage-dependent delays tau = K - k (Sec. 2.3) with the refresh period of each stage taken from
-    the App. I rule (P = 8, f0 = 3: periods 1, 2, 4, 9 for delays 5, 4, 3, 2), one handle, tensor-core
+    the App. I rule (P = 8, f0 = 6: periods 3, 4, 9, 18 for delays 5, 4, 3, 2), one handle, tensor-core
     path: every layer follows its own delay and schedule."""
     import paper_2602_03515_b200 as br
     taus = [5, 4, 3, 2]
-    freqs = [br.br_stage_aware_freq(8, t, 3) for t in taus]
-    assert freqs == [1, 2, 4, 9]
+    freqs = [br.br_stage_aware_freq(8, t, 6) for t in taus]
+    assert freqs == [3, 4, 9, 18]
     layers = [LayerSpec(f"stage{i}", 128, 136, GEOM_BI, SRC_SECOND, t, f) for i, (t, f) in enumerate(zip(taus, freqs))]
-    w = Workload("stages", layers, "bf16", "iid_normal", 0.02, tau=5, freq=3, calls=16, seed=12)
-    _run(w, 16, tau=-1)
+    w = Workload("stages", layers, "bf16", "iid_normal", 0.02, tau=5, freq=6, calls=22, seed=12)
+    _run(w, 22, tau=-1)
+
+
+def test_bilateral_first_moment_rectangular_completion():
+    """Bilateral S=1st on rectangular matrices: M M^T (or M^T M) is short of rank on the larger side
+    at every refresh, so the basis there is completed from the previous one (same rule in the oracle
+    and in the library); tensor-core path, both orientations."""
+    layers = [LayerSpec("wide", 128, 200, GEOM_BI, SRC_FIRST, 1), LayerSpec("tall", 264, 136, GEOM_BI, SRC_FIRST, 1)]
+    w = Workload("bi1st", layers, "bf16", "iid_normal", 0.02, tau=1, freq=4, calls=14, seed=13)
+    _run(w, 14, tau=1)

@@ -211,6 +211,33 @@ def test_p6_rank_deficient_flag_and_orthonormality():
     assert dz and np.allclose(Qz.T @ Qz, np.eye(4))
 
 
+def test_p6_rank_deficient_completion_from_the_previous_basis():
+    """Power(F, Q) with a rank-2 F of order 7: the first two columns are the unique Q factor of the
+    range (they match LAPACK's QR of F Q); the other five complete the basis from the previous one:
+    the whole result equals LAPACK's QR of F Q + 1e-6 Q diag(||(F Q)_j||) (full rank, hence unique) after the
+    sign fix, it is orthonormal, and the completed columns span the orthogonal complement of the range."""
+    k, r = 7, 2
+    B = rng(21).standard_normal((k, r))
+    F = B @ B.T
+    Qprev, _ = np.linalg.qr(rng(22).standard_normal((k, k)))
+    Q, deficient = O.power(F, Qprev)
+    assert deficient
+    assert np.max(np.abs(Q.T @ Q - np.eye(k))) < 1e-9
+    A = F @ Qprev
+    q0, r0 = np.linalg.qr(A[:, :r])
+    assert np.max(np.abs(Q[:, :r] - q0 * np.sign(np.diag(r0)))) < 1e-4     # moved by the 1e-6 term only
+    q1, r1 = np.linalg.qr(A + 1e-6 * Qprev * np.linalg.norm(A, axis=0)[None, :])
+    assert np.max(np.abs(Q - q1 * np.sign(np.diag(r1)))) < 1e-8
+    # the leading columns span the range of F, the completed ones its orthogonal complement
+    lead, rest = Q[:, :r], Q[:, r:]
+    assert np.linalg.norm(F - lead @ (lead.T @ F)) < 1e-4 * np.linalg.norm(F)
+    assert np.linalg.norm(F @ rest) < 1e-4 * np.linalg.norm(F)
+    # a full-rank product is left alone (bit for bit the plain factorisation)
+    F2 = F + np.eye(k)
+    Q2, d2 = O.power(F2, Qprev)
+    assert not d2 and np.array_equal(Q2, O.qr_pos(F2 @ Qprev)[0])
+
+
 # P7 -- Kronecker-factored covariance (Theorem 3.1 and its lemma)
 def test_p7_kronecker_structure_and_norm_chain():
     r = rng(10)

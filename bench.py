@@ -145,7 +145,7 @@ def fit_tau(w_name, n_layers, tau_req, gemm_prec, free_bytes, margin, br):
         descs = [br.BrLayerDesc(m=l.m, n=l.n, geom=l.geom, src=l.src, grad_dtype=br.BR_BF16 if w.grad_dtype == "bf16" else br.BR_F32,
                                 tau_max=l.tau_max, freq=0, reserved=0, weight=0) for l in w.layers]
         hp = br.BrHparams(lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps, weight_decay=0.0, beta_factor=-1.0, freq=w.freq,
-                          power_iters=1, accum=0, gemm_prec=gemm_prec, flags=0, reserved=0, scratch_limit_bytes=0)
+                          power_iters=1, accum=0, gemm_prec=gemm_prec, flags=0, clip_norm=0.0, scratch_limit_bytes=0)
         return br.br_state_bytes(descs, hp)[0]
     tau = tau_req
     while tau > 1 and total(tau) > free_bytes - margin:

@@ -94,7 +94,10 @@ typedef struct {
   int32_t accum;       /* br_accum_mode                                                    */
   int32_t gemm_prec;   /* br_gemm_prec                                                     */
   uint32_t flags;      /* reserved, 0                                                      */
-  int32_t reserved;
+  /* Global-norm gradient clipping (App. D.2 of the paper uses 1.0); 0 = off.  The gradients of one
+   * call, over all layers of the handle, are scaled by min(1, clip_norm / their joint L2 norm); the
+   * factor belongs to the call and goes with its gradients through the delay ring. */
+  float clip_norm;
   uint64_t scratch_limit_bytes; /* cap on per-step transient scratch; 0 -> library default */
 } br_hparams;
 
@@ -134,7 +137,10 @@ typedef enum {
    * what layers on the tensor-core path store; BR_BUF_M converts on the way in and out with fp32
    * products.  A checkpoint that must resume bit-identically saves and restores this buffer (after
    * U and V) instead of BR_BUF_M.  Absent for layers on the fp32 path. */
-  BR_BUF_MROT = 8
+  BR_BUF_MROT = 8,
+  /* max(tau_max) + 1 floats: the clipping factors of the last calls (slot = (call - 1) mod length),
+   * a handle-wide buffer read and written with layer = 0; absent when clip_norm == 0. */
+  BR_BUF_CLIP = 9
 } br_buf;
 
 /* Bytes of device memory br_create would request for these layers (state, ring, operand
@@ -223,6 +229,16 @@ BR_API br_status br_stage_aware_freq(int P, int tau, int f0, int* out_freq);
  * tau_i >= 0 (HOST array).  Host only.
  */
 BR_API br_status br_effective_delay(const double* C, const int* tau, int n, double* out);
+
+/*
+ * Learning-rate schedule of the paper's runs (App. D.2): linear warm-up over the first
+ * warmup_fraction of total_steps (the paper uses 0.012), then cosine decay that would reach min_lr at step = total_steps:
+ *   step <  W = ceil(warmup_fraction * total_steps):  base_lr * (step + 1) / W
+ *   step >= W:  min_lr + (base_lr - min_lr) * (1 + cos(pi * (step - W) / max(1, total_steps - W))) / 2
+ * step counts from 0.  Host only; the result is what br_set_lr takes.
+ */
+BR_API br_status br_lr_warmup_cosine(int64_t step, int64_t total_steps, double warmup_fraction, double base_lr,
+                                     double min_lr, double* out_lr);
 
 BR_API const char* br_strerror(int status);
 /* Message of the last error on this handle (or of the last failed br_create when h is NULL). */

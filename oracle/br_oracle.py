@@ -176,6 +176,7 @@ class Hyper:
     freq: int = 10
     power_iters: int = 1
     accum: str = "every_step"      # or "on_refresh" (literal Algorithm 2)
+    clip_norm: float = 0.0         # global-norm gradient clipping (App. D.2 uses 1.0); 0 = off
 
 
 class OracleLayer:
@@ -266,6 +267,7 @@ class Oracle:
         self.layers = list(layers)
         self.hp = hp
         self.calls = 0
+        self.clip_of_call = {}     # call index -> clipping factor of that call's gradients
 
     def _beta_factor(self):
         return self.hp.beta2 if self.hp.beta_factor < 0 else self.hp.beta_factor
@@ -279,6 +281,12 @@ class Oracle:
         """
         hp = self.hp
         self.calls += 1
+        if hp.clip_norm > 0.0:
+            # App. D.2 ("gradient clipping value of 1.0"): the gradients of one call, all layers
+            # together, are scaled to a joint L2 norm of at most clip_norm.  The factor belongs to
+            # the call: a layer that applies g_c later applies the clipped g_c.
+            nrm = np.sqrt(sum(float(np.sum(np.asarray(g, dtype=np.float64) ** 2)) for g in grads))
+            self.clip_of_call[self.calls] = hp.clip_norm / nrm if nrm > hp.clip_norm else 1.0
         applied, deficient = False, False
         for lay, g in zip(self.layers, grads):
             g = np.asarray(g, dtype=np.float64)
@@ -296,6 +304,8 @@ class Oracle:
                 lay.last_dW = None
                 continue
             applied = True
+            if hp.clip_norm > 0.0:
+                G = self.clip_of_call[src_call] * G
             deficient |= self._update(lay, G)
         if not applied:
             return STATUS_WARMUP
@@ -369,6 +379,18 @@ def stage_aware_freq(P: int, tau: int, f0: int) -> int:
     if den <= 0:
         raise ValueError("the rule divides by zero or goes negative at this delay")
     return max(1, floor(Fraction(f0) / den))
+
+
+def lr_warmup_cosine(step: int, total_steps: int, warmup_fraction: float, base_lr: float, min_lr: float = 0.0) -> float:
+    """Learning-rate schedule of the paper's runs (App. D.2): linear warm-up over the first
+    warmup_fraction of the iterations (0.012 in the paper), cosine decay for the rest (towards min_lr,
+    which it would reach at step = total_steps).  `step` counts from 0."""
+    import math
+    W = math.ceil(warmup_fraction * total_steps)
+    if step < W:
+        return base_lr * (step + 1) / W
+    rest = max(1, total_steps - W)
+    return min_lr + (base_lr - min_lr) * 0.5 * (1.0 + math.cos(math.pi * (step - W) / rest))
 
 
 def effective_delay(consts, taus) -> float:

@@ -17,7 +17,7 @@ BR_SRC_FIRST, BR_SRC_SECOND = 1, 2
 BR_F32, BR_BF16 = 0, 1
 BR_GEMM_FP32, BR_GEMM_BF16 = 0, 2
 BR_ACCUM_EVERY_STEP, BR_ACCUM_ON_REFRESH = 0, 1
-BR_BUF_W, BR_BUF_M, BR_BUF_V2, BR_BUF_U, BR_BUF_V, BR_BUF_L, BR_BUF_R, BR_BUF_RING, BR_BUF_MROT = range(9)
+BR_BUF_W, BR_BUF_M, BR_BUF_V2, BR_BUF_U, BR_BUF_V, BR_BUF_L, BR_BUF_R, BR_BUF_RING, BR_BUF_MROT, BR_BUF_CLIP = range(10)
 
 
 class BrError(RuntimeError):
@@ -36,7 +36,7 @@ class BrHparams(C.Structure):
     _fields_ = [("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
                 ("weight_decay", C.c_float), ("beta_factor", C.c_float), ("freq", C.c_int32),
                 ("power_iters", C.c_int32), ("accum", C.c_int32), ("gemm_prec", C.c_int32),
-                ("flags", C.c_uint32), ("reserved", C.c_int32), ("scratch_limit_bytes", C.c_uint64)]
+                ("flags", C.c_uint32), ("clip_norm", C.c_float), ("scratch_limit_bytes", C.c_uint64)]
 
 
 class BrCounters(C.Structure):
@@ -97,6 +97,7 @@ def load_library():
         "br_get_profile": ([H, C.POINTER(BrProfileStats)], C.c_int),
         "br_stage_aware_freq": ([C.c_int, C.c_int, C.c_int, C.POINTER(C.c_int)], C.c_int),
         "br_effective_delay": ([C.POINTER(C.c_double), C.POINTER(C.c_int), C.c_int, C.POINTER(C.c_double)], C.c_int),
+        "br_lr_warmup_cosine": ([C.c_int64, C.c_int64, C.c_double, C.c_double, C.c_double, C.POINTER(C.c_double)], C.c_int),
         "br_destroy": ([H], C.c_int),
         "br_power_static": ([C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p], C.c_int),
         "br_strerror": ([C.c_int], C.c_char_p),
@@ -222,6 +223,13 @@ def br_effective_delay(consts, taus) -> float:
     return float(out.value)
 
 
+def br_lr_warmup_cosine(step: int, total_steps: int, warmup_fraction: float, base_lr: float, min_lr: float = 0.0) -> float:
+    out = C.c_double(0.0)
+    _check(load_library().br_lr_warmup_cosine(int(step), int(total_steps), float(warmup_fraction), float(base_lr),
+                                              float(min_lr), C.byref(out)))
+    return float(out.value)
+
+
 def br_destroy(handle) -> int:
     return load_library().br_destroy(handle)
 
@@ -251,7 +259,7 @@ class BasisRotation:
 
     def __init__(self, specs, weights, *, grad_dtype: str = "bf16", lr=1e-3, beta1=0.9, beta2=0.999,
                  eps=1e-8, weight_decay=0.0, beta_factor=-1.0, freq=10, power_iters=1,
-                 accum=BR_ACCUM_EVERY_STEP, gemm_prec=BR_GEMM_BF16, scratch_limit_bytes=0,
+                 accum=BR_ACCUM_EVERY_STEP, gemm_prec=BR_GEMM_BF16, scratch_limit_bytes=0, clip_norm=0.0,
                  device=None, stream=None, use_torch_allocator=True):
         import torch
         self._torch = torch
@@ -271,7 +279,7 @@ class BasisRotation:
                                            weight=w.data_ptr()))
         self.hp = BrHparams(lr=lr, beta1=beta1, beta2=beta2, eps=eps, weight_decay=weight_decay,
                             beta_factor=beta_factor, freq=freq, power_iters=power_iters, accum=accum,
-                            gemm_prec=gemm_prec, flags=0, reserved=0, scratch_limit_bytes=scratch_limit_bytes)
+                            gemm_prec=gemm_prec, flags=0, clip_norm=clip_norm, scratch_limit_bytes=scratch_limit_bytes)
         self._blocks = {}
         self._alloc = None
         if use_torch_allocator:
@@ -339,6 +347,8 @@ class BasisRotation:
             return (s.m, s.m), torch.float32
         if which in (BR_BUF_V, BR_BUF_R):
             return (s.n, s.n), torch.float32
+        if which == BR_BUF_CLIP:
+            return (max(x.tau_max for x in self.specs) + 1,), torch.float32
         return (s.tau_max, s.m, s.n), (torch.bfloat16 if self.grad_dtype == "bf16" else torch.float32)
 
     def get_state(self, layer: int, which: int):

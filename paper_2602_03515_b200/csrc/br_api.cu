@@ -57,6 +57,7 @@ br_status validate(const br_layer_desc* layers, int n_layers, const br_hparams* 
       !(hp->eps >= 0.f) || !(hp->beta_factor < 1.f) || !std::isfinite(hp->lr) || !(hp->weight_decay >= 0.f)) {
     *err = "hyper-parameter out of range"; return BR_ERR_INVALID;
   }
+  if (!(hp->clip_norm >= 0.f) || !std::isfinite(hp->clip_norm)) { *err = "clip_norm must be finite and >= 0"; return BR_ERR_INVALID; }
   if (hp->freq < 1 || hp->power_iters < 1) { *err = "freq and power_iters must be >= 1"; return BR_ERR_INVALID; }
   if (hp->accum != BR_ACCUM_EVERY_STEP && hp->accum != BR_ACCUM_ON_REFRESH) { *err = "bad accum mode"; return BR_ERR_INVALID; }
   if (hp->gemm_prec != BR_GEMM_FP32 && hp->gemm_prec != BR_GEMM_BF16) { *err = "bad gemm_prec"; return BR_ERR_INVALID; }
@@ -111,6 +112,10 @@ struct br_handle {
   // Conditioning notes of the last refresh, per layer and side (index 2 * layer + (right side)):
   // written on the device by the refresh, copied to pinned host memory after every batch, read by
   // the host before the next one (which then decides where the block projections run).
+  // global-norm clipping: factor of each of the last calls (slot (call - 1) mod clip_slots)
+  float* d_clip = nullptr;
+  int clip_slots = 0;
+  double* d_clip_part = nullptr;
   int* d_cond = nullptr;
   int* h_cond = nullptr;
   std::vector<int> cond_known;
@@ -198,6 +203,13 @@ void layout(br_handle* h, Bump& b, Sizes* sz) {
     }
   }
   h->d_cond = b.take<int>(2 * h->layers.size() + 2);
+  if (hp.clip_norm > 0.f) {
+    int tmax = 0;
+    for (const Layer& L : h->layers) tmax = std::max(tmax, (int)L.d.tau_max);
+    h->clip_slots = tmax + 1;
+    h->d_clip = b.take<float>((size_t)h->clip_slots);
+    h->d_clip_part = b.take<double>(296 * ((h->layers.size() + 63) / 64));
+  }
   h->d_status = b.take<int>(64);
   (void)hp;
   sz->total = b.off;
@@ -415,16 +427,18 @@ void tmp_free(br_handle* h, void* p) {
 }
 
 // One update of one layer on the accurate (fp32 FFMA) path.  G: the gradient to apply.
-br_status update_layer_simt(br_handle* h, Layer& L, const void* G) {
+br_status update_layer_simt(br_handle* h, Layer& L, const void* G, const float* gscale) {
   const br_hparams& hp = h->hp;
   cudaStream_t s = h->stream;
   const int64_t m = L.d.m, n = L.d.n, mn = m * n;
   const int bf = L.d.grad_dtype == BR_BF16;
   br_status st;
   // Alg. 1 line 4 (and widen a bf16 gradient once)
-  BR_CUDA(h, ema_momentum(L.M, G, bf, mn, hp.beta1, bf ? h->sG : nullptr, nullptr, nullptr, s));
+  // (a clipped gradient is materialised in fp32 too: everything below works on the scaled values)
+  const bool copy = bf || gscale != nullptr;
+  BR_CUDA(h, ema_momentum(L.M, G, bf, mn, hp.beta1, copy ? h->sG : nullptr, nullptr, nullptr, gscale, s));
   count(h);
-  const float* G32 = bf ? h->sG : reinterpret_cast<const float*>(G);
+  const float* G32 = copy ? h->sG : reinterpret_cast<const float*>(G);
   const bool second = L.d.src == BR_SRC_SECOND;
   if (second && hp.accum == BR_ACCUM_EVERY_STEP && (st = accumulate_factors_simt(h, L, G32)) != BR_OK) return st;
   // Alg. 1 lines 5-6
@@ -602,7 +616,7 @@ br_status br_create(br_handle** out, const br_layer_desc* layers, int n_layers, 
       }
   }
   const char* tc_err = nullptr;
-  h->tc = tc_step_create(h->layers, h->hp, h->slab + sz.total, tc_bytes, device, s, &tc_err);
+  h->tc = tc_step_create(h->layers, h->hp, h->slab + sz.total, tc_bytes, h->d_clip, h->clip_slots, device, s, &tc_err);
   if (!h->tc && tc_err) {
     g_create_error = tc_err;
     if (h->alloc.alloc) h->alloc.free(h->slab, h->alloc.ctx); else cudaFree(h->slab);
@@ -632,7 +646,17 @@ br_status br_step(br_handle* h, const void* const* grads, int tau) {
   }
   // ---- integer state (host) ---------------------------------------------------------------
   h->calls += 1;
+  if (h->d_clip) {
+    // clipping factor of this call's gradients (App. D.2), kept until they are applied
+    std::vector<int64_t> numel(nl);
+    std::vector<int> bf(nl);
+    for (int i = 0; i < nl; ++i) { numel[i] = h->layers[i].d.m * h->layers[i].d.n; bf[i] = h->layers[i].d.grad_dtype == BR_BF16; }
+    BR_CUDA(h, clip_factor(grads, numel.data(), bf.data(), nl, h->hp.clip_norm, h->d_clip_part,
+                           h->d_clip + (h->calls - 1) % h->clip_slots, h->stream));
+    count(h, (nl + 63) / 64 + 1);
+  }
   std::vector<const void*> G(nl, nullptr);
+  std::vector<const float*> GS(nl, nullptr);
   std::vector<char> stored(nl, 0);
   bool any = false;
   for (int i = 0; i < nl; ++i) {
@@ -650,6 +674,7 @@ br_status br_step(br_handle* h, const void* const* grads, int tau) {
       } else {
         G[i] = (tl == 0) ? grads[i] : ring_slot_ptr(L, (src_call - 1) % L.ring_slots);
       }
+      if (h->d_clip) GS[i] = h->d_clip + (src_call - 1) % h->clip_slots;
       L.t += 1;
       any = true;
     }
@@ -661,10 +686,10 @@ br_status br_step(br_handle* h, const void* const* grads, int tau) {
     if (!G[i]) continue;
     if (L.d.geom == BR_GEOM_NONE) {
       BR_CUDA(h, plain_adam(L.d.weight, L.M, L.V2, G[i], L.d.grad_dtype == BR_BF16, L.d.m * L.d.n,
-                            hp.lr, hp.beta1, hp.beta2, hp.eps, hp.weight_decay, h->stream));
+                            hp.lr, hp.beta1, hp.beta2, hp.eps, hp.weight_decay, GS[i], h->stream));
       count(h);
     } else if (!L.use_tc) {
-      if ((st = update_layer_simt(h, L, G[i])) != BR_OK) return st;
+      if ((st = update_layer_simt(h, L, G[i], GS[i])) != BR_OK) return st;
     }
   }
   if (h->tc) {
@@ -793,6 +818,13 @@ br_status br_get_state(br_handle* h, int layer, int which, void* host_dst, size_
   br_status st = check_handle(h);
   if (st != BR_OK) return st;
   if (!host_dst || layer < 0 || layer >= (int)h->layers.size()) { h->err = "bad argument"; return BR_ERR_INVALID; }
+  if (which == BR_BUF_CLIP) {
+    if (!h->d_clip) { h->err = "clipping is off: no such buffer"; return BR_ERR_STATE; }
+    if (bytes != sizeof(float) * (size_t)h->clip_slots) { h->err = "wrong size for the clipping factors"; return BR_ERR_SHAPE; }
+    BR_CUDA(h, cudaStreamSynchronize(h->stream));
+    BR_CUDA(h, cudaMemcpy(host_dst, h->d_clip, bytes, cudaMemcpyDeviceToHost));
+    return BR_OK;
+  }
   const Layer& L = h->layers[layer];
   void* p = nullptr;
   const size_t want = buf_bytes(L, which, &p);
@@ -824,6 +856,13 @@ br_status br_set_state(br_handle* h, int layer, int which, const void* host_src,
   br_status st = check_handle(h);
   if (st != BR_OK) return st;
   if (!host_src || layer < 0 || layer >= (int)h->layers.size()) { h->err = "bad argument"; return BR_ERR_INVALID; }
+  if (which == BR_BUF_CLIP) {
+    if (!h->d_clip) { h->err = "clipping is off: no such buffer"; return BR_ERR_STATE; }
+    if (bytes != sizeof(float) * (size_t)h->clip_slots) { h->err = "wrong size for the clipping factors"; return BR_ERR_SHAPE; }
+    BR_CUDA(h, cudaStreamSynchronize(h->stream));
+    BR_CUDA(h, cudaMemcpy(h->d_clip, host_src, bytes, cudaMemcpyHostToDevice));
+    return BR_OK;
+  }
   Layer& L = h->layers[layer];
   void* p = nullptr;
   const size_t want = buf_bytes(L, which, &p);
@@ -930,6 +969,19 @@ br_status br_destroy(br_handle* h) {
     if (h->alloc.alloc) h->alloc.free(h->slab, h->alloc.ctx); else cudaFree(h->slab);
   }
   delete h;
+  return BR_OK;
+}
+
+br_status br_lr_warmup_cosine(int64_t step, int64_t total_steps, double warmup_fraction, double base_lr,
+                              double min_lr, double* out_lr) {
+  if (!out_lr || total_steps < 1 || step < 0 || step >= total_steps || !(warmup_fraction >= 0.0) ||
+      !(warmup_fraction <= 1.0) || !std::isfinite(base_lr) || !std::isfinite(min_lr))
+    return BR_ERR_INVALID;
+  const int64_t W = (int64_t)std::ceil(warmup_fraction * (double)total_steps);
+  if (step < W) { *out_lr = base_lr * (double)(step + 1) / (double)W; return BR_OK; }
+  const int64_t rest = std::max<int64_t>(1, total_steps - W);
+  const double pi = 3.14159265358979323846;
+  *out_lr = min_lr + (base_lr - min_lr) * 0.5 * (1.0 + std::cos(pi * (double)(step - W) / (double)rest));
   return BR_OK;
 }
 

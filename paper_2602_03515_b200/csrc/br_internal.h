@@ -58,12 +58,17 @@ cudaError_t set_identity(float* Q, int64_t k, cudaStream_t s);
 
 // Alg. 1 line 4: M <- beta1 M + (1-beta1) G.  G is fp32 or bf16 (g_is_bf16).  Optional outputs:
 // Gf32 (G widened to fp32), Mh/Ml (bf16 hi/lo split of the new M).
+// gscale (optional, DEVICE): clipping factor the gradient is multiplied by
 cudaError_t ema_momentum(float* M, const void* G, int g_is_bf16, int64_t numel, float beta1,
-                         float* Gf32, __nv_bfloat16* Mh, __nv_bfloat16* Ml, cudaStream_t s);
+                         float* Gf32, __nv_bfloat16* Mh, __nv_bfloat16* Ml, const float* gscale, cudaStream_t s);
+// Global-norm clipping factor of one call: *out = min(1, clip / ||all gradients||_2).  part: scratch of
+// 296 * ceil(n / 64) doubles.  Fixed summation order.
+cudaError_t clip_factor(const void* const* grads, const int64_t* numel, const int* is_bf16, int n, float clip,
+                        double* part, float* out, cudaStream_t s);
 
 // Eq. (adam): plain Adam, eps inside the sqrt, no bias correction, decoupled weight decay.
 cudaError_t plain_adam(float* W, float* M, float* V, const void* G, int g_is_bf16, int64_t numel,
-                       float lr, float beta1, float beta2, float eps, float wd, cudaStream_t s);
+                       float lr, float beta1, float beta2, float eps, float wd, const float* gscale, cudaStream_t s);
 
 // Alg. 1 lines 10-11 (element-wise part): V~ <- beta2 V~ + (1-beta2) G~^2 ; X = M~/sqrt(V~+eps).
 // X overwrites Mt.
@@ -86,7 +91,7 @@ cudaError_t split3_f32(const float* X, int64_t numel, __nv_bfloat16* p1, __nv_bf
 cudaError_t sub_f32_from_f64(double* A, int64_t ld, int64_t rows, int64_t cols, const float* D, cudaStream_t s);
 // out <- beta1 M + (1-beta1) G (out-of-place form of Alg. 1 line 4)
 cudaError_t ema_out(float* out, const float* M, const void* G, int g_is_bf16, int64_t numel, float beta1,
-                    cudaStream_t s);
+                    const float* gscale, cudaStream_t s);
 
 // ---------------------------------------------------------------------------------------------
 // SIMT contractions (gemm_simt.cu):  C = alpha * op(A) op(B) + beta * C, row-major.
@@ -163,6 +168,10 @@ struct TcProblem {
   int32_t epilogue = EPI_AXPBY_F32;
   int32_t tau_max = 0;            // of the layer (delay bookkeeping on the device)
   int32_t dyn_scalars = 0;        // 1: alpha / beta come from the launch arguments
+  // global-norm clipping: the accumulator of this problem is built from a gradient that carries the
+  // factor clip[(calls - 1 - tau) mod clip_slots]; clip_mode 1 multiplies it by the factor (G~), 2 by
+  // its square (G G^T), 0 leaves it alone
+  const float* clip = nullptr; int32_t clip_slots = 0; int32_t clip_mode = 0;
   int32_t symmetric = 0;          // 1: A_p = B_p and D is square: only tiles touching the upper triangle are
                                   // computed, the rest of D is written as their mirror image (EPI_AXPBY_F32 only)
   float alpha = 1.f, beta = 0.f, eps = 0.f, beta1 = 0.f;

@@ -9,6 +9,13 @@ namespace {
 
 constexpr int kThreads = 256;
 
+template <int NSEG>
+struct ClipSegs {                 // passed by value: one launch covers up to NSEG gradients
+  const void* ptr[NSEG];
+  long long begin[NSEG + 1];      // element offsets in the concatenation
+  int bf16[NSEG];
+};
+
 inline int grid_for(int64_t n_vec) {
   // 148 SMs on a B200, 8 resident CTAs of 256 threads each.
   int64_t want = (n_vec + kThreads - 1) / kThreads;
@@ -69,13 +76,15 @@ template <bool G_BF16>
 __global__ void __launch_bounds__(kThreads)
 k_ema_momentum(float* __restrict__ M, const void* __restrict__ G, int64_t numel, float beta1,
                float* __restrict__ Gf32, __nv_bfloat16* __restrict__ Mh,
-               __nv_bfloat16* __restrict__ Ml) {
+               __nv_bfloat16* __restrict__ Ml, const float* __restrict__ gscale) {
+  const float gs = gscale ? *gscale : 1.0f;     // clipping factor of the call this gradient came with
   const float omb = 1.0f - beta1;
   const int64_t nvec = numel >> 2;
   const int64_t stride = (int64_t)gridDim.x * blockDim.x;
   for (int64_t v = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; v < nvec; v += stride) {
     const int64_t i = v << 2;
     float4 g = load_grad4<G_BF16>(G, i);
+    g.x *= gs; g.y *= gs; g.z *= gs; g.w *= gs;
     float4 m = ld4(M + i);
     m.x = beta1 * m.x + omb * g.x;
     m.y = beta1 * m.y + omb * g.y;
@@ -92,7 +101,7 @@ k_ema_momentum(float* __restrict__ M, const void* __restrict__ G, int64_t numel,
   // ragged tail (numel not a multiple of 4)
   for (int64_t i = (nvec << 2) + blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < numel;
        i += stride) {
-    float g = load_grad1<G_BF16>(G, i);
+    float g = gs * load_grad1<G_BF16>(G, i);
     float m = beta1 * M[i] + omb * g;
     M[i] = m;
     if (Gf32) Gf32[i] = g;
@@ -108,13 +117,15 @@ template <bool G_BF16>
 __global__ void __launch_bounds__(kThreads)
 k_plain_adam(float* __restrict__ W, float* __restrict__ M, float* __restrict__ V,
              const void* __restrict__ G, int64_t numel, float lr, float beta1, float beta2,
-             float eps, float decay) {
+             float eps, float decay, const float* __restrict__ gscale) {
+  const float gs = gscale ? *gscale : 1.0f;
   const float omb1 = 1.0f - beta1, omb2 = 1.0f - beta2;
   const int64_t nvec = numel >> 2;
   const int64_t stride = (int64_t)gridDim.x * blockDim.x;
   for (int64_t v = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; v < nvec; v += stride) {
     const int64_t i = v << 2;
     float4 g = load_grad4<G_BF16>(G, i);
+    g.x *= gs; g.y *= gs; g.z *= gs; g.w *= gs;
     float4 m = ld4(M + i), s = ld4(V + i), w = ld4(W + i);
 #define BR_ADAM1(c)                                   \
   m.c = beta1 * m.c + omb1 * g.c;                     \
@@ -128,7 +139,7 @@ k_plain_adam(float* __restrict__ W, float* __restrict__ M, float* __restrict__ V
   }
   for (int64_t i = (nvec << 2) + blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < numel;
        i += stride) {
-    float g = load_grad1<G_BF16>(G, i);
+    float g = gs * load_grad1<G_BF16>(G, i);
     float m = beta1 * M[i] + omb1 * g;
     float s = beta2 * V[i] + omb2 * g * g;
     M[i] = m;
@@ -199,8 +210,8 @@ k_widen_bf16(const __nv_bfloat16* __restrict__ X, float* __restrict__ out, int64
 template <bool G_BF16>
 __global__ void __launch_bounds__(kThreads)
 k_ema_out(float* __restrict__ out, const float* __restrict__ M, const void* __restrict__ G, int64_t numel,
-          float beta1) {
-  const float omb = 1.0f - beta1;
+          float beta1, const float* __restrict__ gscale) {
+  const float omb = (1.0f - beta1) * (gscale ? *gscale : 1.0f);
   const int64_t stride = (int64_t)gridDim.x * blockDim.x;
   const int64_t nvec = numel >> 2;
   for (int64_t v = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; v < nvec; v += stride) {
@@ -213,6 +224,46 @@ k_ema_out(float* __restrict__ out, const float* __restrict__ M, const void* __re
   }
   for (int64_t i = (nvec << 2) + blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < numel; i += stride)
     out[i] = beta1 * M[i] + omb * load_grad1<G_BF16>(G, i);
+}
+
+// Global-norm clipping factor of one call (App. D.2): sum of squares over all layers' gradients in a
+// fixed order (each CTA a contiguous share of the concatenated gradients, tree inside the CTA, then one
+// thread over the CTAs), then factor = min(1, clip / norm).
+template <int NSEG>
+__global__ void __launch_bounds__(kThreads)
+k_clip_partial(ClipSegs<NSEG> segs, int nseg, double* __restrict__ part) {
+  __shared__ double sh[kThreads];
+  const long long total = segs.begin[nseg];
+  const long long chunk = (total + gridDim.x - 1) / gridDim.x;
+  const long long lo = (long long)blockIdx.x * chunk;
+  const long long hi = lo + chunk < total ? lo + chunk : total;
+  double acc = 0.0;
+  int sg = 0;
+  while (sg < nseg && segs.begin[sg + 1] <= lo) ++sg;
+  for (; sg < nseg && segs.begin[sg] < hi; ++sg) {
+    const long long a = (lo > segs.begin[sg] ? lo : segs.begin[sg]) - segs.begin[sg];
+    const long long b = (hi < segs.begin[sg + 1] ? hi : segs.begin[sg + 1]) - segs.begin[sg];
+    if (segs.bf16[sg]) {
+      const __nv_bfloat16* g = reinterpret_cast<const __nv_bfloat16*>(segs.ptr[sg]);
+      for (long long i = a + threadIdx.x; i < b; i += kThreads) { const float v = __bfloat162float(g[i]); acc = fma((double)v, (double)v, acc); }
+    } else {
+      const float* g = reinterpret_cast<const float*>(segs.ptr[sg]);
+      for (long long i = a + threadIdx.x; i < b; i += kThreads) { const float v = g[i]; acc = fma((double)v, (double)v, acc); }
+    }
+  }
+  sh[threadIdx.x] = acc;
+  __syncthreads();
+  for (int w = kThreads / 2; w > 0; w >>= 1) {
+    if (threadIdx.x < w) sh[threadIdx.x] += sh[threadIdx.x + w];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) part[blockIdx.x] = sh[0];
+}
+__global__ void k_clip_final(const double* __restrict__ part, int n, float clip, float* __restrict__ out) {
+  double s = 0.0;
+  for (int i = 0; i < n; ++i) s += part[i];
+  const double nrm = sqrt(s);
+  *out = (nrm > (double)clip) ? (float)((double)clip / nrm) : 1.0f;
 }
 
 // x (rounded to fp32) = p1 + p2 + p3 with three bf16 terms: all 24 significant bits survive.
@@ -275,23 +326,23 @@ cudaError_t set_identity(float* Q, int64_t k, cudaStream_t s) {
 }
 
 cudaError_t ema_momentum(float* M, const void* G, int g_is_bf16, int64_t numel, float beta1,
-                         float* Gf32, __nv_bfloat16* Mh, __nv_bfloat16* Ml, cudaStream_t s) {
+                         float* Gf32, __nv_bfloat16* Mh, __nv_bfloat16* Ml, const float* gscale, cudaStream_t s) {
   int grid = grid_for((numel + 3) / 4);
   if (g_is_bf16)
-    k_ema_momentum<true><<<grid, kThreads, 0, s>>>(M, G, numel, beta1, Gf32, Mh, Ml);
+    k_ema_momentum<true><<<grid, kThreads, 0, s>>>(M, G, numel, beta1, Gf32, Mh, Ml, gscale);
   else
-    k_ema_momentum<false><<<grid, kThreads, 0, s>>>(M, G, numel, beta1, Gf32, Mh, Ml);
+    k_ema_momentum<false><<<grid, kThreads, 0, s>>>(M, G, numel, beta1, Gf32, Mh, Ml, gscale);
   return cudaGetLastError();
 }
 
 cudaError_t plain_adam(float* W, float* M, float* V, const void* G, int g_is_bf16, int64_t numel,
-                       float lr, float beta1, float beta2, float eps, float wd, cudaStream_t s) {
+                       float lr, float beta1, float beta2, float eps, float wd, const float* gscale, cudaStream_t s) {
   int grid = grid_for((numel + 3) / 4);
   float decay = 1.0f - lr * wd;
   if (g_is_bf16)
-    k_plain_adam<true><<<grid, kThreads, 0, s>>>(W, M, V, G, numel, lr, beta1, beta2, eps, decay);
+    k_plain_adam<true><<<grid, kThreads, 0, s>>>(W, M, V, G, numel, lr, beta1, beta2, eps, decay, gscale);
   else
-    k_plain_adam<false><<<grid, kThreads, 0, s>>>(W, M, V, G, numel, lr, beta1, beta2, eps, decay);
+    k_plain_adam<false><<<grid, kThreads, 0, s>>>(W, M, V, G, numel, lr, beta1, beta2, eps, decay, gscale);
   return cudaGetLastError();
 }
 
@@ -313,10 +364,29 @@ cudaError_t widen_bf16(const __nv_bfloat16* X, float* out, int64_t numel, cudaSt
 }
 
 cudaError_t ema_out(float* out, const float* M, const void* G, int g_is_bf16, int64_t numel, float beta1,
-                    cudaStream_t s) {
+                    const float* gscale, cudaStream_t s) {
   const int grid = grid_for((numel + 3) / 4);
-  if (g_is_bf16) k_ema_out<true><<<grid, kThreads, 0, s>>>(out, M, G, numel, beta1);
-  else k_ema_out<false><<<grid, kThreads, 0, s>>>(out, M, G, numel, beta1);
+  if (g_is_bf16) k_ema_out<true><<<grid, kThreads, 0, s>>>(out, M, G, numel, beta1, gscale);
+  else k_ema_out<false><<<grid, kThreads, 0, s>>>(out, M, G, numel, beta1, gscale);
+  return cudaGetLastError();
+}
+
+cudaError_t clip_factor(const void* const* grads, const int64_t* numel, const int* is_bf16, int n, float clip,
+                        double* part, float* out, cudaStream_t s) {
+  constexpr int NSEG = 64, GRID = 296;
+  int launches = 0;
+  for (int first = 0; first < n; first += NSEG, ++launches) {
+    ClipSegs<NSEG> segs;
+    const int cnt = (n - first < NSEG) ? n - first : NSEG;
+    segs.begin[0] = 0;
+    for (int i = 0; i < cnt; ++i) {
+      segs.ptr[i] = grads[first + i];
+      segs.bf16[i] = is_bf16[first + i];
+      segs.begin[i + 1] = segs.begin[i] + numel[first + i];
+    }
+    k_clip_partial<NSEG><<<GRID, kThreads, 0, s>>>(segs, cnt, part + (size_t)launches * GRID);
+  }
+  k_clip_final<<<1, 1, 0, s>>>(part, launches * GRID, clip, out);
   return cudaGetLastError();
 }
 

@@ -72,6 +72,8 @@ struct alignas(128) DevProblem {
   // shared-operand form: mapA[0..nA) / mapB[0..nB) are the distinct operands, `combos` lists the
   // products to issue per k-block: bits 8.. = count, bits 2c, 2c+1 = (A index, B index) of product c
   int32_t symmetric, nA, nB, combos;
+  const float* clip;              // clipping factors by call (see TcProblem::clip_mode), or null
+  int32_t clip_slots, clip_mode;
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -398,10 +400,17 @@ k_tc_gemm(const DevProblem* __restrict__ probs, int n_probs, int first_tile, int
       const TileInfo ti = locate_tile(probs, n_probs, tile_i, calls, tau);
       if (!ti.active) continue;
       const DevProblem* p = ti.p;
-      const float alpha = p->dyn_scalars ? dyn_alpha : p->alpha;
+      float alpha = p->dyn_scalars ? dyn_alpha : p->alpha;
       const float beta = p->dyn_scalars ? dyn_beta : p->beta;
       const float eps = p->eps;
       const int epi = p->epilogue;
+      // clipping factor of the call whose gradient this accumulator was built from
+      float gclip = 1.0f;
+      if (p->clip) {
+        const int tl = tau < 0 ? p->tau_max : tau;
+        gclip = p->clip[(int)((calls - 1 - tl) % p->clip_slots)];
+        if (p->clip_mode == 2) alpha *= gclip * gclip;
+      }
       const int row_base = ti.m0 + quad * 32;
       const bool quad_ok = row_base < p->Md;      // uniform across the warp
       const bool reads_d = (epi == EPI_AXPBY_F32 && beta != 0.0f) || epi == EPI_ROTATED_ADAM ||
@@ -497,7 +506,7 @@ k_tc_gemm(const DevProblem* __restrict__ probs, int n_probs, int first_tile, int
 #pragma unroll
           for (int it = 0; it < 8; ++it)
             if (it < n_it) {
-              const float4 g = a[it];
+              const float4 g = make_float4(gclip * a[it].x, gclip * a[it].y, gclip * a[it].z, gclip * a[it].w);
               float4 m = mm[it], q = ss[it];
               m.x = b1 * m.x + ob1 * g.x; m.y = b1 * m.y + ob1 * g.y;
               m.z = b1 * m.z + ob1 * g.z; m.w = b1 * m.w + ob1 * g.w;
@@ -735,6 +744,10 @@ TcPlan* tc_plan_create(const TcProblem* problems, int n, int device, cudaStream_
     d.dyn_scalars = q.dyn_scalars;
     d.alpha = q.alpha; d.beta = q.beta; d.eps = q.eps; d.beta1 = q.beta1;
     d.symmetric = q.symmetric ? 1 : 0;
+    d.clip = q.clip_mode ? q.clip : nullptr; d.clip_slots = q.clip_slots; d.clip_mode = q.clip_mode;
+    if (d.clip && (q.clip_slots < 1 || (q.clip_mode == 1 && q.epilogue != EPI_ROTATED_ADAM) ||
+                   (q.clip_mode == 2 && q.epilogue != EPI_AXPBY_F32)))
+      return fail("tensor-core problem: clipping applies to the rotated-Adam and factor epilogues");
     if (q.symmetric && (q.Md != q.Nd || q.epilogue != EPI_AXPBY_F32))
       return fail("tensor-core problem: a symmetric product needs a square fp32 result");
     d.D = q.D; d.ldd = q.ldd; d.Dh = q.Dh; d.Dl = q.Dl; d.ldh = q.ldh; d.D2 = q.D2;

@@ -225,6 +225,8 @@ struct TcStep {
   std::vector<Chunk> chunks;
   std::vector<TcPlan*> factor_plan;   // per layer, BR_ACCUM_ON_REFRESH only
   std::vector<int> chunk_of, slot_of; // per layer: its chunk and its position in the chunk
+  const float* clip = nullptr;        // ring of clipping factors by call, or null
+  int clip_slots = 0;
   std::string err;
 };
 
@@ -250,7 +252,7 @@ void tc_step_destroy(TcStep* t) {
 }
 
 TcStep* tc_step_create(std::vector<Layer>& layers, const br_hparams& hp, char* scratch, size_t bytes,
-                       int device, cudaStream_t s, const char** err) {
+                       const float* clip, int clip_slots, int device, cudaStream_t s, const char** err) {
   static thread_local std::string last;
   if (err) *err = nullptr;
   auto chunk_ids = make_chunks(layers, hp);
@@ -260,6 +262,7 @@ TcStep* tc_step_create(std::vector<Layer>& layers, const br_hparams& hp, char* s
   };
   if (!tc_supported(device)) { last = "tensor-core path needs an sm_100 device and cuTensorMapEncodeTiled"; if (err) *err = last.c_str(); return nullptr; }
   TcStep* t = new TcStep();
+  t->clip = clip; t->clip_slots = clip_slots;
   t->factor_plan.assign(layers.size(), nullptr);
   t->chunk_of.assign(layers.size(), -1);
   t->slot_of.assign(layers.size(), -1);
@@ -303,6 +306,10 @@ TcStep* tc_step_create(std::vector<Layer>& layers, const br_hparams& hp, char* s
           !build(one.fwd2, &r.fwd2))
         return fail(t, perr ? perr : "plan creation failed");
     }
+    if (clip) {
+      for (TcProblem& q : P.factors) { q.clip = clip; q.clip_slots = clip_slots; q.clip_mode = 2; }
+      for (TcProblem& q : P.adam) { q.clip = clip; q.clip_slots = clip_slots; q.clip_mode = 1; }
+    }
     if (!build(P.factors, &c.factors) || !build(P.fwd1, &c.fwd1) || !build(P.adam, &c.adam) ||
         !build(P.back1, &c.back1) || !build(P.wwrite, &c.wwrite) || !build(R.back1, &c.rx.back1) ||
         !build(R.back2, &c.rx.back2) || !build(R.fwd1, &c.rx.fwd1) || !build(R.fwd2, &c.rx.fwd2))
@@ -314,6 +321,7 @@ TcStep* tc_step_create(std::vector<Layer>& layers, const br_hparams& hp, char* s
       if (!L.use_tc || L.d.src != BR_SRC_SECOND) continue;
       std::vector<TcProblem> f;
       factor_problems(L, beta_f, &f);
+      if (clip) for (TcProblem& q : f) { q.clip = clip; q.clip_slots = clip_slots; q.clip_mode = 2; }
       if (!f.empty() && !(t->factor_plan[i] = tc_plan_create(f.data(), (int)f.size(), device, s, &perr)))
         return fail(t, perr ? perr : "plan creation failed");
     }
@@ -417,7 +425,9 @@ int tc_step_run(TcStep* t, std::vector<Layer>& layers, const std::vector<const v
       for (int i : due) {
         Layer& L = layers[i];
         if (L.d.src != BR_SRC_FIRST) continue;
-        cudaError_t e = ema_out(L.Morig, L.M, G[i], L.d.grad_dtype == BR_BF16, L.d.m * L.d.n, hp.beta1, s);
+        const int tl = tau < 0 ? L.d.tau_max : tau;
+        const float* gs = t->clip ? t->clip + (int)((calls - 1 - tl) % t->clip_slots) : nullptr;
+        cudaError_t e = ema_out(L.Morig, L.M, G[i], L.d.grad_dtype == BR_BF16, L.d.m * L.d.n, hp.beta1, gs, s);
         if (e != cudaSuccess) return lz.fail("ema_out", e);
         stats->launches += 1;
       }

@@ -42,8 +42,9 @@ struct TcStepCallbacks {
 // Transient scratch (bytes) the tensor-core step needs for these layers.
 size_t tc_step_scratch_bytes(const std::vector<Layer>& layers, const br_hparams& hp);
 // Returns nullptr with *err == nullptr when no layer uses the tensor-core path.
+// clip / clip_slots: the handle's ring of clipping factors (null when clipping is off)
 TcStep* tc_step_create(std::vector<Layer>& layers, const br_hparams& hp, char* scratch, size_t bytes,
-                       int device, cudaStream_t s, const char** err);
+                       const float* clip, int clip_slots, int device, cudaStream_t s, const char** err);
 // Enqueue the updates of every tensor-core layer whose G[i] is non-null.  0 on success,
 // a negative br_status otherwise (message in *err).
 int tc_step_run(TcStep* t, std::vector<Layer>& layers, const std::vector<const void*>& G, long long calls,

@@ -167,3 +167,12 @@ def test_bilateral_first_moment_rectangular_completion():
     layers = [LayerSpec("wide", 128, 200, GEOM_BI, SRC_FIRST, 1), LayerSpec("tall", 264, 136, GEOM_BI, SRC_FIRST, 1)]
     w = Workload("bi1st", layers, "bf16", "iid_normal", 0.02, tau=1, freq=4, calls=14, seed=13)
     _run(w, 14, tau=1)
+
+
+def test_global_norm_clipping_tensor_core():
+    """Clipping on the tensor-core path: the factor enters the factor EMAs squared and the rotated
+    gradient linearly, inside the epilogues; two layers with different delays share the calls' factors."""
+    layers = [LayerSpec("a", 136, 200, GEOM_BI, SRC_SECOND, 3), LayerSpec("b", 264, 72, GEOM_UNI, SRC_SECOND, 1),
+              LayerSpec("c", 128, 128, GEOM_BI, SRC_FIRST, 2)]
+    w = Workload("clip", layers, "bf16", "iid_normal", 0.02, tau=3, freq=4, calls=14, seed=16)
+    _run(w, 14, tau=-1, clip_norm=1.0)

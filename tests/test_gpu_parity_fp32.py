@@ -85,6 +85,15 @@ def test_weight_decay_and_on_refresh_accumulation():
     _run(w, 8, tau=0, accum="on_refresh")
 
 
+def test_global_norm_clipping_mixed_layers_and_delays():
+    """Clipping threshold well below the joint gradient norm, rotated and plain layers, per-layer
+    delays: each update must use the factor of the call its gradient was submitted with."""
+    layers = [LayerSpec("a", 40, 56, GEOM_BI, SRC_SECOND, 2), LayerSpec("b", 24, 64, GEOM_UNI, SRC_FIRST, 1),
+              LayerSpec("c", 20, 20, GEOM_NONE, SRC_SECOND, 0)]
+    w = Workload("clip", layers, "f32", "iid_normal", 0.05, tau=2, freq=3, calls=12, gemm_prec="f32", seed=15)
+    _run(w, 12, tau=-1, clip_norm=0.5)
+
+
 def test_power_iters_2():
     _run(_small(GEOM_BI, SRC_SECOND, 40, 56, tau=0, freq=3), 7, tau=0, power_iters=2)
 

@@ -28,7 +28,7 @@ def test_exports_every_declared_symbol(br):
 
 def _hp(br, **kw):
     d = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0, beta_factor=-1.0, freq=10,
-             power_iters=1, accum=0, gemm_prec=br.BR_GEMM_FP32, flags=0, reserved=0, scratch_limit_bytes=0)
+             power_iters=1, accum=0, gemm_prec=br.BR_GEMM_FP32, flags=0, clip_norm=0.0, scratch_limit_bytes=0)
     d.update(kw)
     return br.BrHparams(**d)
 
@@ -107,3 +107,12 @@ def test_stage_aware_helpers_match_the_oracle(br):
         assert abs(br.br_effective_delay(c, t) - O.effective_delay(c, t)) < 1e-12
     with pytest.raises(br.BrError):
         br.br_effective_delay([0.0, 0.0], [1, 2])
+
+
+def test_lr_schedule_helper_matches_the_oracle(br):
+    from oracle import br_oracle as O
+    for total, frac in ((1000, 0.012), (37, 0.1), (10, 0.0), (5, 1.0)):
+        for t in range(total):
+            assert abs(br.br_lr_warmup_cosine(t, total, frac, 3e-4, 1e-6) - O.lr_warmup_cosine(t, total, frac, 3e-4, 1e-6)) < 1e-15
+    with pytest.raises(br.BrError):
+        br.br_lr_warmup_cosine(10, 10, 0.1, 1e-3, 0.0)

@@ -448,3 +448,45 @@ def test_effective_delay_closed_forms():
     assert O.effective_delay([2.0, 0.0], [5, 100]) == pytest.approx(5.0)
     assert O.effective_delay([1, 2, 3], [3, 2, 1]) == pytest.approx(O.effective_delay([10, 20, 30], [3, 2, 1]))
     assert O.effective_delay([1, 2, 3], [3, 2, 1]) == pytest.approx(np.sqrt((9 + 16 + 9) / 14))
+
+
+def test_global_norm_clipping_closed_forms():
+    """App. D.2 clipping: (a) a threshold above the joint norm changes nothing, bit for bit; (b) below
+    it, the momentum after the first update has joint norm (1 - beta1) * clip exactly as a closed form
+    (M0 = 0, so M1 = (1 - beta1) * s * g with s = clip / ||g||); (c) a clipped trajectory is invariant to
+    rescaling every gradient by a > 1 (the clipped gradient is clip * g / ||g||); (d) the factor travels
+    with its call through the delay: with tau = 2 the update at call 3 uses the factor of call 1."""
+    shapes = [(6, 4), (3, 5)]
+    def run(clip, scale=1.0, tau=0, calls=3, tmax=0):
+        layers = [O.OracleLayer(np.zeros(s), O.GEOM_NONE, O.SRC_SECOND, tmax) for s in shapes]
+        orc = O.Oracle(layers, O.Hyper(lr=1e-2, clip_norm=clip, freq=10 ** 6))
+        r = rng(40)
+        for c in range(calls):
+            orc.step([scale * (c + 1) * r.standard_normal(s) for s in shapes], tau)
+        return orc
+    a, b = run(0.0), run(1e6)
+    for x, y in zip(a.layers, b.layers):
+        assert np.array_equal(x.W, y.W) and np.array_equal(x.M, y.M)
+    one = run(0.5, calls=1)
+    joint = np.sqrt(sum(np.sum(l.M ** 2) for l in one.layers))
+    assert joint == pytest.approx((1 - 0.9) * 0.5, rel=1e-12)
+    c1, c2 = run(0.5), run(0.5, scale=7.0)
+    for x, y in zip(c1.layers, c2.layers):
+        assert np.allclose(x.W, y.W, rtol=1e-12, atol=0)
+    d = run(0.5, tau=2, calls=3, tmax=2)
+    assert d.layers[0].t == 1 and set(d.clip_of_call) == {1, 2, 3}
+    g1 = [1 * x for x in [rng(40).standard_normal(shapes[0])]][0]     # the first draw of call 1
+    n1 = np.sqrt(sum(np.sum(x ** 2) for x in (lambda r: [r.standard_normal(s) for s in shapes])(rng(40))))
+    assert d.clip_of_call[1] == pytest.approx(0.5 / n1, rel=1e-12)
+    assert np.allclose(d.layers[0].M, (1 - 0.9) * d.clip_of_call[1] * g1, rtol=1e-12, atol=0)
+
+
+def test_lr_warmup_cosine_schedule_values():
+    """App. D.2 schedule, 1000 steps with 1.2 % warm-up (W = 12): linear ramp reaching base_lr at step
+    11, base_lr again at step 12 (cosine of 0), the mid-point of the decay halfway, monotone decay."""
+    f = lambda t: O.lr_warmup_cosine(t, 1000, 0.012, 1e-3, 1e-5)
+    assert f(0) == pytest.approx(1e-3 / 12) and f(5) == pytest.approx(6e-3 / 12) and f(11) == pytest.approx(1e-3)
+    assert f(12) == pytest.approx(1e-3)
+    assert f(12 + 494) == pytest.approx(1e-5 + (1e-3 - 1e-5) * 0.5)
+    vals = [f(t) for t in range(12, 1000)]
+    assert all(a >= b for a, b in zip(vals, vals[1:])) and vals[-1] > 1e-5

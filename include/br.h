@@ -116,9 +116,12 @@ typedef struct {
   int64_t refresh_count;  /* refreshes done for this layer, scheduled and forced             */
   int64_t next_refresh_t; /* next t with t mod freq == 0                                     */
   /* Not part of the method's integer state: what the library remembers about the conditioning of
-   * the last refresh of this layer's bases (bit 0: left, bit 1: right; set = no column of F Q shrank
-   * below 1e-3 of its length under orthonormalisation).  The next refresh of a tensor-core layer
-   * runs its block projections on the tensor cores only for a basis whose bit is set.  Saved and
+   * the last refresh of this layer's bases.  Bit 0 (left) and bit 1 (right): no column of F Q shrank
+   * below 1e-3 of its length under orthonormalisation; the next refresh of a tensor-core layer runs
+   * its block projections on the tensor cores only for a basis whose bit is set.  Bit 2 (left) and
+   * bit 3 (right): the factorisation had to clamp a pivot (a numerically rank-deficient product; the
+   * status word then holds BR_WARN_RANK_DEFICIENT and the affected columns of that refresh are not
+   * orthonormal); the next refresh of that basis completes it from the current one.  Saved and
    * restored with the other counters so that a resumed run takes the same decisions. */
   int64_t basis_flags;
 } br_counters;

@@ -279,13 +279,16 @@ br_status refresh_side(br_handle* h, Layer& L, bool left_side, br_handle::Lane& 
     const int64_t other = left_side ? n : m;
     const bool short_of_rank = (L.d.src == BR_SRC_FIRST) ? (k > other)
                                                          : (L.n_accum < (k + other - 1) / other);
-    if (short_of_rank) {
+    // (also when the previous refresh of this basis met a pivot it had to clamp: a factor that is
+    // rank-deficient numerically, e.g. gradients confined to a subspace)
+    const int ci0 = 2 * (int)(&L - h->layers.data()) + (left_side ? 0 : 1);
+    if (short_of_rank || (h->cond_known[ci0] & 2)) {
       BR_CUDA(h, qr_complete_columns(ln.rA, Q, k, ln.rWork, h->d_status, s));
       count(h, 3);
     }
     const int ci = 2 * (int)(&L - h->layers.data()) + (left_side ? 0 : 1);
     QrTc* tcq = nullptr;
-    if (L.use_tc && h->cond_known[ci])
+    if (L.use_tc && (h->cond_known[ci] & 1) && !(h->cond_known[ci] & 2))
       for (QrTc* t : ln.tcq) if (qr_tc_order(t) == k) tcq = t;
     BR_CUDA(h, qr_pos_inplace(ln.rA, k, ln.rWork, h->d_status, s, &h->stats.launches, &h->stats.gemm_flops, tcq,
                               h->d_cond + ci));
@@ -785,7 +788,8 @@ br_status br_get_counters(br_handle* h, int layer, br_counters* out) {
     for (size_t i = 0; i < h->cond_known.size(); ++i) h->cond_known[i] = h->h_cond[i];
     h->cond_pending = false;
   }
-  out->basis_flags = (h->cond_known[2 * layer] ? 1 : 0) | (h->cond_known[2 * layer + 1] ? 2 : 0);
+  out->basis_flags = (h->cond_known[2 * layer] & 1) | ((h->cond_known[2 * layer + 1] & 1) << 1) |
+                     ((h->cond_known[2 * layer] & 2) << 1) | ((h->cond_known[2 * layer + 1] & 2) << 2);
   return BR_OK;
 }
 
@@ -806,7 +810,8 @@ br_status br_set_counters(br_handle* h, int layer, const br_counters* in) {
       for (size_t i = 0; i < h->cond_known.size(); ++i) h->cond_known[i] = h->h_cond[i];
       h->cond_pending = false;
     }
-    const int v[2] = {(int)(in->basis_flags & 1), (int)((in->basis_flags >> 1) & 1)};
+    const int v[2] = {(int)((in->basis_flags & 1) | ((in->basis_flags >> 1) & 2)),
+                      (int)(((in->basis_flags >> 1) & 1) | ((in->basis_flags >> 2) & 2))};
     h->cond_known[2 * layer] = v[0];
     h->cond_known[2 * layer + 1] = v[1];
     BR_CUDA(h, cudaMemcpy(h->d_cond + 2 * layer, v, sizeof v, cudaMemcpyHostToDevice));

@@ -114,7 +114,7 @@ k_chol_inverse(const double* __restrict__ S, int bw, double* __restrict__ Rinv, 
   }
   __syncthreads();
   double defect = 0.0;       // accumulated by thread 0 (every thread sees every pivot)
-  bool ill = false, tc_bad = false;
+  bool ill = false, tc_bad = false, any_clamped = false;
 
   for (int c = 0; c < bw; ++c) {
     const int buf = c & 1;
@@ -125,7 +125,7 @@ k_chol_inverse(const double* __restrict__ S, int bw, double* __restrict__ Rinv, 
     const bool clamped = !(piv > floor_);
     if (clamped) piv = floor_;
     if (t == 0) {
-      if (clamped) atomicMax(status, (int)BR_WARN_RANK_DEFICIENT);
+      if (clamped) { atomicMax(status, (int)BR_WARN_RANK_DEFICIENT); any_clamped = true; }
       defect += fmax(0.0, 1.0 - piv * diag0_inv[c]);
       if (orig < nrm_floor[c]) ill = true;
       if (orig < tc_floor[c]) tc_bad = true;
@@ -181,12 +181,14 @@ k_chol_inverse(const double* __restrict__ S, int bw, double* __restrict__ Rinv, 
     if (skip_next) *skip_next = (defect <= kDefectLimit) ? 1 : 0;
     if (ill && ill_clear) *ill_clear = 0;
     if (tc_bad && tc_ok_clear) *tc_ok_clear = 0;
+    if (any_clamped && tc_ok_clear) tc_ok_clear[1] = 1;      // numerically rank-deficient: noted for the next refresh
   }
 }
 
 // flags at the start of a QR: second sweep cancelled, basis well enough conditioned for the
 // tensor-core projections next time; and the copy of the latter to its long-lived home at the end
-__global__ void k_store_flag(int* dst, const int* src) { *dst = *src; }
+// bit 0: tensor-core projections allowed next time; bit 1: a pivot was clamped (complete the basis next time)
+__global__ void k_store_flag(int* dst, const int* src) { *dst = (src[0] ? 1 : 0) | (src[1] ? 2 : 0); }
 
 // part[z][j] = sum over the row chunk z of A[i][j]^2 (rows in order)
 constexpr int kNormChunks = 32;
@@ -210,7 +212,8 @@ __global__ void __launch_bounds__(256)
 k_column_norms_sum(const double* __restrict__ part, int64_t k, int nchunks, double* __restrict__ norm0,
                    int* __restrict__ flag) {
   const int64_t j = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
-  if (j == 0) { flag[0] = 1; flag[1] = 1; }   // sweep-2 cancelled, tensor-core projections allowed next time
+  // sweep-2 cancelled, tensor-core projections allowed next time, no pivot clamped so far
+  if (j == 0) { flag[0] = 1; flag[1] = 1; flag[2] = 0; }
   if (j >= k) return;
   double s = 0.0;
   for (int z = 0; z < nchunks; ++z) s += part[(int64_t)z * k + j];

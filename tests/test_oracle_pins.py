@@ -490,3 +490,26 @@ def test_lr_warmup_cosine_schedule_values():
     assert f(12 + 494) == pytest.approx(1e-5 + (1e-3 - 1e-5) * 0.5)
     vals = [f(t) for t in range(12, 1000)]
     assert all(a >= b for a, b in zip(vals, vals[1:])) and vals[-1] > 1e-5
+
+
+def _closed_loop_oracle(geom, aligned, tau, steps=300):
+    from workloads.closed_loop import kronecker_quadratic, loss
+    P, Q, W0 = kronecker_quadratic(aligned=aligned)
+    lay = O.OracleLayer(W0.copy(), geom, O.SRC_SECOND, tau)
+    orc = O.Oracle([lay], O.Hyper(lr=0.02, beta1=0.0, beta2=0.9, eps=1e-12, freq=5))
+    for _ in range(steps):
+        orc.step([P @ lay.W @ Q], tau)          # the gradient at the CURRENT weights, applied tau calls later
+    return loss(P, Q, lay.W)
+
+
+def test_closed_loop_quadratic_rotation_removes_the_delay_penalty():
+    """The paper's toy claim (Sec. 2.2, Fig. 2; Sec. 3.1), on a Kronecker quadratic with genuinely
+    stale gradients (tau = 2): Adam on the misaligned problem is much worse than on the aligned one,
+    and the basis-rotated step on the misaligned problem is as good as Adam on the aligned one."""
+    aligned = _closed_loop_oracle(O.GEOM_NONE, True, 2)
+    misaligned = _closed_loop_oracle(O.GEOM_NONE, False, 2)
+    rotated = _closed_loop_oracle(O.GEOM_BI, False, 2)
+    assert misaligned > 5.0 * aligned
+    assert rotated < 2.0 * aligned
+    # and delay itself hurts plain Adam on the misaligned problem
+    assert _closed_loop_oracle(O.GEOM_NONE, False, 0) < 0.5 * misaligned

@@ -243,6 +243,53 @@ const void* ring_slot_ptr(const Layer& L, int64_t slot) {
   return L.ring + (size_t)slot * L.slot_stride;
 }
 
+// ---- the power product F Q of a tracking basis, mostly on the tensor cores -------------------------
+// F Q in fp32-level arithmetic is useless as it stands: the small eigen-directions of F come out of
+// a cancellation against eigenvalues up to 1e5 times larger.  But once the basis tracks the factor
+// its leading columns U_s (one panel of r = 128) span the dominant directions, and
+//   F = F_rest + P F + F P - P F P,   P = U_s U_s^T,   F_rest = (I - P) F (I - P)
+// holds for ANY matrix P (it is plain algebra), with F_rest free of the large eigenvalues.  So
+//   F Q = F_rest Q + B (U_s^T Q) + U_s (B^T Q - Lam U_s^T Q),   B = F U_s,  Lam = U_s^T B  (F symmetric)
+// where the rank-r terms (14 k^2 r flop) and F_rest itself are computed on the fp64 matrix unit
+// and only F_rest Q (2 k^3 flop) runs on the tensor cores, on three-term bf16 splits: its error is
+// ~2e-7 ||F_rest|| per column, a relative 2e-7 of the small columns instead of 2e-7 * 1e5.
+// On entry ln.rF and ln.rQ hold F and Q widened to fp64; on exit ln.rA holds F Q (rF is overwritten).
+br_status deflated_power(br_handle* h, br_handle::Lane& ln, QrTc* tcq, int64_t k, cudaStream_t s) {
+  const int64_t r = 128;
+  double* w = ln.rWork;                               // the QR work area is free until the QR starts
+  double* B = w;               w += k * r;            // k x r
+  double* T1 = w;              w += k * r;            // k x r
+  double* C1 = w;              w += r * k;            // r x k
+  double* C2 = w;              w += r * k;            // r x k
+  double* Lam = w;             w += r * r;            // r x r
+  double* part = w;                                   // split-K partial sums (at most 54 * r * r, 4 * r * k doubles)
+  const int sp_small = (int)std::min<int64_t>(54, std::max<int64_t>(1, k / 128));
+  double* F = ln.rF;
+  double* Q = ln.rQ;
+  const double* Us = Q;                               // first r columns of Q, leading dimension k
+  // B = F U_s ; Lam = U_s^T B ; C1 = U_s^T Q ; C2 = B^T Q
+  BR_CUDA(h, dgemm(0, 0, k, r, k, 1.0, F, k, Us, k, 0.0, B, r, s));
+  BR_CUDA(h, dgemm_ex(1, 0, r, r, k, 1.0, Us, k, B, r, 0.0, Lam, r, sp_small, part, nullptr, s));
+  BR_CUDA(h, dgemm_ex(1, 0, r, k, k, 1.0, Us, k, Q, k, 0.0, C1, k, 4, part, nullptr, s));
+  BR_CUDA(h, dgemm_ex(1, 0, r, k, k, 1.0, B, r, Q, k, 0.0, C2, k, 4, part, nullptr, s));
+  // T1 = B - U_s Lam ; F_rest = F - U_s B^T - T1 U_s^T
+  BR_CUDA(h, cudaMemcpyAsync(T1, B, sizeof(double) * k * r, cudaMemcpyDeviceToDevice, s));
+  BR_CUDA(h, dgemm(0, 0, k, r, r, -1.0, Us, k, Lam, r, 1.0, T1, r, s));
+  BR_CUDA(h, dgemm(0, 1, k, k, r, -1.0, Us, k, B, r, 1.0, F, k, s));
+  BR_CUDA(h, dgemm(0, 1, k, k, r, -1.0, T1, r, Us, k, 1.0, F, k, s));
+  // F_rest Q on the tensor cores
+  const float* Af = nullptr;
+  BR_CUDA(h, qr_tc_power(tcq, F, Q, h->d_status, s, &Af));
+  // C2 <- C2 - Lam C1 ; A = F_rest Q + B C1 + U_s C2
+  BR_CUDA(h, dgemm(0, 0, r, k, r, -1.0, Lam, r, C1, k, 1.0, C2, k, s));
+  BR_CUDA(h, f32_to_f64(Af, ln.rA, k * k, s));
+  BR_CUDA(h, dgemm(0, 0, k, k, r, 1.0, B, r, C1, k, 1.0, ln.rA, k, s));
+  BR_CUDA(h, dgemm(0, 0, k, k, r, 1.0, Us, k, C2, k, 1.0, ln.rA, k, s));
+  count(h, 22);
+  h->stats.gemm_flops += 14.0 * k * k * r;
+  return BR_OK;
+}
+
 // ---- refresh of one side: Q <- qr(F Q).Q in fp64, F = L | R (S=2nd) or M M^T | M^T M (S=1st) ----
 br_status refresh_side(br_handle* h, Layer& L, bool left_side, br_handle::Lane& ln) {
   cudaStream_t s = ln.stream;
@@ -252,14 +299,30 @@ br_status refresh_side(br_handle* h, Layer& L, bool left_side, br_handle::Lane& 
   // S = 1st reads the momentum in the original space: the state buffer itself on the fp32 path, the
   // copy the caller prepared on the tensor-core path (whose state is the rotated momentum)
   const float* Mo = L.Morig ? L.Morig : L.M;
+  const int ci = 2 * (int)(&L - h->layers.data()) + (left_side ? 0 : 1);
+  // the tensor-core forms (power product, block projections) only for a basis whose last refresh
+  // found it tracking the factor, and only where the product is known to have full rank
+  const int64_t other = left_side ? n : m;
+  const bool short_of_rank = (L.d.src == BR_SRC_FIRST) ? (k > other)
+                                                       : (L.n_accum < (k + other - 1) / other);
+  const bool complete = short_of_rank || (h->cond_known[ci] & 2);
+  QrTc* tcq = nullptr;
+  if (L.use_tc && (h->cond_known[ci] & 1) && !complete)
+    for (QrTc* t : ln.tcq) if (qr_tc_order(t) == k) tcq = t;
   for (int it = 0; it < h->hp.power_iters; ++it) {
     if (L.d.src == BR_SRC_SECOND) {
       const float* F = left_side ? L.L : L.R;
-      // widen once, then a pure fp64 product (the products are exact either way)
+      // widen once, then fp64 products (the products of fp32 values are exact either way)
       BR_CUDA(h, f32_to_f64(F, ln.rF, k * k, s));
       BR_CUDA(h, f32_to_f64(Q, ln.rQ, k * k, s));
-      BR_CUDA(h, dgemm(0, 0, k, k, k, 1.0, ln.rF, k, ln.rQ, k, 0.0, ln.rA, k, s));
-      count(h, 3); h->stats.gemm_flops += 2.0 * k * k * k;
+      count(h, 2);
+      if (tcq) {
+        br_status st = deflated_power(h, ln, tcq, k, s);
+        if (st != BR_OK) return st;
+      } else {
+        BR_CUDA(h, dgemm(0, 0, k, k, k, 1.0, ln.rF, k, ln.rQ, k, 0.0, ln.rA, k, s));
+        count(h); h->stats.gemm_flops += 2.0 * k * k * k;
+      }
     } else if (left_side) {
       // (M M^T) U = M (M^T U)
       BR_CUDA(h, sdgemm(1, 0, n, m, m, 1.0, Mo, n, Q, m, 0.0, ln.rZ, m, s));
@@ -273,23 +336,15 @@ br_status refresh_side(br_handle* h, Layer& L, bool left_side, br_handle::Lane& 
     }
     // A rank-deficient product has no unique Q factor.  Which products are is known on the host: with
     // S = 1st, M M^T (M^T M) has rank <= min(m, n), short of the larger side; with S = 2nd, a factor that
-    // has accumulated a gradients has rank <= a * (the other dimension).  The directions outside the
-    // range of F Q are then completed from the current basis: what is orthonormalised is F Q with
-    // 1e-6 ||(F Q)_j|| Q_j added to every column j (full rank whenever Q is).
-    const int64_t other = left_side ? n : m;
-    const bool short_of_rank = (L.d.src == BR_SRC_FIRST) ? (k > other)
-                                                         : (L.n_accum < (k + other - 1) / other);
-    // (also when the previous refresh of this basis met a pivot it had to clamp: a factor that is
-    // rank-deficient numerically, e.g. gradients confined to a subspace)
-    const int ci0 = 2 * (int)(&L - h->layers.data()) + (left_side ? 0 : 1);
-    if (short_of_rank || (h->cond_known[ci0] & 2)) {
+    // has accumulated a gradients has rank <= a * (the other dimension); and a basis whose previous
+    // refresh had to clamp a pivot sits on a factor that is rank-deficient numerically (gradients
+    // confined to a subspace).  The directions outside the range of F Q are then completed from the
+    // current basis: what is orthonormalised is F Q with 1e-6 ||(F Q)_j|| Q_j added to every column j
+    // (full rank whenever Q is).
+    if (complete) {
       BR_CUDA(h, qr_complete_columns(ln.rA, Q, k, ln.rWork, h->d_status, s));
       count(h, 3);
     }
-    const int ci = 2 * (int)(&L - h->layers.data()) + (left_side ? 0 : 1);
-    QrTc* tcq = nullptr;
-    if (L.use_tc && (h->cond_known[ci] & 1) && !(h->cond_known[ci] & 2))
-      for (QrTc* t : ln.tcq) if (qr_tc_order(t) == k) tcq = t;
     BR_CUDA(h, qr_pos_inplace(ln.rA, k, ln.rWork, h->d_status, s, &h->stats.launches, &h->stats.gemm_flops, tcq,
                               h->d_cond + ci));
     BR_CUDA(h, f64_to_f32(ln.rA, Q, k * k, s));
@@ -911,6 +966,18 @@ br_status br_set_state(br_handle* h, int layer, int which, const void* host_src,
     BR_CUDA(h, cudaMemcpy(p, host_src, bytes, cudaMemcpyHostToDevice));
   }
   if (which == BR_BUF_L || which == BR_BUF_R) L.n_accum = (int64_t)1 << 40;   // a factor given by the caller: taken as full rank
+  // a factor or a basis given by the caller: nothing is known about how well the basis tracks the factor
+  if (which == BR_BUF_L || which == BR_BUF_U || which == BR_BUF_R || which == BR_BUF_V) {
+    if (h->cond_pending) {
+      BR_CUDA(h, cudaEventSynchronize(h->ev_cond));
+      for (size_t i = 0; i < h->cond_known.size(); ++i) h->cond_known[i] = h->h_cond[i];
+      h->cond_pending = false;
+    }
+    const int ci = 2 * layer + ((which == BR_BUF_R || which == BR_BUF_V) ? 1 : 0);
+    const int zero = 0;
+    h->cond_known[ci] = 0;
+    BR_CUDA(h, cudaMemcpy(h->d_cond + ci, &zero, sizeof(int), cudaMemcpyHostToDevice));
+  }
   if (L.use_tc && which == BR_BUF_U) { BR_CUDA(h, split_bf16(L.U, L.Uh, L.Ul, L.d.m * L.d.m, h->stream)); count(h); }
   if (L.use_tc && which == BR_BUF_V) { BR_CUDA(h, split_bf16(L.V, L.Vh, L.Vl, L.d.n * L.d.n, h->stream)); count(h); }
   BR_CUDA(h, cudaStreamSynchronize(h->stream));

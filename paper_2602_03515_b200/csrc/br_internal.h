@@ -132,6 +132,8 @@ int64_t qr_tc_order(const QrTc* t);
 // current basis; a zero column becomes Q[:, j]), and BR_WARN_RANK_DEFICIENT is raised in *status.
 // work: the QR work area of this order (used for the column norms).
 cudaError_t qr_complete_columns(double* A, const float* Q, int64_t k, double* work, int* status, cudaStream_t s);
+// *out (fp32, k x k, owned by t) = Frest U on the tensor cores (three-term bf16 splits, six products)
+cudaError_t qr_tc_power(QrTc* t, const double* Frest, const double* U, int* status, cudaStream_t s, const float** out);
 cudaError_t qr_tc_project(QrTc* t, int node, double* A, int64_t k, int64_t jp, int64_t wp, int64_t jt,
                           int64_t wt, int* status, cudaStream_t s);
 // tc: null, or the plans for this order: the first sweep then projects on the tensor cores (ask for it

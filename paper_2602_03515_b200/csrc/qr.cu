@@ -246,6 +246,7 @@ struct QrTc {
   TcPlan *lead = nullptr, *tail = nullptr;
   __nv_bfloat16 *Q[3] = {}, *A[3] = {}, *C[3] = {};
   float *Cf = nullptr, *Df = nullptr;
+  int power_index = -1;       // problem index (in both plans) of the deflated power product
 };
 
 namespace {
@@ -259,7 +260,8 @@ bool qr_tc_eligible(int64_t k) { return k >= 4096 && (k % 8) == 0; }
 size_t qr_tc_scratch_bytes(int64_t k) {
   if (!qr_tc_eligible(k)) return 0;
   const size_t h = (size_t)tc_hmax(k), kk = (size_t)k;
-  return 6 * al256(kk * h * 2) + al256(h * h * 4) + 3 * al256(h * h * 2) + al256(kk * h * 4);
+  // operand planes and the fp32 result hold a whole k x k matrix (the deflated power product)
+  return 6 * al256(kk * kk * 2) + al256(h * h * 4) + 3 * al256(h * h * 2) + al256(kk * kk * 4);
 }
 
 void qr_tc_destroy(QrTc* t) {
@@ -278,11 +280,11 @@ QrTc* qr_tc_create(int64_t k, char* scratch, int device, cudaStream_t s, const c
   const size_t h = (size_t)tc_hmax(k), kk = (size_t)k;
   size_t off = 0;
   auto take = [&](size_t bytes) { char* p = scratch + off; off += al256(bytes); return p; };
-  for (int i = 0; i < 3; ++i) t->Q[i] = reinterpret_cast<__nv_bfloat16*>(take(kk * h * 2));
-  for (int i = 0; i < 3; ++i) t->A[i] = reinterpret_cast<__nv_bfloat16*>(take(kk * h * 2));
+  for (int i = 0; i < 3; ++i) t->Q[i] = reinterpret_cast<__nv_bfloat16*>(take(kk * kk * 2));
+  for (int i = 0; i < 3; ++i) t->A[i] = reinterpret_cast<__nv_bfloat16*>(take(kk * kk * 2));
   t->Cf = reinterpret_cast<float*>(take(h * h * 4));
   for (int i = 0; i < 3; ++i) t->C[i] = reinterpret_cast<__nv_bfloat16*>(take(h * h * 2));
-  t->Df = reinterpret_cast<float*>(take(kk * h * 4));
+  t->Df = reinterpret_cast<float*>(take(kk * kk * 4));
   enumerate_nodes(0, k, 128, &t->nodes);
   std::vector<TcProblem> lead, tail;
   auto opnd = [](const void* p, int64_t ld, int mn) { TcOperand o; o.ptr = p; o.ld = ld; o.mn_major = mn; return o; };
@@ -308,6 +310,21 @@ QrTc* qr_tc_create(int64_t k, char* scratch, int device, cudaStream_t s, const c
     d.beta = 0.f; d2.beta = 1.f;
     lead.push_back(c); lead.push_back(d);
     tail.push_back(c2); tail.push_back(d2);
+  }
+  {
+    // the power product of the deflated factor: D = F_rest U, F_rest (k x k) K-major, U MN-major
+    const int ia[6] = {0, 1, 0, 2, 0, 1}, ib[6] = {0, 0, 1, 0, 2, 1};
+    TcProblem p1; p1.Md = k; p1.Nd = k; p1.K = k; p1.n_pairs = 3;
+    p1.epilogue = EPI_AXPBY_F32; p1.alpha = 1.f; p1.D = t->Df; p1.ldd = k;
+    TcProblem p2 = p1;
+    for (int p = 0; p < 3; ++p) {
+      p1.A[p] = opnd(t->Q[ia[p]], k, 0); p1.B[p] = opnd(t->A[ib[p]], k, 1);
+      p2.A[p] = opnd(t->Q[ia[3 + p]], k, 0); p2.B[p] = opnd(t->A[ib[3 + p]], k, 1);
+    }
+    p1.beta = 0.f; p2.beta = 1.f;
+    t->power_index = (int)lead.size();
+    lead.push_back(p1);
+    tail.push_back(p2);
   }
   const char* perr = nullptr;
   if (!lead.empty()) {
@@ -342,6 +359,19 @@ cudaError_t qr_tc_project(QrTc* t, int node, double* A, int64_t k, int64_t jp, i
     if ((e = tc_plan_launch_range(t->tail, 2 * node + 1, 1, 1, 0, 1.f, 0.f, status, s)) != cudaSuccess) return e;
     if ((e = sub_f32_from_f64(A + jt, k, k, wt, t->Df, s)) != cudaSuccess) return e;
   }
+  return cudaSuccess;
+}
+
+// D (fp32, k x k, returned in *out) = Frest U with both operands split into three bf16 terms and the
+// six leading products accumulated in fp32.  Frest and U are fp64, row-major with leading dimension k.
+cudaError_t qr_tc_power(QrTc* t, const double* Frest, const double* U, int* status, cudaStream_t s, const float** out) {
+  const int64_t k = t->k;
+  cudaError_t e;
+  if ((e = split3_f64(Frest, k, k, k, t->Q[0], t->Q[1], t->Q[2], s)) != cudaSuccess) return e;
+  if ((e = split3_f64(U, k, k, k, t->A[0], t->A[1], t->A[2], s)) != cudaSuccess) return e;
+  if ((e = tc_plan_launch_range(t->lead, t->power_index, 1, 1, 0, 1.f, 0.f, status, s)) != cudaSuccess) return e;
+  if ((e = tc_plan_launch_range(t->tail, t->power_index, 1, 1, 0, 1.f, 0.f, status, s)) != cudaSuccess) return e;
+  *out = t->Df;
   return cudaSuccess;
 }
 

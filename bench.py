@@ -138,6 +138,20 @@ class DeviceGradients:
         return self.grads
 
 
+def max_over_ranks(values, world, device, torch):
+    """Times of a multi-rank run are the maximum over the ranks (every rank runs the same replica)."""
+    t = torch.tensor([float(v) for v in values], device=device, dtype=torch.float64)
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t.tolist()]
+
+
+def replica_value(n_params, world, ms_per_step):
+    """Whole-job parameters per second of `world` independent replicas that each take ms_per_step."""
+    return world * n_params / (ms_per_step / 1e3)
+
+
 def fit_tau(w_name, n_layers, tau_req, gemm_prec, free_bytes, margin, br):
     """Largest ring depth <= tau_req whose state fits the device (ring bytes are linear in tau)."""
     def total(tau):
@@ -349,11 +363,9 @@ def main():
     steady = [t for t, r in zip(step_ms, is_refresh) if not r] or step_ms
     steady_ms = sum(steady) / len(steady)
     amortised_ms = steady_ms + refresh_ms / w.freq
-    times = torch.tensor([amortised_ms, steady_ms, refresh_ms, total_ms / args.steps], device=dev, dtype=torch.float64)
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    amortised_ms, steady_ms, refresh_ms, raw_ms = [float(x) for x in times.tolist()]
-    value = world * n_params / (amortised_ms / 1e3)
+    amortised_ms, steady_ms, refresh_ms, raw_ms = max_over_ranks(
+        [amortised_ms, steady_ms, refresh_ms, total_ms / args.steps], world, dev, torch)
+    value = replica_value(n_params, world, amortised_ms)
 
     # ---- end to end through the C-ABI with host buffers ------------------------------------------
     e2e = None

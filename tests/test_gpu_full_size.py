@@ -24,6 +24,10 @@ from workloads.configs import GEOM_BI, GEOM_UNI, SRC_SECOND
 pytestmark = pytest.mark.gpu
 
 TOL_DW = 2e-2
+# Factors: bf16 gradients are exact operands, the error is the fp32 accumulation in the tensor cores
+# (one rounding toward zero per 16-deep slice): on the diagonal, a sum of up to 32000 squares, that is a
+# one-sided error of about (32000 / 16) x 2^-24 = 1.2e-4 of the sum; 3e-4 leaves a factor of 2.5.
+TOL_FACTOR = 3e-4
 
 
 def _orthogonal(k, seed):
@@ -65,9 +69,9 @@ def _teacher_forced_steps(w, updates=2):
             assert rel_l2(sbs.state(li, br.BR_BUF_V2), lay.V2) < 2e-2
             assert rel_l2(sbs.state(li, br.BR_BUF_M), lay.M) < 1e-3
             if lay.L is not None:
-                assert rel_l2(sbs.state(li, br.BR_BUF_L), lay.L) < 1e-4
+                assert rel_l2(sbs.state(li, br.BR_BUF_L), lay.L) < TOL_FACTOR
             if lay.R is not None:
-                assert rel_l2(sbs.state(li, br.BR_BUF_R), lay.R) < 1e-4
+                assert rel_l2(sbs.state(li, br.BR_BUF_R), lay.R) < TOL_FACTOR
     finally:
         sbs.close()
 
@@ -187,3 +191,21 @@ def test_refresh_order_6912_properties():
         below = np.arange(k)[:, None] > cols[None, :]
         assert np.max(np.abs(R * below) / scale[None, :]) < 1e-3
         assert np.all(R[cols, np.arange(len(cols))] > 0)
+
+
+def test_c3_full_size_block_unilateral_first_moment():
+    """The block of C3 at full size: unilateral rotation of the smaller side (left for 1024x3072,
+    1024x1024, 1024x4096; right for 4096x1024), S = 1st, teacher-forced bases, two updates."""
+    w = replace(get_workload("c3"), tau=1, freq=10 ** 6)
+    w = replace(w, layers=[replace(l, tau_max=1) for l in w.layers])
+    _teacher_forced_steps(w, updates=2)
+
+
+def test_c4_shapes_full_size_student_t_gradients():
+    """One matrix of each distinct shape of C4 (d_model 2048, ffn 5632, embedding 32000x2048 unilateral)
+    with the heavy-tailed gradients of that configuration (1e-3 x Student-t, 3 degrees of freedom)."""
+    layers = [LayerSpec("wq", 2048, 2048, GEOM_BI, SRC_SECOND, 1), LayerSpec("wup", 2048, 5632, GEOM_BI, SRC_SECOND, 1),
+              LayerSpec("wdown", 5632, 2048, GEOM_BI, SRC_SECOND, 1), LayerSpec("emb", 32000, 2048, GEOM_UNI, SRC_SECOND, 1)]
+    base = get_workload("c4", n_layers=1, tau=1)
+    w = replace(base, layers=layers, tau=1, freq=10 ** 6)
+    _teacher_forced_steps(w, updates=1)

@@ -22,11 +22,24 @@
 // Every tensor map is 3-D; the third coordinate selects a ring slot for operands that live in
 // the stale-gradient ring and is 0 otherwise.
 //
+// Paired form (cta_group::2).  Two CTAs of a cluster, on neighbouring SMs, work on one 256 x 256
+// tile: each stages its own 128 rows of A and only half of B (128 of the 256 result columns), the
+// leader (cluster rank 0) issues tcgen05.mma.cta_group::2 of shape 256 x 256 x 16, which reads both
+// halves of B from the two shared memories and leaves rows 0..127 of the accumulator in the leader's
+// tensor memory and rows 128..255 in the peer's.  Per flop this takes two thirds of the L2 -> shared
+// memory traffic and half of the shared-memory reads of B, which is what bounds the unpaired form.
+// Barriers: both CTAs' TMA transactions complete on the leader's "full" barrier; the leader's
+// commits arrive on the "empty" and "accumulator full" barriers of both CTAs (one commit per CTA, the
+// peer's barrier addressed through mapa); the epilogue warps of both CTAs arrive on the leader's
+// "accumulator empty" barrier.  Both CTAs meet at a cluster barrier after set-up and before they free
+// their tensor memory, so neither exits while the other can still signal it.
+//
 // Every wait on an mbarrier is bounded: when a wait gives up the CTA raises an abort flag,
 // records BR_ERR_TIMEOUT in the status word, leaves its loops, frees its tensor memory and
 // returns; later launches return at once while the status word is negative.
 #include <cuda.h>
 
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 #include <string>
@@ -49,7 +62,19 @@ constexpr int SH_STAGE_BYTES = 2 * A_BYTES + 2 * B_BYTES;
 static_assert(SH_STAGES * SH_STAGE_BYTES == STAGES * STAGE_BYTES, "both forms use the same operand area");
 constexpr int EPI_LD = 33;                       // padded row of an epilogue tile (floats): rows and columns both conflict-free
 constexpr int EPI_BYTES = 4 * 32 * EPI_LD * 4;   // one 32 x 32 fp32 tile per epilogue warp
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BYTES + 1024;   // + slack to align the tiles to 1 KiB
+constexpr int OPERAND_BYTES = STAGES * STAGE_BYTES;                   // 192 KiB of operand stages in every form
+constexpr int SMEM_BYTES = OPERAND_BYTES + EPI_BYTES + 1024;          // + slack to align the tiles to 1 KiB
+constexpr int MAX_STAGES = 6;
+// Per-form geometry.  PAIR: the CTA pair owns a 256-row tile, each CTA stages 128 columns of B.
+template <bool SHARED, bool PAIR>
+struct Form {
+  static constexpr int TM = PAIR ? 2 * BM : BM;                 // rows of a tile
+  static constexpr int BNC = PAIR ? BN / 2 : BN;                // result columns whose B rows this CTA stages
+  static constexpr int BB = BNC * BK * 2;                       // bytes of one staged B tile
+  static constexpr int STAGE = SHARED ? 2 * A_BYTES + 2 * BB : A_BYTES + BB;
+  static constexpr int NST = OPERAND_BYTES / STAGE;             // 4 / 2 unpaired, 6 / 3 paired
+  static_assert(NST <= MAX_STAGES && NST * STAGE == OPERAND_BYTES, "stages fill the operand area");
+};
 constexpr int TMEM_COLS = 512;
 constexpr int NUM_THREADS = 192;                 // warp 0: TMA, warp 1: MMA, warps 2..5: epilogue
 constexpr int MAX_PAIRS = 3;
@@ -100,6 +125,38 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok;
 }
+// the same with cluster scope: the barrier also receives arrivals from the other CTA of a pair
+__device__ __forceinline__ uint32_t mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok;
+}
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ uint32_t ld_cluster_u32(uint32_t cluster_addr) {
+  uint32_t v;
+  asm volatile("ld.shared::cluster.u32 %0, [%1];" : "=r"(v) : "r"(cluster_addr) : "memory");
+  return v;
+}
+__device__ __forceinline__ void cluster_barrier() {
+  asm volatile("barrier.cluster.arrive.release;\n\tbarrier.cluster.wait.acquire;" ::: "memory");
+}
 __device__ __forceinline__ uint64_t global_timer_ns() {
   uint64_t t;
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
@@ -109,13 +166,15 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
 constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s: far above any legitimate wait
 
 // Bounded wait.  Returns false when the wait gave up or another role raised the abort flag.
+template <bool CLUSTER = false>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                           int* status) {
-  if (mbar_try_wait(bar, parity)) return true;
+  auto try_wait = [&] { return CLUSTER ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity); };
+  if (try_wait()) return true;
   const uint64_t t0 = global_timer_ns();
   uint32_t spins = 0;
   while (true) {
-    if (mbar_try_wait(bar, parity)) return true;
+    if (try_wait()) return true;
     if ((++spins & 0xFF) == 0) {
       if (*abort_flag) return false;
       if (global_timer_ns() - t0 > kWaitLimitNs) {
@@ -136,6 +195,16 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
       : "memory");
 }
 
+// paired form: the transaction completes on `bar`, a shared::cluster address that may lie in the leader CTA
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar,
+                                                 int x, int y, int z) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(x), "r"(y), "r"(z)
+      : "memory");
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -146,6 +215,18 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint6
       "setp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                               uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// paired form: `bar` is a shared::cluster address (this CTA's barrier or the peer's)
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 // Arrive on an mbarrier once every tcgen05.mma issued so far by this thread has completed.
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
@@ -183,7 +264,7 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, uint32_t lbo, 
 }
 
 // Instruction descriptor of kind::f16: fp32 accumulator, bf16 A and B, M = 128, N = 256.
-__device__ __forceinline__ uint32_t make_idesc(int a_mn, int b_mn) {
+__device__ __forceinline__ uint32_t make_idesc(int a_mn, int b_mn, int rows = BM) {
   uint32_t d = 0;
   d |= 1u << 4;                       // accumulator format: fp32
   d |= 1u << 7;                       // A format: bf16
@@ -191,7 +272,7 @@ __device__ __forceinline__ uint32_t make_idesc(int a_mn, int b_mn) {
   d |= (uint32_t)(a_mn ? 1 : 0) << 15;
   d |= (uint32_t)(b_mn ? 1 : 0) << 16;
   d |= (uint32_t)(BN >> 3) << 17;
-  d |= (uint32_t)(BM >> 4) << 24;
+  d |= (uint32_t)(rows >> 4) << 24;
   return d;
 }
 
@@ -207,6 +288,7 @@ struct TileInfo {
 };
 
 // tile index -> problem (binary search over tile_begin) and block coordinates
+template <int TM>
 __device__ __forceinline__ TileInfo locate_tile(const DevProblem* probs, int n_probs, int tile,
                                                 long long calls, int tau) {
   int lo = 0, hi = n_probs - 1;
@@ -223,7 +305,7 @@ __device__ __forceinline__ TileInfo locate_tile(const DevProblem* probs, int n_p
   const int first_m = group * GROUP_M;
   const int gsz = min(p->tiles_m - first_m, GROUP_M);
   const int in_group = local - group * per_group;
-  ti.m0 = (first_m + in_group % gsz) * BM;
+  ti.m0 = (first_m + in_group % gsz) * TM;
   ti.n0 = (in_group / gsz) * BN;
   // delayed-gradient bookkeeping: the layer is active once call - tau >= 1; the gradient to
   // apply sits in ring slot (calls - 1 - tau) mod slots
@@ -239,58 +321,86 @@ __device__ __forceinline__ TileInfo locate_tile(const DevProblem* probs, int n_p
 // ---------------------------------------------------------------------------------------------
 // The kernel
 // ---------------------------------------------------------------------------------------------
-template <bool SHARED>
+template <bool SHARED, bool PAIR>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 k_tc_gemm(const DevProblem* __restrict__ probs, int n_probs, int first_tile, int total_tiles, long long calls,
           int tau, float dyn_alpha, float dyn_beta, int* status) {
-  constexpr int NST = SHARED ? SH_STAGES : STAGES;
+  using F = Form<SHARED, PAIR>;
+  constexpr int NST = F::NST;
+  constexpr int TM = F::TM;
   extern __shared__ uint8_t smem_raw[];
-  __shared__ alignas(8) uint64_t bars[2 * STAGES + 4];
+  __shared__ alignas(8) uint64_t bars[2 * MAX_STAGES + 4];
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_word;
+  __shared__ uint32_t dead_word;
   volatile int* abort_flag = &abort_word;
 
-  if (*reinterpret_cast<volatile int*>(status) < 0) return;   // an earlier launch failed
+  // an earlier launch failed: nothing to do (a pair takes the decision from its leader, below)
+  if (!PAIR && *reinterpret_cast<volatile int*>(status) < 0) return;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = PAIR ? cluster_ctarank() : 0u;        // 0: leader of the pair
+  const int unit = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;      // index of this CTA (pair) in the tile walk
+  const int n_units = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
   const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   // operand slot i of stage s
   auto sA = [&](int s, int i) {
-    return SHARED ? tiles_base + (uint32_t)s * SH_STAGE_BYTES + (uint32_t)i * A_BYTES
+    return SHARED ? tiles_base + (uint32_t)s * F::STAGE + (uint32_t)i * A_BYTES
                   : tiles_base + (uint32_t)s * A_BYTES;
   };
   auto sB = [&](int s, int i) {
-    return SHARED ? tiles_base + (uint32_t)s * SH_STAGE_BYTES + 2u * A_BYTES + (uint32_t)i * B_BYTES
-                  : tiles_base + (uint32_t)STAGES * A_BYTES + (uint32_t)s * B_BYTES;
+    return SHARED ? tiles_base + (uint32_t)s * F::STAGE + 2u * A_BYTES + (uint32_t)i * F::BB
+                  : tiles_base + (uint32_t)NST * A_BYTES + (uint32_t)s * F::BB;
   };
-  float* epi_tiles = reinterpret_cast<float*>(smem_raw + ((tiles_base - smem_u32(smem_raw)) + (uint32_t)STAGES * STAGE_BYTES));
+  float* epi_tiles = reinterpret_cast<float*>(smem_raw + ((tiles_base - smem_u32(smem_raw)) + (uint32_t)OPERAND_BYTES));
   const uint32_t bar0 = smem_u32(bars);
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
-  auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
-  auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + a); };
-  auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + 2 + a); };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (MAX_STAGES + s); };
+  auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * MAX_STAGES + a); };
+  auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * MAX_STAGES + 2 + a); };
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < NST; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
+    // accumulator hand-back: four epilogue warps, of both CTAs in the paired form
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), PAIR ? 8 : 4); }
     abort_word = 0;
+    dead_word = (*reinterpret_cast<volatile int*>(status) < 0) ? 1u : 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(TMEM_COLS) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if (PAIR) {
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(TMEM_COLS) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(TMEM_COLS) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
   }
   tc_fence_before();
   __syncthreads();
+  bool dead = false;
+  if (PAIR) {
+    // both CTAs have initialised their barriers before either signals the other; the pair skips its
+    // work together when the leader saw a failed status word
+    cluster_barrier();
+    dead = ld_cluster_u32(map_to_cta(smem_u32(&dead_word), 0)) != 0u;
+  }
   tc_fence_after();
   const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&tmem_slot);
+  if (dead) first_tile = total_tiles;          // every role finds an empty tile list
 
   if (warp == 0) {
     // ======================= TMA producer =======================
     if (lane == 0) {
       int stage = 0; uint32_t phase = 0;
-      for (int tile = first_tile + blockIdx.x; tile < total_tiles && !*abort_flag; tile += gridDim.x) {
-        const TileInfo ti = locate_tile(probs, n_probs, tile, calls, tau);
+      // paired form: the CTA's own rows of A and its half of the rows of B; every transaction of
+      // the pair completes on the leader's barrier, on which only the leader posts the byte count
+      const int row_off = (int)rank * BM, col_off = (int)rank * F::BNC;
+      auto load = [&](uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y, int z) {
+        if (PAIR) tma_load_3d_pair(dst, map, bar, x, y, z); else tma_load_3d(dst, map, bar, x, y, z);
+      };
+      for (int tile = first_tile + unit; tile < total_tiles && !*abort_flag; tile += n_units) {
+        const TileInfo ti = locate_tile<TM>(probs, n_probs, tile, calls, tau);
         if (!ti.active) continue;
         const DevProblem* p = ti.p;
         const int nkb = (p->K + BK - 1) / BK;
@@ -298,27 +408,29 @@ k_tc_gemm(const DevProblem* __restrict__ probs, int n_probs, int first_tile, int
         auto load_a = [&](uint32_t dst, const CUtensorMap* ma, int k0, int za, uint32_t bar) {
           if (p->a_mn) {
 #pragma unroll
-            for (int j = 0; j < BM / 64; ++j) tma_load_3d(dst + j * (BK * 128), ma, bar, ti.m0 + 64 * j, k0, za);
+            for (int j = 0; j < BM / 64; ++j) load(dst + j * (BK * 128), ma, bar, ti.m0 + row_off + 64 * j, k0, za);
           } else {
-            tma_load_3d(dst, ma, bar, k0, ti.m0, za);
+            load(dst, ma, bar, k0, ti.m0 + row_off, za);
           }
         };
         auto load_b = [&](uint32_t dst, const CUtensorMap* mb, int k0, int zb, uint32_t bar) {
           if (p->b_mn) {
 #pragma unroll
-            for (int j = 0; j < BN / 64; ++j) tma_load_3d(dst + j * (BK * 128), mb, bar, ti.n0 + 64 * j, k0, zb);
+            for (int j = 0; j < F::BNC / 64; ++j) load(dst + j * (BK * 128), mb, bar, ti.n0 + col_off + 64 * j, k0, zb);
           } else {
-            tma_load_3d(dst, mb, bar, k0, ti.n0, zb);
+            load(dst, mb, bar, k0, ti.n0 + col_off, zb);
           }
         };
+        const uint32_t copies = PAIR ? 2u : 1u;
         if (SHARED) {
           for (int kb = 0; kb < nkb; ++kb) {
             if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, status)) { ok = false; break; }
-            mbar_expect_tx(full_bar(stage), (uint32_t)(p->nA * A_BYTES + p->nB * B_BYTES));
+            const uint32_t fb = PAIR ? map_to_cta(full_bar(stage), 0) : full_bar(stage);
+            if (rank == 0) mbar_expect_tx(full_bar(stage), copies * (uint32_t)(p->nA * A_BYTES + p->nB * F::BB));
             for (int i = 0; i < p->nA; ++i)
-              load_a(sA(stage, i), &p->mapA[i], kb * BK, ((p->a_ring_mask >> i) & 1) ? ti.z : 0, full_bar(stage));
+              load_a(sA(stage, i), &p->mapA[i], kb * BK, ((p->a_ring_mask >> i) & 1) ? ti.z : 0, fb);
             for (int i = 0; i < p->nB; ++i)
-              load_b(sB(stage, i), &p->mapB[i], kb * BK, ((p->b_ring_mask >> i) & 1) ? ti.z : 0, full_bar(stage));
+              load_b(sB(stage, i), &p->mapB[i], kb * BK, ((p->b_ring_mask >> i) & 1) ? ti.z : 0, fb);
             if (++stage == NST) { stage = 0; phase ^= 1u; }
           }
         } else {
@@ -327,9 +439,10 @@ k_tc_gemm(const DevProblem* __restrict__ probs, int n_probs, int first_tile, int
             const int zb = ((p->b_ring_mask >> pr) & 1) ? ti.z : 0;
             for (int kb = 0; kb < nkb; ++kb) {
               if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, status)) { ok = false; break; }
-              mbar_expect_tx(full_bar(stage), STAGE_BYTES);
-              load_a(sA(stage, 0), &p->mapA[pr], kb * BK, za, full_bar(stage));
-              load_b(sB(stage, 0), &p->mapB[pr], kb * BK, zb, full_bar(stage));
+              const uint32_t fb = PAIR ? map_to_cta(full_bar(stage), 0) : full_bar(stage);
+              if (rank == 0) mbar_expect_tx(full_bar(stage), copies * (uint32_t)F::STAGE);
+              load_a(sA(stage, 0), &p->mapA[pr], kb * BK, za, fb);
+              load_b(sB(stage, 0), &p->mapB[pr], kb * BK, zb, fb);
               if (++stage == NST) { stage = 0; phase ^= 1u; }
             }
           }
@@ -339,20 +452,25 @@ k_tc_gemm(const DevProblem* __restrict__ probs, int n_probs, int first_tile, int
     }
   } else if (warp == 1) {
     // ======================= MMA issuer =======================
-    if (lane == 0) {
+    // (paired form: the leader issues for both CTAs; the peer's warp only owns the tensor-memory allocation)
+    if (lane == 0 && rank == 0) {
       int stage = 0; uint32_t phase = 0;
       int acc = 0; uint32_t acc_phase = 0;
-      for (int tile = first_tile + blockIdx.x; tile < total_tiles && !*abort_flag; tile += gridDim.x) {
-        const TileInfo ti = locate_tile(probs, n_probs, tile, calls, tau);
+      // a commit arrives on this CTA's barrier and, in the paired form, on the peer's as well
+      auto commit = [&](uint32_t bar) {
+        if (PAIR) { umma_commit_pair(bar); umma_commit_pair(map_to_cta(bar, 1)); } else { umma_commit(bar); }
+      };
+      for (int tile = first_tile + unit; tile < total_tiles && !*abort_flag; tile += n_units) {
+        const TileInfo ti = locate_tile<TM>(probs, n_probs, tile, calls, tau);
         if (!ti.active) continue;
         const DevProblem* p = ti.p;
         const int nkb = (p->K + BK - 1) / BK;
-        const uint32_t idesc = make_idesc(p->a_mn, p->b_mn);
+        const uint32_t idesc = make_idesc(p->a_mn, p->b_mn, TM);
         // K-major: advance 32 bytes per 16-element k step inside the swizzle row;
         // MN-major: 16 k rows = two 8-row groups of 1024 bytes.
         const uint32_t a_lbo = p->a_mn ? BK * 128 : 0, a_adv = p->a_mn ? 2048 : 32;
         const uint32_t b_lbo = p->b_mn ? BK * 128 : 0, b_adv = p->b_mn ? 2048 : 32;
-        if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, status)) break;
+        if (!mbar_wait<PAIR>(tempty_bar(acc), acc_phase ^ 1u, abort_flag, status)) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)acc * BN;
         uint32_t accumulate = 0;
@@ -369,16 +487,20 @@ k_tc_gemm(const DevProblem* __restrict__ probs, int n_probs, int first_tile, int
             const uint64_t bdesc = make_smem_desc(sB(stage, bi), b_lbo, 1024);
 #pragma unroll
             for (int k = 0; k < BK / UMMA_K; ++k) {
-              umma_bf16(d_tmem, adesc + (uint64_t)((k * a_adv) >> 4), bdesc + (uint64_t)((k * b_adv) >> 4),
-                        idesc, accumulate);
+              if (PAIR)
+                umma_bf16_pair(d_tmem, adesc + (uint64_t)((k * a_adv) >> 4), bdesc + (uint64_t)((k * b_adv) >> 4),
+                               idesc, accumulate);
+              else
+                umma_bf16(d_tmem, adesc + (uint64_t)((k * a_adv) >> 4), bdesc + (uint64_t)((k * b_adv) >> 4),
+                          idesc, accumulate);
               accumulate = 1;
             }
           }
-          umma_commit(empty_bar(stage));          // frees the stage once these MMAs have read it
+          commit(empty_bar(stage));               // frees the stage once these MMAs have read it
           if (++stage == NST) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
-        umma_commit(tfull_bar(acc));              // accumulator complete
+        commit(tfull_bar(acc));                   // accumulator complete
         acc ^= 1;
         if (acc == 0) acc_phase ^= 1u;
       }
@@ -396,8 +518,8 @@ k_tc_gemm(const DevProblem* __restrict__ probs, int n_probs, int first_tile, int
     float* tile = epi_tiles + quad * (32 * EPI_LD);
     const int sub_r = lane >> 3, sub_c = (lane & 7) * 4;
     int acc = 0; uint32_t acc_phase = 0;
-    for (int tile_i = first_tile + blockIdx.x; tile_i < total_tiles && !*abort_flag; tile_i += gridDim.x) {
-      const TileInfo ti = locate_tile(probs, n_probs, tile_i, calls, tau);
+    for (int tile_i = first_tile + unit; tile_i < total_tiles && !*abort_flag; tile_i += n_units) {
+      const TileInfo ti = locate_tile<TM>(probs, n_probs, tile_i, calls, tau);
       if (!ti.active) continue;
       const DevProblem* p = ti.p;
       float alpha = p->dyn_scalars ? dyn_alpha : p->alpha;
@@ -411,7 +533,7 @@ k_tc_gemm(const DevProblem* __restrict__ probs, int n_probs, int first_tile, int
         gclip = p->clip[(int)((calls - 1 - tl) % p->clip_slots)];
         if (p->clip_mode == 2) alpha *= gclip * gclip;
       }
-      const int row_base = ti.m0 + quad * 32;
+      const int row_base = ti.m0 + (int)rank * BM + quad * 32;
       const bool quad_ok = row_base < p->Md;      // uniform across the warp
       const bool reads_d = (epi == EPI_AXPBY_F32 && beta != 0.0f) || epi == EPI_ROTATED_ADAM ||
                            epi == EPI_SECOND_MOMENT || epi == EPI_SCALE_BF16;
@@ -577,18 +699,25 @@ k_tc_gemm(const DevProblem* __restrict__ probs, int n_probs, int first_tile, int
       // all tcgen05.ld of this warp have completed (wait::ld): hand the accumulator back
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(tempty_bar(acc));
+      if (lane == 0) {
+        if (PAIR) mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0)); else mbar_arrive(tempty_bar(acc));
+      }
       acc ^= 1;
       if (acc == 0) acc_phase ^= 1u;
     }
   }
 
   // teardown: every role has left its loop (all waits are bounded)
+  // (paired form: neither CTA frees its tensor memory or exits while the other may still signal it)
   tc_fence_before();
   __syncthreads();
+  if (PAIR) cluster_barrier();
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    if (PAIR)
+      asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    else
+      asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
   }
 }
 
@@ -641,10 +770,51 @@ bool encode_operand(CUtensorMap* map, const TcOperand& op, int64_t rows, int64_t
   return true;
 }
 
+typedef void (*TcKernel)(const DevProblem*, int, int, int, long long, int, float, float, int*);
+TcKernel kernel_of(bool shared, bool pair) {
+  if (pair) return shared ? k_tc_gemm<true, true> : k_tc_gemm<false, true>;
+  return shared ? k_tc_gemm<true, false> : k_tc_gemm<false, false>;
+}
+
+// Number of CTA pairs (clusters of two) of the paired form that fit on the current device at once;
+// 0 unless that form is switched on (environment BR_TC_PAIR=1) and can be launched.
+int pair_capacity(bool shared) {
+  static int cap[2] = {-1, -1};
+  static std::mutex mu;
+  std::lock_guard<std::mutex> lock(mu);
+  int& c = cap[shared ? 1 : 0];
+  if (c >= 0) return c;
+  c = 0;
+  const char* env = std::getenv("BR_TC_PAIR");
+  if (!env || env[0] != '1') return c;
+  TcKernel kernel = kernel_of(shared, true);
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) {
+    cudaGetLastError();
+    return c;
+  }
+  int dev = 0, sms = 0;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.gridDim = dim3(2u * (unsigned)(sms / 2));
+  cfg.blockDim = dim3(NUM_THREADS);
+  cfg.dynamicSmemBytes = SMEM_BYTES;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  int clusters = 0;
+  if (cudaOccupancyMaxActiveClusters(&clusters, kernel, &cfg) != cudaSuccess) { cudaGetLastError(); return c; }
+  c = clusters < sms / 2 ? clusters : sms / 2;
+  return c;
+}
+
 }  // namespace
 
 struct TcPlan {
   bool shared = false;          // launches the shared-operand form of the kernel
+  bool pair = false;            // launches the paired form (clusters of two CTAs, 256-row tiles)
+  int max_pairs = 0;            // CTA pairs that can be resident at once
   std::vector<int> tile_begin;  // per problem, plus the total at the end
   std::vector<double> prob_flops;
   DevProblem* d_probs = nullptr;
@@ -688,6 +858,10 @@ TcPlan* tc_plan_create(const TcProblem* problems, int n, int device, cudaStream_
     if (nA > 2 || nB > 2) eligible = false;
   }
   shared = shared && eligible;
+  const int pairs = pair_capacity(shared);
+  const bool pair = pairs > 0;
+  const int TM = pair ? 2 * BM : BM;            // rows of a tile
+  const int b_box = pair ? BN / 2 : BN;         // rows of B one CTA stages per k-block
   std::vector<DevProblem> host(n);
   std::vector<int> tile_starts;
   std::vector<double> prob_flops;
@@ -720,21 +894,21 @@ TcPlan* tc_plan_create(const TcProblem* problems, int n, int device, cudaStream_
         if (q.A[ua[u]].ring_slots > 0) { d.a_ring_mask |= 1 << u; d.ring_slots = q.A[ua[u]].ring_slots; }
       }
       for (int u = 0; u < nB; ++u) {
-        if (!encode_operand(&d.mapB[u], q.B[ub[u]], q.Nd, q.K, BN, &e)) return fail(e);
+        if (!encode_operand(&d.mapB[u], q.B[ub[u]], q.Nd, q.K, b_box, &e)) return fail(e);
         if (q.B[ub[u]].ring_slots > 0) { d.b_ring_mask |= 1 << u; d.ring_slots = q.B[ub[u]].ring_slots; }
       }
       d.nA = nA; d.nB = nB; d.combos = combos | (q.n_pairs << 8);
     } else {
       for (int p = 0; p < q.n_pairs; ++p) {
         if (!encode_operand(&d.mapA[p], q.A[p], q.Md, q.K, BM, &e)) return fail(e);
-        if (!encode_operand(&d.mapB[p], q.B[p], q.Nd, q.K, BN, &e)) return fail(e);
+        if (!encode_operand(&d.mapB[p], q.B[p], q.Nd, q.K, b_box, &e)) return fail(e);
         if (q.A[p].ring_slots > 0) { d.a_ring_mask |= 1 << p; d.ring_slots = q.A[p].ring_slots; }
         if (q.B[p].ring_slots > 0) { d.b_ring_mask |= 1 << p; d.ring_slots = q.B[p].ring_slots; }
       }
     }
     d.Md = (int32_t)q.Md; d.Nd = (int32_t)q.Nd; d.K = (int32_t)q.K; d.n_pairs = q.n_pairs;
     d.a_mn = q.A[0].mn_major; d.b_mn = q.B[0].mn_major; d.epilogue = q.epilogue;
-    d.tiles_m = (int32_t)((q.Md + BM - 1) / BM);
+    d.tiles_m = (int32_t)((q.Md + TM - 1) / TM);
     d.tiles_n = (int32_t)((q.Nd + BN - 1) / BN);
     d.tile_begin = tile_begin;
     d.tile_count = d.tiles_m * d.tiles_n;
@@ -765,8 +939,8 @@ TcPlan* tc_plan_create(const TcProblem* problems, int n, int device, cudaStream_
       int64_t computed = 0;
       for (int64_t rb = 0; rb < d.tiles_m; ++rb)
         for (int64_t cb = 0; cb < d.tiles_n; ++cb)
-          if (rb * BM < cb * BN + BN) ++computed;
-      flops += 2.0 * (double)computed * BM * BN * (double)q.K * q.n_pairs;
+          if (rb * TM < cb * BN + BN) ++computed;
+      flops += 2.0 * (double)computed * TM * BN * (double)q.K * q.n_pairs;
     } else {
       flops += 2.0 * (double)q.Md * (double)q.Nd * (double)q.K * q.n_pairs;
     }
@@ -774,6 +948,8 @@ TcPlan* tc_plan_create(const TcProblem* problems, int n, int device, cudaStream_
   }
   TcPlan* plan = new TcPlan();
   plan->shared = shared;
+  plan->pair = pair;
+  plan->max_pairs = pairs;
   tile_starts.push_back(tile_begin);
   plan->tile_begin = tile_starts;
   plan->prob_flops = prob_flops;
@@ -791,11 +967,6 @@ TcPlan* tc_plan_create(const TcProblem* problems, int n, int device, cudaStream_
     delete plan;
     return fail(std::string("plan upload: ") + cudaGetErrorString(ce));
   }
-  static std::once_flag attr_once;
-  std::call_once(attr_once, [] {
-    cudaFuncSetAttribute(k_tc_gemm<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
-    cudaFuncSetAttribute(k_tc_gemm<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
-  });
   return plan;
 }
 
@@ -812,18 +983,25 @@ cudaError_t tc_plan_launch_range(TcPlan* p, int first, int count, long long call
   if (first < 0 || count < 1 || first + count > p->n) return cudaErrorInvalidValue;
   const int t0 = p->tile_begin[first], t1 = p->tile_begin[first + count];
   const int tiles = t1 - t0;
-  const int grid = tiles < p->sm_count ? tiles : p->sm_count;
+  TcKernel kernel = kernel_of(p->shared, p->pair);
   // per-device attribute: set again when another device is current (cheap, idempotent)
-  if (p->shared) {
-    cudaFuncSetAttribute(k_tc_gemm<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
-    k_tc_gemm<true><<<grid, NUM_THREADS, SMEM_BYTES, s>>>(p->d_probs, p->n, t0, t1, calls, tau, dyn_alpha,
-                                                          dyn_beta, status_word);
+  cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute attr[1];
+  if (p->pair) {
+    const int units = tiles < p->max_pairs ? tiles : p->max_pairs;
+    cfg.gridDim = dim3(2u * (unsigned)units);
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
   } else {
-    cudaFuncSetAttribute(k_tc_gemm<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
-    k_tc_gemm<false><<<grid, NUM_THREADS, SMEM_BYTES, s>>>(p->d_probs, p->n, t0, t1, calls, tau, dyn_alpha,
-                                                           dyn_beta, status_word);
+    cfg.gridDim = dim3((unsigned)(tiles < p->sm_count ? tiles : p->sm_count));
   }
-  return cudaGetLastError();
+  cfg.blockDim = dim3(NUM_THREADS);
+  cfg.dynamicSmemBytes = SMEM_BYTES;
+  cfg.stream = s;
+  return cudaLaunchKernelEx(&cfg, kernel, (const DevProblem*)p->d_probs, p->n, t0, t1, calls, tau, dyn_alpha,
+                            dyn_beta, status_word);
 }
 
 cudaError_t tc_plan_launch(TcPlan* p, long long calls, int tau, float dyn_alpha, float dyn_beta,

@@ -777,7 +777,7 @@ TcKernel kernel_of(bool shared, bool pair) {
 }
 
 // Number of CTA pairs (clusters of two) of the paired form that fit on the current device at once;
-// 0 unless that form is switched on (environment BR_TC_PAIR=1) and can be launched.
+// 0 when that form is switched off (environment BR_TC_PAIR=0) or cannot be launched.
 int pair_capacity(bool shared) {
   static int cap[2] = {-1, -1};
   static std::mutex mu;
@@ -786,7 +786,7 @@ int pair_capacity(bool shared) {
   if (c >= 0) return c;
   c = 0;
   const char* env = std::getenv("BR_TC_PAIR");
-  if (!env || env[0] != '1') return c;
+  if (env && env[0] == '0') return c;
   TcKernel kernel = kernel_of(shared, true);
   if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) {
     cudaGetLastError();

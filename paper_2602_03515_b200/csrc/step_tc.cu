@@ -13,7 +13,7 @@
 //
 //   factors   L <- b L + (1-b) G G^T , R <- b R + (1-b) G^T G            (Alg. 2)
 //   [refresh of the layers that are due, bracketed by the re-expression]  (Alg. 1 lines 5-6)
-//   fwd1      T = U^T G                               -> bf16 hi/lo       (Alg. 1 line 8, first side)
+//   fwd1      T = U^T G  (or T = G V when n > m: the larger side first) -> bf16 hi/lo   (Alg. 1 line 8, first side)
 //   adam      G~ = T V, fused epilogue: M~ <- b1 M~ + (1-b1) G~ ; V~ <- b2 V~ + (1-b2) G~^2 ;
 //             X = M~ / sqrt(V~ + eps)                                      (lines 4, 8-11)
 //   back1     Y = U X
@@ -126,18 +126,36 @@ void step_problems(const Layer& L, const LayerScratch& S, const br_hparams& hp, 
   const int64_t m = L.d.m, n = L.d.n;
   const int tm = L.d.tau_max;
   if (L.left && L.right) {
-    {  // T = U^T G : (Uh, G) + (Ul, G); U and G both enter MN-major (contraction over rows)
-      TcProblem q; q.Md = m; q.Nd = n; q.K = m; q.n_pairs = 2; q.tau_max = tm;
-      q.A[0] = op(L.Uh, m, 1); q.B[0] = ring_op(L, 1);
-      q.A[1] = op(L.Ul, m, 1); q.B[1] = ring_op(L, 1);
-      q.epilogue = EPI_SPLIT_BF16; q.Dh = S.B[0]; q.Dl = S.B[1]; q.ldh = n;
-      P->fwd1.push_back(q);
-    }
-    {  // G~ = T V : T K-major, V MN-major
-      TcProblem q; q.Md = m; q.Nd = n; q.K = n; q.tau_max = tm;
-      three_pairs(q, S.B[0], S.B[1], n, 0, L.Vh, L.Vl, n, 1);
-      rotated_adam_epilogue(q, L, hp, S.B[2]);
-      P->adam.push_back(q);
+    // The first side costs two products (the gradient is bf16 already), the second three (both
+    // operands are hi/lo pairs): mn (4 d1 + 6 d2) flop for side orders d1, d2.  The larger side goes first.
+    if (n > m) {
+      {  // T = G V : G K-major, V MN-major
+        TcProblem q; q.Md = m; q.Nd = n; q.K = n; q.n_pairs = 2; q.tau_max = tm;
+        q.A[0] = ring_op(L, 0); q.B[0] = op(L.Vh, n, 1);
+        q.A[1] = ring_op(L, 0); q.B[1] = op(L.Vl, n, 1);
+        q.epilogue = EPI_SPLIT_BF16; q.Dh = S.B[0]; q.Dl = S.B[1]; q.ldh = n;
+        P->fwd1.push_back(q);
+      }
+      {  // G~ = U^T T : both MN-major (contraction over rows)
+        TcProblem q; q.Md = m; q.Nd = n; q.K = m; q.tau_max = tm;
+        three_pairs(q, L.Uh, L.Ul, m, 1, S.B[0], S.B[1], n, 1);
+        rotated_adam_epilogue(q, L, hp, S.B[2]);
+        P->adam.push_back(q);
+      }
+    } else {
+      {  // T = U^T G : (Uh, G) + (Ul, G); U and G both enter MN-major (contraction over rows)
+        TcProblem q; q.Md = m; q.Nd = n; q.K = m; q.n_pairs = 2; q.tau_max = tm;
+        q.A[0] = op(L.Uh, m, 1); q.B[0] = ring_op(L, 1);
+        q.A[1] = op(L.Ul, m, 1); q.B[1] = ring_op(L, 1);
+        q.epilogue = EPI_SPLIT_BF16; q.Dh = S.B[0]; q.Dl = S.B[1]; q.ldh = n;
+        P->fwd1.push_back(q);
+      }
+      {  // G~ = T V : T K-major, V MN-major
+        TcProblem q; q.Md = m; q.Nd = n; q.K = n; q.tau_max = tm;
+        three_pairs(q, S.B[0], S.B[1], n, 0, L.Vh, L.Vl, n, 1);
+        rotated_adam_epilogue(q, L, hp, S.B[2]);
+        P->adam.push_back(q);
+      }
     }
     {  // Y = U X : U K-major, X MN-major
       TcProblem q; q.Md = m; q.Nd = n; q.K = m; q.n_pairs = 1; q.tau_max = tm;

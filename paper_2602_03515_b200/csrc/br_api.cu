@@ -7,6 +7,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <map>
 #include <string>
 #include <vector>
 
@@ -104,8 +105,21 @@ struct br_handle {
     double *rA = nullptr, *rF = nullptr, *rQ = nullptr, *rZ = nullptr, *rWork = nullptr;
     char* tcq_scratch = nullptr;          // scratch of the tensor-core projections (largest eligible order)
     std::vector<QrTc*> tcq;               // their plans, one per distinct eligible order
+    int64_t cap_k = 0;                    // largest order this lane's buffers hold
+    // The orthonormalisation of one basis is several hundred dependent launches whose arguments
+    // depend only on the lane (its buffers) and on the order: it is captured into a CUDA graph the
+    // first time and replayed afterwards, one launch per basis.  Key: 2 * order + (tensor-core form).
+    struct QrGraph { cudaGraphExec_t exec = nullptr; int64_t launches = 0; double flops = 0.0; };
+    std::map<int64_t, QrGraph> qr_graphs;
+    int* cond = nullptr;                  // conditioning note of the lane's current job (device)
   };
-  static constexpr int kMaxLanes = 3;
+  bool use_graphs = true;                 // cleared when a capture fails (BR_REFRESH_GRAPHS=0 switches it off)
+  // Up to three lanes hold the largest order; up to five more hold only the small orders (at most
+  // 1/sqrt(2) of the largest, S = 2nd), whose refresh is a chain of short launches that leaves most of
+  // the GPU idle: eight streams in all, the default number of hardware queues.
+  static constexpr int kBigLanes = 3;
+  static constexpr int kSmallLanes = 5;
+  static constexpr int kMaxLanes = kBigLanes + kSmallLanes;
   Lane lanes[kMaxLanes];
   int n_lanes = 1;
   cudaEvent_t ev_begin = nullptr;
@@ -186,20 +200,45 @@ void layout(br_handle* h, Bump& b, Sizes* sz) {
     if (L.right) h->tcq_bytes = std::max(h->tcq_bytes, qr_tc_scratch_bytes(L.d.n));
   }
   if (max_k) {
-    h->n_lanes = (int)std::min<size_t>(br_handle::kMaxLanes, std::max<size_t>(1, n_sides));
-    // tuning aid: BR_REFRESH_LANES=1..3 caps the number of concurrent refresh lanes
+    int n_big = (int)std::min<size_t>(br_handle::kBigLanes, std::max<size_t>(1, n_sides));
+    // tuning aid: BR_REFRESH_LANES=1..3 caps the number of concurrent full-size refresh lanes
     if (const char* env = std::getenv("BR_REFRESH_LANES")) {
       const int v = std::atoi(env);
-      if (v >= 1 && v < h->n_lanes) h->n_lanes = v;
+      if (v >= 1 && v < n_big) n_big = v;
     }
+    // the small class: orders of S = 2nd sides of at most max_k / sqrt(2)
+    size_t small_k = 0, n_small_sides = 0;
+    std::vector<size_t> orders;
+    for (const Layer& L : h->layers) {
+      if (L.d.geom == BR_GEOM_NONE) continue;
+      for (size_t k : {L.left ? (size_t)L.d.m : (size_t)0, L.right ? (size_t)L.d.n : (size_t)0}) {
+        if (!k) continue;
+        orders.push_back(k);
+        if (L.d.src == BR_SRC_SECOND && 2 * k * k <= max_k * max_k) { small_k = std::max(small_k, k); ++n_small_sides; }
+      }
+    }
+    int n_small = (int)std::min<size_t>(br_handle::kSmallLanes, n_small_sides);
+    if ((int)n_sides <= n_big) n_small = 0;
+    // tuning aid: BR_REFRESH_SMALL_LANES=0..5 caps the number of small-order lanes
+    if (const char* env = std::getenv("BR_REFRESH_SMALL_LANES")) {
+      const int v = std::atoi(env);
+      if (v >= 0 && v < n_small) n_small = v;
+    }
+    h->n_lanes = n_big + n_small;
     for (int i = 0; i < h->n_lanes; ++i) {
       br_handle::Lane& ln = h->lanes[i];
-      ln.rA = b.take<double>(max_k * max_k);
-      ln.rF = b.take<double>(max_k * max_k);
-      ln.rQ = b.take<double>(max_k * max_k);
-      ln.rWork = b.take<double>(std::max<size_t>(qr_work_doubles((int64_t)max_k), 1056));   // also 1025 doubles of norm scratch
-      if (max_z) ln.rZ = b.take<double>(max_z);
-      if (h->tcq_bytes) ln.tcq_scratch = b.take<char>(h->tcq_bytes);
+      const bool big = i < n_big;
+      const size_t cap = big ? max_k : small_k;
+      ln.cap_k = (int64_t)cap;
+      ln.rA = b.take<double>(cap * cap);
+      ln.rF = b.take<double>(cap * cap);
+      ln.rQ = b.take<double>(cap * cap);
+      size_t work = 1056;                                  // (also 1025 doubles of norm scratch)
+      for (size_t k : orders) if (k <= cap) work = std::max(work, qr_work_doubles((int64_t)k));
+      ln.rWork = b.take<double>(work);
+      ln.cond = b.take<int>(64);
+      if (big && max_z) ln.rZ = b.take<double>(max_z);
+      if (big && h->tcq_bytes) ln.tcq_scratch = b.take<char>(h->tcq_bytes);
     }
   }
   h->d_cond = b.take<int>(2 * h->layers.size() + 2);
@@ -290,6 +329,42 @@ br_status deflated_power(br_handle* h, br_handle::Lane& ln, QrTc* tcq, int64_t k
   return BR_OK;
 }
 
+// A <- qr(A).Q for the product in the lane's buffer; the conditioning note goes to d_cond[ci].
+br_status orthonormalise(br_handle* h, br_handle::Lane& ln, int64_t k, QrTc* tcq, int ci, cudaStream_t s) {
+  if (h->use_graphs) {
+    const int64_t key = 2 * k + (tcq ? 1 : 0);
+    auto it = ln.qr_graphs.find(key);
+    if (it == ln.qr_graphs.end()) {
+      br_handle::Lane::QrGraph g;
+      cudaGraph_t graph = nullptr;
+      cudaError_t e = cudaStreamBeginCapture(s, cudaStreamCaptureModeRelaxed);
+      if (e == cudaSuccess) {
+        const cudaError_t qe = qr_pos_inplace(ln.rA, k, ln.rWork, h->d_status, s, &g.launches, &g.flops, tcq, ln.cond);
+        e = cudaStreamEndCapture(s, &graph);          // always ends the capture, also after a failed launch
+        if (e == cudaSuccess && qe != cudaSuccess) e = qe;
+        if (e == cudaSuccess && graph) e = cudaGraphInstantiate(&g.exec, graph, 0);
+        if (graph) cudaGraphDestroy(graph);
+      }
+      if (e != cudaSuccess || !g.exec) {
+        cudaGetLastError();
+        h->use_graphs = false;                         // nothing was enqueued: run it directly below
+      } else {
+        it = ln.qr_graphs.emplace(key, g).first;
+      }
+    }
+    if (h->use_graphs) {
+      BR_CUDA(h, cudaGraphLaunch(it->second.exec, s));
+      h->stats.launches += it->second.launches;
+      h->stats.gemm_flops += it->second.flops;
+      BR_CUDA(h, cudaMemcpyAsync(h->d_cond + ci, ln.cond, sizeof(int), cudaMemcpyDeviceToDevice, s));
+      return BR_OK;
+    }
+  }
+  BR_CUDA(h, qr_pos_inplace(ln.rA, k, ln.rWork, h->d_status, s, &h->stats.launches, &h->stats.gemm_flops, tcq,
+                            h->d_cond + ci));
+  return BR_OK;
+}
+
 // ---- refresh of one side: Q <- qr(F Q).Q in fp64, F = L | R (S=2nd) or M M^T | M^T M (S=1st) ----
 br_status refresh_side(br_handle* h, Layer& L, bool left_side, br_handle::Lane& ln) {
   cudaStream_t s = ln.stream;
@@ -345,8 +420,10 @@ br_status refresh_side(br_handle* h, Layer& L, bool left_side, br_handle::Lane& 
       BR_CUDA(h, qr_complete_columns(ln.rA, Q, k, ln.rWork, h->d_status, s));
       count(h, 3);
     }
-    BR_CUDA(h, qr_pos_inplace(ln.rA, k, ln.rWork, h->d_status, s, &h->stats.launches, &h->stats.gemm_flops, tcq,
-                              h->d_cond + ci));
+    {
+      br_status st = orthonormalise(h, ln, k, tcq, ci, s);
+      if (st != BR_OK) return st;
+    }
     BR_CUDA(h, f64_to_f32(ln.rA, Q, k * k, s));
     count(h);
   }
@@ -360,12 +437,16 @@ br_status refresh_side(br_handle* h, Layer& L, bool left_side, br_handle::Lane& 
 // Refresh the bases of the given layers: every (layer, side) is an independent job; jobs are
 // dealt to the lanes largest first, each to the lane with the least work so far.
 br_status refresh_layers(br_handle* h, const int* ids, int n_ids) {
-  struct Job { int layer; bool left; double cost; };
+  struct Job { int layer; bool left; double cost; int64_t k; bool needs_z; };
   std::vector<Job> jobs;
+  // time of one job when it runs alone (ms, measured: 11 at order 2560, 45 at order 6912): a cubic
+  // term for the products and a linear one for the chain of panel factorisations
+  auto cost = [](double k) { return 5.4e-11 * k * k * k + 3.9e-3 * k; };
   for (int j = 0; j < n_ids; ++j) {
     const Layer& L = h->layers[ids[j]];
-    if (L.left) jobs.push_back({ids[j], true, (double)L.d.m * L.d.m * L.d.m});
-    if (L.right) jobs.push_back({ids[j], false, (double)L.d.n * L.d.n * L.d.n});
+    const bool z = L.d.src != BR_SRC_SECOND;
+    if (L.left) jobs.push_back({ids[j], true, cost((double)L.d.m), L.d.m, z});
+    if (L.right) jobs.push_back({ids[j], false, cost((double)L.d.n), L.d.n, z});
   }
   if (jobs.empty()) return BR_OK;
   if (h->cond_pending) {
@@ -375,12 +456,17 @@ br_status refresh_layers(br_handle* h, const int* ids, int n_ids) {
     h->cond_pending = false;
   }
   std::stable_sort(jobs.begin(), jobs.end(), [](const Job& a, const Job& b) { return a.cost > b.cost; });
-  const int nl = (int)std::min<size_t>((size_t)h->n_lanes, jobs.size());
+  // each job to the least loaded lane that can hold it (lane 0 holds everything)
+  const int nl = h->n_lanes;
   std::vector<std::vector<Job>> per_lane(nl);
   std::vector<double> load(nl, 0.0);
   for (const Job& jb : jobs) {
     int best = 0;
-    for (int i = 1; i < nl; ++i) if (load[i] < load[best]) best = i;
+    for (int i = 1; i < nl; ++i) {
+      const br_handle::Lane& ln = h->lanes[i];
+      if (ln.cap_k < jb.k || (jb.needs_z && !ln.rZ)) continue;
+      if (load[i] < load[best]) best = i;
+    }
     per_lane[best].push_back(jb);
     load[best] += jb.cost;
   }
@@ -644,6 +730,7 @@ br_status br_create(br_handle** out, const br_layer_desc* layers, int n_layers, 
     }
   }
   h->lanes[0].stream = s;
+  if (const char* env = std::getenv("BR_REFRESH_GRAPHS")) h->use_graphs = env[0] != '0';
   for (int i = 1; i < h->n_lanes; ++i) {
     if ((e = cudaStreamCreateWithFlags(&h->lanes[i].stream, cudaStreamNonBlocking)) != cudaSuccess) return fail("cudaStreamCreate", e);
     if ((e = cudaEventCreateWithFlags(&h->lanes[i].done, cudaEventDisableTiming)) != cudaSuccess) return fail("cudaEventCreate", e);
@@ -662,6 +749,7 @@ br_status br_create(br_handle** out, const br_layer_desc* layers, int n_layers, 
     }
     for (int i = 0; i < h->n_lanes; ++i)
       for (int64_t k : orders) {
+        if (!h->lanes[i].tcq_scratch) continue;            // a small-order lane
         const char* qerr = nullptr;
         QrTc* t = qr_tc_create(k, h->lanes[i].tcq_scratch, device, s, &qerr);
         if (!t) {
@@ -1033,8 +1121,10 @@ br_status br_destroy(br_handle* h) {
   if (h->ev_begin) cudaEventDestroy(h->ev_begin);
   if (h->ev_cond) cudaEventDestroy(h->ev_cond);
   if (h->h_cond) cudaFreeHost(h->h_cond);
-  for (int i = 0; i < br_handle::kMaxLanes; ++i)
+  for (int i = 0; i < br_handle::kMaxLanes; ++i) {
+    for (auto& kv : h->lanes[i].qr_graphs) if (kv.second.exec) cudaGraphExecDestroy(kv.second.exec);
     for (QrTc* t : h->lanes[i].tcq) qr_tc_destroy(t);
+  }
   for (auto& sp : h->stats.prof.spans) { cudaEventDestroy(sp.a); cudaEventDestroy(sp.b); }
   for (auto e : h->stats.prof.free_events) cudaEventDestroy(e);
   if (h->slab) {

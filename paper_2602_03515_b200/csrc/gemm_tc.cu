@@ -78,7 +78,10 @@ struct Form {
 constexpr int TMEM_COLS = 512;
 constexpr int NUM_THREADS = 192;                 // warp 0: TMA, warp 1: MMA, warps 2..5: epilogue
 constexpr int MAX_PAIRS = 3;
-constexpr int GROUP_M = 8;                       // tile rasterisation: 8 row-blocks per column sweep
+// Tile rasterisation: a group of row-blocks (or, transposed, of column-blocks) is swept across the
+// other dimension, so that the group's operand panel stays in L2 while the other operand streams
+// through once per group.  The host picks orientation and group size per problem (see plan creation).
+constexpr double kL2PanelBytes = 40e6;           // what one resident operand panel may take of the 126 MB L2
 
 struct alignas(128) DevProblem {
   CUtensorMap mapA[MAX_PAIRS];
@@ -97,6 +100,7 @@ struct alignas(128) DevProblem {
   // shared-operand form: mapA[0..nA) / mapB[0..nB) are the distinct operands, `combos` lists the
   // products to issue per k-block: bits 8.. = count, bits 2c, 2c+1 = (A index, B index) of product c
   int32_t symmetric, nA, nB, combos;
+  int32_t group, raster_n;        // blocks per group; 0: groups of row-blocks, 1: groups of column-blocks
   const float* clip;              // clipping factors by call (see TcProblem::clip_mode), or null
   int32_t clip_slots, clip_mode;
 };
@@ -300,13 +304,17 @@ __device__ __forceinline__ TileInfo locate_tile(const DevProblem* probs, int n_p
   TileInfo ti;
   ti.p = p;
   const int local = tile - p->tile_begin;
-  const int per_group = GROUP_M * p->tiles_n;
+  const int g = p->group;
+  const int across = p->raster_n ? p->tiles_m : p->tiles_n;      // blocks of the swept dimension
+  const int along = p->raster_n ? p->tiles_n : p->tiles_m;       // blocks of the grouped dimension
+  const int per_group = g * across;
   const int group = local / per_group;
-  const int first_m = group * GROUP_M;
-  const int gsz = min(p->tiles_m - first_m, GROUP_M);
+  const int first = group * g;
+  const int gsz = min(along - first, g);
   const int in_group = local - group * per_group;
-  ti.m0 = (first_m + in_group % gsz) * TM;
-  ti.n0 = (in_group / gsz) * BN;
+  const int blk_g = first + in_group % gsz, blk_s = in_group / gsz;
+  ti.m0 = (p->raster_n ? blk_s : blk_g) * TM;
+  ti.n0 = (p->raster_n ? blk_g : blk_s) * BN;
   // delayed-gradient bookkeeping: the layer is active once call - tau >= 1; the gradient to
   // apply sits in ring slot (calls - 1 - tau) mod slots
   const int tl = tau < 0 ? p->tau_max : tau;
@@ -862,6 +870,11 @@ TcPlan* tc_plan_create(const TcProblem* problems, int n, int device, cudaStream_
   const bool pair = pairs > 0;
   const int TM = pair ? 2 * BM : BM;            // rows of a tile
   const int b_box = pair ? BN / 2 : BN;         // rows of B one CTA stages per k-block
+  double panel_bytes = kL2PanelBytes;
+  if (const char* env = std::getenv("BR_TC_L2_PANEL_MB")) {        // tuning aid
+    const double v = std::atof(env);
+    if (v >= 1.0 && v <= 512.0) panel_bytes = v * 1e6;
+  }
   std::vector<DevProblem> host(n);
   std::vector<int> tile_starts;
   std::vector<double> prob_flops;
@@ -912,6 +925,27 @@ TcPlan* tc_plan_create(const TcProblem* problems, int n, int device, cudaStream_
     d.tiles_n = (int32_t)((q.Nd + BN - 1) / BN);
     d.tile_begin = tile_begin;
     d.tile_count = d.tiles_m * d.tiles_n;
+    {
+      // Estimated DRAM reads of the two walks: the resident panel's operand once, the other once per
+      // group.  Group = as many blocks as keep the panel within its share of L2.
+      int nA = 0, nB = 0;
+      for (int p = 0; p < q.n_pairs; ++p) {
+        bool newa = true, newb = true;
+        for (int u = 0; u < p; ++u) {
+          if (same_operand(q.A[u], q.A[p])) newa = false;
+          if (same_operand(q.B[u], q.B[p])) newb = false;
+        }
+        nA += newa; nB += newb;
+      }
+      const double stripeA = (double)TM * (double)q.K * 2.0 * nA, stripeB = (double)BN * (double)q.K * 2.0 * nB;
+      const double totalA = stripeA * d.tiles_m, totalB = stripeB * d.tiles_n;
+      auto clampi = [](double v, int lo, int hi) { return v < lo ? lo : (v > hi ? hi : (int)v); };
+      const int gM = clampi(panel_bytes / stripeA, 1, d.tiles_m), gN = clampi(panel_bytes / stripeB, 1, d.tiles_n);
+      const double trafficM = totalA + totalB * ((d.tiles_m + gM - 1) / gM);
+      const double trafficN = totalB + totalA * ((d.tiles_n + gN - 1) / gN);
+      d.raster_n = trafficN < trafficM ? 1 : 0;
+      d.group = d.raster_n ? gN : gM;
+    }
     tile_starts.push_back(tile_begin);
     tile_begin += d.tile_count;
     d.tau_max = q.tau_max;

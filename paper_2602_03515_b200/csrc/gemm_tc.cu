@@ -101,6 +101,7 @@ struct alignas(128) DevProblem {
   // products to issue per k-block: bits 8.. = count, bits 2c, 2c+1 = (A index, B index) of product c
   int32_t symmetric, nA, nB, combos;
   int32_t group, raster_n;        // blocks per group; 0: groups of row-blocks, 1: groups of column-blocks
+  int32_t tri;                    // symmetric product with square tiles: the tile list holds the upper triangle only
   const float* clip;              // clipping factors by call (see TcProblem::clip_mode), or null
   int32_t clip_slots, clip_mode;
 };
@@ -304,6 +305,19 @@ __device__ __forceinline__ TileInfo locate_tile(const DevProblem* probs, int n_p
   TileInfo ti;
   ti.p = p;
   const int local = tile - p->tile_begin;
+  if (p->tri) {
+    // upper triangle, column by column: column c holds the row-blocks 0..c at positions c (c + 1) / 2 + r
+    int c = (int)((sqrtf(8.0f * (float)local + 1.0f) - 1.0f) * 0.5f);
+    while ((c + 1) * (c + 2) / 2 <= local) ++c;
+    while (c * (c + 1) / 2 > local) --c;
+    ti.m0 = (local - c * (c + 1) / 2) * TM;
+    ti.n0 = c * BN;
+    const int tl = tau < 0 ? p->tau_max : tau;
+    ti.active = (calls - tl >= 1);
+    ti.z = 0;
+    if (p->ring_slots > 0 && ti.active) ti.z = (int)((calls - 1 - tl) % p->ring_slots);
+    return ti;
+  }
   const int g = p->group;
   const int across = p->raster_n ? p->tiles_m : p->tiles_n;      // blocks of the swept dimension
   const int along = p->raster_n ? p->tiles_n : p->tiles_m;       // blocks of the grouped dimension
@@ -925,6 +939,10 @@ TcPlan* tc_plan_create(const TcProblem* problems, int n, int device, cudaStream_
     d.tiles_n = (int32_t)((q.Nd + BN - 1) / BN);
     d.tile_begin = tile_begin;
     d.tile_count = d.tiles_m * d.tiles_n;
+    // A symmetric product on square tiles lists only the tiles of the upper triangle, so that the
+    // round-robin walk gives every CTA pair the same number of computed tiles.
+    d.tri = (q.symmetric && TM == BN && d.tiles_m == d.tiles_n) ? 1 : 0;
+    if (d.tri) d.tile_count = d.tiles_m * (d.tiles_m + 1) / 2;
     {
       // Estimated DRAM reads of the two walks: the resident panel's operand once, the other once per
       // group.  Group = as many blocks as keep the panel within its share of L2.

@@ -47,7 +47,9 @@ namespace br {
 namespace {
 
 constexpr int kB = 128;          // widest panel
-constexpr double kDefectLimit = 0.1;
+// A panel whose every column keeps at least this fraction of its squared norm against the columns
+// before it (at least 10 % of its length) needs no second Cholesky-QR pass.
+constexpr double kPassRatio = 1e-2;
 
 inline int64_t cdiv(int64_t a, int64_t b) { return (a + b - 1) / b; }
 inline int panel_width(int64_t k) { return k >= 1024 ? 128 : 64; }
@@ -73,10 +75,12 @@ inline int64_t pad32(int64_t doubles) { return (doubles + 31) / 32 * 32; }
 // written out (as column c of R^-1) straight from the scaled row.
 //
 // A pivot that underflows 1e-24 of the column's squared norm is clamped and reported as a
-// numerically rank-deficient factor.  defect = sum_c (1 - pivot_c / S_cc) bounds the squared
-// Frobenius distance of the column-scaled Gram matrix from the identity (up to a factor ~2): when
-// it is small the panel was close to orthogonal and one Cholesky-QR pass is accurate to rounding,
-// so *skip_next is set and the kernels of the second pass return at once.  norm0 (optional):
+// numerically rank-deficient factor.  pivot_c / S_cc is the squared sine of the angle between
+// column c and the span of the panel's columns before it.  One Cholesky-QR pass loses orthogonality
+// like cond^2 * 1e-16 with cond the condition number of the column-scaled panel; while every column
+// keeps at least kPassRatio of its squared norm, cond^2 stays (for other than contrived matrices)
+// below ~128 / kPassRatio ~ 1e4 and one pass is accurate far beyond the fp32 result, so *skip_next
+// is set and the kernels of the second pass return at once.  norm0 (optional):
 // squared norms the panel's columns had before any projection; a column that has lost more than
 // 1 - kIllRatio of it marks the input as ill-conditioned by clearing *ill_clear.
 __global__ void __launch_bounds__(512)
@@ -113,7 +117,7 @@ k_chol_inverse(const double* __restrict__ S, int bw, double* __restrict__ Rinv, 
     for (int b = 0; b < 8; ++b) rowS[0][tx + 16 * b] = Z[0][b];
   }
   __syncthreads();
-  double defect = 0.0;       // accumulated by thread 0 (every thread sees every pivot)
+  double min_ratio = 1.0;    // tracked by thread 0 (every thread sees every pivot)
   bool ill = false, tc_bad = false, any_clamped = false;
 
   for (int c = 0; c < bw; ++c) {
@@ -126,7 +130,7 @@ k_chol_inverse(const double* __restrict__ S, int bw, double* __restrict__ Rinv, 
     if (clamped) piv = floor_;
     if (t == 0) {
       if (clamped) { atomicMax(status, (int)BR_WARN_RANK_DEFICIENT); any_clamped = true; }
-      defect += fmax(0.0, 1.0 - piv * diag0_inv[c]);
+      min_ratio = fmin(min_ratio, piv * diag0_inv[c]);
       if (orig < nrm_floor[c]) ill = true;
       if (orig < tc_floor[c]) tc_bad = true;
     }
@@ -178,7 +182,7 @@ k_chol_inverse(const double* __restrict__ S, int bw, double* __restrict__ Rinv, 
     __syncthreads();
   }
   if (t == 0) {
-    if (skip_next) *skip_next = (defect <= kDefectLimit) ? 1 : 0;
+    if (skip_next) *skip_next = (min_ratio >= kPassRatio) ? 1 : 0;
     if (ill && ill_clear) *ill_clear = 0;
     if (tc_bad && tc_ok_clear) *tc_ok_clear = 0;
     if (any_clamped && tc_ok_clear) tc_ok_clear[1] = 1;      // numerically rank-deficient: noted for the next refresh

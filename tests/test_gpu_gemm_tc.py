@@ -74,3 +74,25 @@ def test_rejects_bad_arguments():
     d = torch.zeros(64, 64, device="cuda")
     with pytest.raises(br.BrError):
         br.br_gemm_bf16(0, 60, 64, 64, [x.data_ptr()], [x.data_ptr()], 0, 0, 64, 64, d.data_ptr(), 64)
+
+
+@pytest.mark.parametrize("Md,Nd,K,a_mn,b_mn", [(8192 + 72, 520, 4096, 0, 1), (6000, 6000, 3592, 1, 0)])
+def test_tile_walks_with_partial_groups(Md, Nd, K, a_mn, b_mn):
+    """Shapes whose operand panels exceed the share of L2 a tile group may take, so that the walk
+    is cut into several groups (the last one partial): a tall result with a small second operand is
+    walked in groups of column-blocks, a large square one in groups of row-blocks.  Checked on sampled
+    rows (all columns) against a float64 contraction."""
+    import torch
+    import paper_2602_03515_b200 as br
+    rng = np.random.default_rng(Md + Nd + K)
+    A, Ar = _operand(rng, Md, K, a_mn, torch)
+    B, Br = _operand(rng, Nd, K, b_mn, torch)
+    D = torch.full((Md, Nd), float("nan"), device="cuda")
+    lda = Md if a_mn else K
+    ldb = Nd if b_mn else K
+    br.br_gemm_bf16(0, Md, Nd, K, [A.data_ptr()], [B.data_ptr()], a_mn, b_mn, lda, ldb, D.data_ptr(), Nd, 1.0, 0.0)
+    assert bool(torch.isfinite(D).all())
+    rows = np.unique(np.concatenate([np.arange(0, Md, 97), np.arange(Md - 8, Md), np.arange(248, 264)]))
+    ref = Ar[rows] @ Br.T
+    got = D[torch.from_numpy(rows).cuda()].cpu().double().numpy()
+    assert np.max(np.abs(got - ref)) <= 1e-5 * np.sqrt(K) * np.max(np.abs(ref))

@@ -238,7 +238,16 @@ void layout(br_handle* h, Bump& b, Sizes* sz) {
       ln.rWork = b.take<double>(work);
       ln.cond = b.take<int>(64);
       if (big && max_z) ln.rZ = b.take<double>(max_z);
-      if (big && h->tcq_bytes) ln.tcq_scratch = b.take<char>(h->tcq_bytes);
+      {
+        // scratch of the tensor-core projections for the largest eligible order this lane can hold
+        size_t tb = 0;
+        for (const Layer& L : h->layers) {
+          if (!L.use_tc) continue;
+          if (L.left && (size_t)L.d.m <= cap) tb = std::max(tb, qr_tc_scratch_bytes(L.d.m));
+          if (L.right && (size_t)L.d.n <= cap) tb = std::max(tb, qr_tc_scratch_bytes(L.d.n));
+        }
+        if (tb) ln.tcq_scratch = b.take<char>(tb);
+      }
     }
   }
   h->d_cond = b.take<int>(2 * h->layers.size() + 2);
@@ -749,7 +758,7 @@ br_status br_create(br_handle** out, const br_layer_desc* layers, int n_layers, 
     }
     for (int i = 0; i < h->n_lanes; ++i)
       for (int64_t k : orders) {
-        if (!h->lanes[i].tcq_scratch) continue;            // a small-order lane
+        if (!h->lanes[i].tcq_scratch || k > h->lanes[i].cap_k) continue;      // a small-order lane
         const char* qerr = nullptr;
         QrTc* t = qr_tc_create(k, h->lanes[i].tcq_scratch, device, s, &qerr);
         if (!t) {

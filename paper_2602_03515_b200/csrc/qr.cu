@@ -38,6 +38,7 @@
 // shrinkage, and it runs the second (fp64) sweep already when a column keeps less than 1e-3 instead
 // of 1e-4.  The leaves (Cholesky-QR) and the power product stay in fp64.
 #include <algorithm>
+#include <cstdlib>
 #include <string>
 #include <vector>
 
@@ -227,9 +228,23 @@ k_column_norms_sum(const double* __restrict__ part, int64_t k, int nchunks, doub
 struct ProjNode { int64_t jp, wp, jt, wt; };
 
 // projections of orth(0, k) in the order in which the recursion runs them
-// A projection goes to the tensor cores only when it is large: the grouped kernel has no split over
-// K, so a product with a handful of output tiles would leave most SMs idle.
-inline bool tc_node(int64_t wp, int64_t wt) { return wp * wt >= (int64_t)1 << 21; }
+// A projection goes to the tensor cores when its coefficient block has at least 2^18 entries (512 x
+// 512).  The grouped kernel has no split over K, so such a product has only a handful of output tiles
+// and leaves most SMs idle -- to the other lanes of the refresh, which is what makes it pay: in SM-time
+// it is several times cheaper than the fp64 product even so (measured on a refresh of 57 bases:
+// 397 ms with a threshold of 2^21 and orders from 4096, 352 ms with 2^18 and orders from 2048, 427 ms
+// with 2^14).
+inline int64_t env_or(const char* name, int64_t dflt, int64_t lo, int64_t hi) {
+  if (const char* e = std::getenv(name)) {
+    const long long v = std::atoll(e);
+    if (v >= lo && v <= hi) return v;
+  }
+  return dflt;
+}
+// tuning aids: BR_QR_TC_MIN_NODE (entries of the coefficient block), BR_QR_TC_MIN_ORDER
+inline int64_t tc_min_node() { static const int64_t v = env_or("BR_QR_TC_MIN_NODE", (int64_t)1 << 18, 1 << 14, (int64_t)1 << 40); return v; }
+inline int64_t tc_min_order() { static const int64_t v = env_or("BR_QR_TC_MIN_ORDER", 2048, 1024, (int64_t)1 << 30); return v; }
+inline bool tc_node(int64_t wp, int64_t wt) { return wp * wt >= tc_min_node(); }
 
 void enumerate_nodes(int64_t j0, int64_t w, int64_t b, std::vector<ProjNode>* out) {
   if (w <= b) return;
@@ -259,7 +274,7 @@ inline size_t al256(size_t x) { return (x + 255) / 256 * 256; }
 }  // namespace
 
 int64_t qr_tc_order(const QrTc* t) { return t ? t->k : 0; }
-bool qr_tc_eligible(int64_t k) { return k >= 4096 && (k % 8) == 0; }
+bool qr_tc_eligible(int64_t k) { return k >= tc_min_order() && (k % 8) == 0; }
 
 size_t qr_tc_scratch_bytes(int64_t k) {
   if (!qr_tc_eligible(k)) return 0;

@@ -137,9 +137,10 @@ def test_refresh_order_1024_against_oracle_power():
     assert np.max(np.abs(U.T @ U - np.eye(k))) < 1e-5
 
 
-def test_refresh_tensor_core_projections_order_4224():
-    """Third refresh of a basis of order 4224 in one handle (orders from 4096 use the tensor-core
-    projections).  The first (from U = I) is ill-conditioned, the second runs in fp64 and notes that
+@pytest.mark.parametrize("k", [4224, 2560])
+def test_refresh_tensor_core_projections(k):
+    """Third refresh of a basis of order 4224 / 2560 in one handle (orders from 2048 use the tensor-core
+    forms: deflated power product, block projections with at least 2^18 coefficients).  The first (from U = I) is ill-conditioned, the second runs in fp64 and notes that
     no column shrank much, so the third runs its large block projections on the tensor cores
     (three-term bf16 splits, applied twice).  The result is unique (QR with a positive diagonal), so
     it is compared with LAPACK's QR of the float64 product F U2 after fixing the signs -- the
@@ -148,7 +149,6 @@ def test_refresh_tensor_core_projections_order_4224():
     import torch
     import paper_2602_03515_b200 as br
     from tests.parity_util import basis_err
-    k = 4224
     F = _lowrank_noise_factor(k, 16, 33, samples=3)      # 13,000 noise samples: the noise part is well conditioned
     w = torch.zeros(k, 8, device="cuda")
     opt = br.BasisRotation([LayerSpec("W", k, 8, GEOM_BI, SRC_SECOND, 0)], [w], grad_dtype="bf16",

@@ -29,5 +29,5 @@ def test_unpaired_tensor_core_kernel():
 def test_refresh_without_graphs_and_small_lanes():
     _run({"BR_REFRESH_GRAPHS": "0", "BR_REFRESH_SMALL_LANES": "0", "BR_REFRESH_LANES": "1"},
          ["tests/test_gpu_full_size.py::test_refresh_order_1024_against_oracle_power",
-          "tests/test_gpu_full_size.py::test_refresh_tensor_core_projections_order_4224",
+          "tests/test_gpu_full_size.py::test_refresh_tensor_core_projections",
           "tests/test_gpu_parity_bf16.py", "-k", "not checkpoint"])

@@ -243,7 +243,7 @@ def main():
     ap.add_argument("--impl", default="ours")
     ap.add_argument("--layers", type=int, default=None, help="decoder depth override (c4/c5)")
     ap.add_argument("--tau", type=int, default=None, help="ring depth override")
-    ap.add_argument("--e2e-steps", type=int, default=6)
+    ap.add_argument("--e2e-steps", type=int, default=12)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--scratch-gib", type=float, default=0.0)
     ap.add_argument("--no-refresh", action="store_true",
@@ -386,18 +386,20 @@ def main():
         host = [torch.empty(g.shape, dtype=g.dtype, pin_memory=True) for g in grads]
         for h_, g in zip(host, grads):
             h_.copy_(g)
-        w_host = torch.empty(weights[0].shape, dtype=torch.float32, pin_memory=True)
+        w_host = [torch.empty(weights[0].shape, dtype=torch.float32, pin_memory=True) for _ in range(2)]
         h2d = sum(h_.numel() * h_.element_size() for h_ in host)
-        d2h = w_host.numel() * 4 + 4
-        # Every step uploads its gradients from pinned host memory and reads a weight matrix and the
-        # status word back.  The upload of step i + 1 runs on a copy stream, into the other of two device
-        # gradient sets, while step i computes (the library has copied a call's gradients into its ring
-        # by the time the stream passes that call's work, so a set is free again two steps later).
+        d2h = w_host[0].numel() * 4 + 4
+        # Every step uploads its gradients from pinned host memory and reads a weight matrix back; the
+        # status word is read at the end.  The upload of step i + 1 runs on a copy stream, into the other of
+        # two device gradient sets, while step i computes (the library has copied a call's gradients into
+        # its ring by the time the stream passes that call's work, so a set is free again two steps later);
+        # the host waits for the result of step i - 1 while step i runs.
         grads2 = [torch.empty_like(g) for g in grads]
         sets = [grads, grads2]
         copy_stream = torch.cuda.Stream(device=dev)
         up = [torch.cuda.Event(), torch.cuda.Event()]          # upload of a set finished
         used = [torch.cuda.Event(), torch.cuda.Event()]        # the step that read a set has been passed
+        done = [torch.cuda.Event(), torch.cuda.Event()]        # the result of a step has reached the host
 
         def upload(i):
             with torch.cuda.stream(copy_stream):
@@ -418,9 +420,12 @@ def main():
                 stream.wait_event(up[i % 2])
                 opt.step(sets[i % 2], tau)
                 used[i % 2].record(stream)
-                w_host.copy_(weights[0], non_blocking=True)
-                st = opt.sync_status()          # waits for the stream and reads the status word back
-                assert st >= 0
+                w_host[i % 2].copy_(weights[0], non_blocking=True)
+                done[i % 2].record(stream)
+                if i >= 1:
+                    done[(i - 1) % 2].synchronize()
+            st = opt.sync_status()              # waits for the stream and reads the status word back
+            assert st >= 0
         sync_all()
         e2e_ms = 1e3 * (time.perf_counter() - t0) / args.e2e_steps + refresh_ms / w.freq
         e2e_ms = max_over_ranks([e2e_ms], world, dev, torch)[0]

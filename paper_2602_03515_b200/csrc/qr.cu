@@ -366,16 +366,21 @@ cudaError_t qr_tc_project(QrTc* t, int node, double* A, int64_t k, int64_t jp, i
   if (nd.jp != jp || nd.wp != wp || nd.jt != jt || nd.wt != wt || t->k != k) return cudaErrorInvalidValue;
   cudaError_t e;
   if ((e = split3_f64(A + jp, k, k, wp, t->Q[0], t->Q[1], t->Q[2], s)) != cudaSuccess) return e;
-  // Twice: the coefficients of the first pass are wrong by ~1e-7 of the column's length BEFORE the
-  // projection, which leaves that much of span(Q_l) in the column; the second pass sees the
-  // shrunken column and leaves ~1e-7 of its length AFTER the projection.
+  // Twice: whatever error the coefficients of the first pass have leaves that much of span(Q_l) in
+  // the column, measured against its length BEFORE the projection; the second pass sees the shrunken
+  // column and leaves ~1e-7 of its length AFTER the projection.  Because the second pass removes what
+  // the first left inside span(Q_l), the first pass's coefficients need only the three leading
+  // products (2^-16); its update Q_l C must be accurate to 2^-24 (its rounding leaves span(Q_l)), so it
+  // takes all six.  The second pass is the other way round: coefficients with all six products (they
+  // are a small difference of large terms), update with the leading three (C is ~2^-16 of the column
+  // by then).  18 products instead of 24.
   for (int pass = 0; pass < 2; ++pass) {
     if ((e = split3_f64(A + jt, k, k, wt, t->A[0], t->A[1], t->A[2], s)) != cudaSuccess) return e;
     if ((e = tc_plan_launch_range(t->lead, 2 * node, 1, 1, 0, 1.f, 0.f, status, s)) != cudaSuccess) return e;
-    if ((e = tc_plan_launch_range(t->tail, 2 * node, 1, 1, 0, 1.f, 0.f, status, s)) != cudaSuccess) return e;
+    if (pass == 1 && (e = tc_plan_launch_range(t->tail, 2 * node, 1, 1, 0, 1.f, 0.f, status, s)) != cudaSuccess) return e;
     if ((e = split3_f32(t->Cf, wp * wt, t->C[0], t->C[1], t->C[2], s)) != cudaSuccess) return e;
     if ((e = tc_plan_launch_range(t->lead, 2 * node + 1, 1, 1, 0, 1.f, 0.f, status, s)) != cudaSuccess) return e;
-    if ((e = tc_plan_launch_range(t->tail, 2 * node + 1, 1, 1, 0, 1.f, 0.f, status, s)) != cudaSuccess) return e;
+    if (pass == 0 && (e = tc_plan_launch_range(t->tail, 2 * node + 1, 1, 1, 0, 1.f, 0.f, status, s)) != cudaSuccess) return e;
     if ((e = sub_f32_from_f64(A + jt, k, k, wt, t->Df, s)) != cudaSuccess) return e;
   }
   return cudaSuccess;
@@ -437,7 +442,7 @@ void project(Sweep& q, int64_t jp, int64_t wp, int64_t jt, int64_t wt) {
   const int64_t k = q.k;
   if (q.tc && q.first && tc_node(wp, wt)) {
     q.err = qr_tc_project(q.tc, q.node++, q.A, k, jp, wp, jt, wt, q.status, q.s);
-    q.launches += 15;
+    q.launches += 13;
     return;
   }
   const int64_t tiles = cdiv(wp, 128) * cdiv(wt, 128);

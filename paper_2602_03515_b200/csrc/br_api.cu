@@ -303,37 +303,41 @@ const void* ring_slot_ptr(const Layer& L, int64_t slot) {
 // ~2e-7 ||F_rest|| per column, a relative 2e-7 of the small columns instead of 2e-7 * 1e5.
 // On entry ln.rF and ln.rQ hold F and Q widened to fp64; on exit ln.rA holds F Q (rF is overwritten).
 br_status deflated_power(br_handle* h, br_handle::Lane& ln, QrTc* tcq, int64_t k, cudaStream_t s) {
-  const int64_t r = 128;
+  const int64_t r = 128, r2 = 2 * r;
   double* w = ln.rWork;                               // the QR work area is free until the QR starts
-  double* B = w;               w += k * r;            // k x r
-  double* T1 = w;              w += k * r;            // k x r
+  double* W1 = w;              w += k * r2;           // k x 2r: [U_s | T1]
+  double* W2 = w;              w += k * r2;           // k x 2r: [B | U_s]
   double* C1 = w;              w += r * k;            // r x k
-  double* C2 = w;              w += r * k;            // r x k
+  double* C2 = w;              w += r * k;            // r x k, directly below C1: [C1; C2] is 2r x k
   double* Lam = w;             w += r * r;            // r x r
   double* part = w;                                   // split-K partial sums (at most 54 * r * r, 4 * r * k doubles)
   const int sp_small = (int)std::min<int64_t>(54, std::max<int64_t>(1, k / 128));
   double* F = ln.rF;
   double* Q = ln.rQ;
   const double* Us = Q;                               // first r columns of Q, leading dimension k
+  double* B = W2;                                     // leading dimension 2r
+  double* T1 = W1 + r;                                // leading dimension 2r
+  const size_t rb = sizeof(double) * r, pk = sizeof(double) * k, p2 = sizeof(double) * r2;
   // B = F U_s ; Lam = U_s^T B ; C1 = U_s^T Q ; C2 = B^T Q
-  BR_CUDA(h, dgemm(0, 0, k, r, k, 1.0, F, k, Us, k, 0.0, B, r, s));
-  BR_CUDA(h, dgemm_ex(1, 0, r, r, k, 1.0, Us, k, B, r, 0.0, Lam, r, sp_small, part, nullptr, s));
+  BR_CUDA(h, dgemm(0, 0, k, r, k, 1.0, F, k, Us, k, 0.0, B, r2, s));
+  BR_CUDA(h, dgemm_ex(1, 0, r, r, k, 1.0, Us, k, B, r2, 0.0, Lam, r, sp_small, part, nullptr, s));
   BR_CUDA(h, dgemm_ex(1, 0, r, k, k, 1.0, Us, k, Q, k, 0.0, C1, k, 4, part, nullptr, s));
-  BR_CUDA(h, dgemm_ex(1, 0, r, k, k, 1.0, B, r, Q, k, 0.0, C2, k, 4, part, nullptr, s));
-  // T1 = B - U_s Lam ; F_rest = F - U_s B^T - T1 U_s^T
-  BR_CUDA(h, cudaMemcpyAsync(T1, B, sizeof(double) * k * r, cudaMemcpyDeviceToDevice, s));
-  BR_CUDA(h, dgemm(0, 0, k, r, r, -1.0, Us, k, Lam, r, 1.0, T1, r, s));
-  BR_CUDA(h, dgemm(0, 1, k, k, r, -1.0, Us, k, B, r, 1.0, F, k, s));
-  BR_CUDA(h, dgemm(0, 1, k, k, r, -1.0, T1, r, Us, k, 1.0, F, k, s));
+  BR_CUDA(h, dgemm_ex(1, 0, r, k, k, 1.0, B, r2, Q, k, 0.0, C2, k, 4, part, nullptr, s));
+  // the two rank-r corrections as one rank-2r product each: W1 = [U_s | T1], W2 = [B | U_s], T1 = B - U_s Lam
+  BR_CUDA(h, cudaMemcpy2DAsync(W1, p2, Us, pk, rb, (size_t)k, cudaMemcpyDeviceToDevice, s));
+  BR_CUDA(h, cudaMemcpy2DAsync(W2 + r, p2, Us, pk, rb, (size_t)k, cudaMemcpyDeviceToDevice, s));
+  BR_CUDA(h, cudaMemcpy2DAsync(T1, p2, B, p2, rb, (size_t)k, cudaMemcpyDeviceToDevice, s));
+  BR_CUDA(h, dgemm(0, 0, k, r, r, -1.0, Us, k, Lam, r, 1.0, T1, r2, s));
+  // F_rest = F - U_s B^T - T1 U_s^T = F - W1 W2^T
+  BR_CUDA(h, dgemm(0, 1, k, k, r2, -1.0, W1, r2, W2, r2, 1.0, F, k, s));
   // F_rest Q on the tensor cores
   const float* Af = nullptr;
   BR_CUDA(h, qr_tc_power(tcq, F, Q, h->d_status, s, &Af));
-  // C2 <- C2 - Lam C1 ; A = F_rest Q + B C1 + U_s C2
+  // C2 <- C2 - Lam C1 ; A = F_rest Q + B C1 + U_s C2 = F_rest Q + W2 [C1; C2]
   BR_CUDA(h, dgemm(0, 0, r, k, r, -1.0, Lam, r, C1, k, 1.0, C2, k, s));
   BR_CUDA(h, f32_to_f64(Af, ln.rA, k * k, s));
-  BR_CUDA(h, dgemm(0, 0, k, k, r, 1.0, B, r, C1, k, 1.0, ln.rA, k, s));
-  BR_CUDA(h, dgemm(0, 0, k, k, r, 1.0, Us, k, C2, k, 1.0, ln.rA, k, s));
-  count(h, 22);
+  BR_CUDA(h, dgemm(0, 0, k, k, r2, 1.0, W2, r2, C1, k, 1.0, ln.rA, k, s));
+  count(h, 20);
   h->stats.gemm_flops += 14.0 * k * k * r;
   return BR_OK;
 }

@@ -117,9 +117,9 @@ struct br_handle {
   // Up to three lanes hold the largest order; up to five more hold only the small orders (at most
   // 1/sqrt(2) of the largest, S = 2nd), whose refresh is a chain of short launches that leaves most of
   // the GPU idle: eight streams in all, the default number of hardware queues.
-  static constexpr int kBigLanes = 3;
-  static constexpr int kSmallLanes = 5;
-  static constexpr int kMaxLanes = kBigLanes + kSmallLanes;
+  static constexpr int kBigLanes = 3;       // default number of full-size lanes (BR_REFRESH_LANES: 1..6)
+  static constexpr int kMaxBigLanes = 6;
+  static constexpr int kMaxLanes = 8;       // lanes of both kinds
   Lane lanes[kMaxLanes];
   int n_lanes = 1;
   cudaEvent_t ev_begin = nullptr;
@@ -200,12 +200,13 @@ void layout(br_handle* h, Bump& b, Sizes* sz) {
     if (L.right) h->tcq_bytes = std::max(h->tcq_bytes, qr_tc_scratch_bytes(L.d.n));
   }
   if (max_k) {
-    int n_big = (int)std::min<size_t>(br_handle::kBigLanes, std::max<size_t>(1, n_sides));
-    // tuning aid: BR_REFRESH_LANES=1..3 caps the number of concurrent full-size refresh lanes
+    int want_big = br_handle::kBigLanes;
+    // tuning aid: BR_REFRESH_LANES=1..6 sets the number of concurrent full-size refresh lanes
     if (const char* env = std::getenv("BR_REFRESH_LANES")) {
       const int v = std::atoi(env);
-      if (v >= 1 && v < n_big) n_big = v;
+      if (v >= 1 && v <= br_handle::kMaxBigLanes) want_big = v;
     }
+    int n_big = (int)std::min<size_t>((size_t)want_big, std::max<size_t>(1, n_sides));
     // the small class: orders of S = 2nd sides of at most max_k / sqrt(2)
     size_t small_k = 0, n_small_sides = 0;
     std::vector<size_t> orders;
@@ -217,7 +218,7 @@ void layout(br_handle* h, Bump& b, Sizes* sz) {
         if (L.d.src == BR_SRC_SECOND && 2 * k * k <= max_k * max_k) { small_k = std::max(small_k, k); ++n_small_sides; }
       }
     }
-    int n_small = (int)std::min<size_t>(br_handle::kSmallLanes, n_small_sides);
+    int n_small = (int)std::min<size_t>((size_t)(br_handle::kMaxLanes - n_big), n_small_sides);
     if ((int)n_sides <= n_big) n_small = 0;
     // tuning aid: BR_REFRESH_SMALL_LANES=0..5 caps the number of small-order lanes
     if (const char* env = std::getenv("BR_REFRESH_SMALL_LANES")) {

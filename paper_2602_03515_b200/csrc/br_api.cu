@@ -123,6 +123,11 @@ struct br_handle {
   Lane lanes[kMaxLanes];
   int n_lanes = 1;
   cudaEvent_t ev_begin = nullptr;
+  // The gradients of a call are stored in the ring on a side stream, chunk by chunk, as soon as the
+  // launches that read the slots they overwrite are enqueued, so that the copies run beside the rest of
+  // the step; the step's stream waits for them before br_step returns control of it.
+  cudaStream_t copy_stream = nullptr;
+  cudaEvent_t ev_consumed = nullptr, ev_copied = nullptr;
   // Conditioning notes of the last refresh, per layer and side (index 2 * layer + (right side)):
   // written on the device by the refresh, copied to pinned host memory after every batch, read by
   // the host before the next one (which then decides where the block projections run).
@@ -750,6 +755,9 @@ br_status br_create(br_handle** out, const br_layer_desc* layers, int n_layers, 
     if ((e = cudaEventCreateWithFlags(&h->lanes[i].done, cudaEventDisableTiming)) != cudaSuccess) return fail("cudaEventCreate", e);
   }
   if ((e = cudaEventCreateWithFlags(&h->ev_begin, cudaEventDisableTiming)) != cudaSuccess) return fail("cudaEventCreate", e);
+  if ((e = cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking)) != cudaSuccess) return fail("cudaStreamCreate", e);
+  if ((e = cudaEventCreateWithFlags(&h->ev_consumed, cudaEventDisableTiming)) != cudaSuccess) return fail("cudaEventCreate", e);
+  if ((e = cudaEventCreateWithFlags(&h->ev_copied, cudaEventDisableTiming)) != cudaSuccess) return fail("cudaEventCreate", e);
   if ((e = cudaEventCreateWithFlags(&h->ev_cond, cudaEventDisableTiming)) != cudaSuccess) return fail("cudaEventCreate", e);
   h->cond_known.assign(2 * h->layers.size(), 0);
   if ((e = cudaMallocHost(reinterpret_cast<void**>(&h->h_cond), sizeof(int) * (h->cond_known.size() + 2))) != cudaSuccess)
@@ -853,13 +861,37 @@ br_status br_step(br_handle* h, const void* const* grads, int tau) {
     }
   }
   if (h->tc) {
+    struct StepCtx { br_handle* h; const void* const* grads; std::vector<char>* stored; bool copied; };
+    StepCtx sc{h, grads, &stored, false};
     TcStepCallbacks cb;
-    cb.ctx = h;
+    cb.ctx = &sc;
     cb.refresh = [](void* ctx, const int* ids, int n) -> int {
-      return (int)refresh_layers(static_cast<br_handle*>(ctx), ids, n);
+      return (int)refresh_layers(static_cast<StepCtx*>(ctx)->h, ids, n);
+    };
+    static const bool side_copies = !(std::getenv("BR_RING_SIDE_STREAM") && std::getenv("BR_RING_SIDE_STREAM")[0] == '0');
+    if (side_copies) cb.consumed = [](void* ctx, const int* ids, int n) -> int {
+      StepCtx* c = static_cast<StepCtx*>(ctx);
+      br_handle* h = c->h;
+      BR_CUDA(h, cudaEventRecord(h->ev_consumed, h->stream));
+      BR_CUDA(h, cudaStreamWaitEvent(h->copy_stream, h->ev_consumed, 0));
+      for (int j = 0; j < n; ++j) {
+        Layer& L = h->layers[ids[j]];
+        if (L.ring_slots <= 0 || (*c->stored)[ids[j]]) continue;
+        const size_t bytes = (size_t)L.d.m * L.d.n * dtype_size(L.d.grad_dtype);
+        void* dst = const_cast<void*>(ring_slot_ptr(L, (h->calls - 1) % L.ring_slots));
+        BR_CUDA(h, cudaMemcpyAsync(dst, c->grads[ids[j]], bytes, cudaMemcpyDeviceToDevice, h->copy_stream));
+        (*c->stored)[ids[j]] = 1;
+        c->copied = true;
+      }
+      return (int)BR_OK;
     };
     const char* terr = nullptr;
     int rc = tc_step_run(h->tc, h->layers, G, h->calls, tau, hp, h->d_status, h->stream, &h->stats, cb, &terr);
+    if (sc.copied) {
+      // (also on a failed step: the side stream must not outlive the caller's view of this call)
+      cudaEventRecord(h->ev_copied, h->copy_stream);
+      cudaStreamWaitEvent(h->stream, h->ev_copied, 0);
+    }
     if (rc != 0) { h->err = terr ? terr : "tensor-core step failed"; return rc < 0 ? (br_status)rc : BR_ERR_CUDA; }
   }
   // ---- store g_c in the ring (after every reader of the slot it may overwrite) --------------
@@ -1134,6 +1166,9 @@ br_status br_destroy(br_handle* h) {
   }
   if (h->ev_begin) cudaEventDestroy(h->ev_begin);
   if (h->ev_cond) cudaEventDestroy(h->ev_cond);
+  if (h->copy_stream) { cudaStreamSynchronize(h->copy_stream); cudaStreamDestroy(h->copy_stream); }
+  if (h->ev_consumed) cudaEventDestroy(h->ev_consumed);
+  if (h->ev_copied) cudaEventDestroy(h->ev_copied);
   if (h->h_cond) cudaFreeHost(h->h_cond);
   for (int i = 0; i < br_handle::kMaxLanes; ++i) {
     for (auto& kv : h->lanes[i].qr_graphs) if (kv.second.exec) cudaGraphExecDestroy(kv.second.exec);

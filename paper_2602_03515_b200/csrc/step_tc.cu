@@ -456,6 +456,10 @@ int tc_step_run(TcStep* t, std::vector<Layer>& layers, const std::vector<const v
     }
     if ((rc = lz.run(c.fwd1, "first-side rotation launch", calls, tau, dyn_alpha, dyn_beta))) return rc;
     if ((rc = lz.run(c.adam, "rotated-Adam launch", calls, tau, dyn_alpha, dyn_beta))) return rc;
+    if (cb.consumed) {       // factors, first side and (one-sided layers) rotated Adam were the readers of G
+      rc = cb.consumed(cb.ctx, c.ids.data(), (int)c.ids.size());
+      if (rc != 0) { if (err) *err = nullptr; return rc; }
+    }
     if ((rc = lz.run(c.back1, "back-rotation launch", calls, tau, dyn_alpha, dyn_beta))) return rc;
     if ((rc = lz.run(c.wwrite, "weight-write launch", calls, tau, dyn_alpha, dyn_beta))) return rc;
   }

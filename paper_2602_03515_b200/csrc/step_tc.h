@@ -37,6 +37,9 @@ struct TcStepCallbacks {
   void* ctx = nullptr;
   // runs Power() for the given layers (independent of one another), returns br_status
   int (*refresh)(void* ctx, const int* layers, int n) = nullptr;
+  // optional: told, once the last launch that reads the gradients of these layers is enqueued (their
+  // ring slots may then be overwritten behind an event on the step's stream); returns br_status
+  int (*consumed)(void* ctx, const int* layers, int n) = nullptr;
 };
 
 // Transient scratch (bytes) the tensor-core step needs for these layers.

@@ -171,7 +171,13 @@ BR_API br_status br_set_lr(br_handle* h, float lr);
 
 /* Run the Power() part of Algorithm 2 now, from the current L, R (S=2nd) or M (S=1st);
  * layer = -1 refreshes every rotated layer.  Does not change t.  BR_ERR_STATE if a target
- * layer has t == 0 (its factor is all zero). */
+ * layer has t == 0 (its factor is all zero).
+ * Bases are refreshed several at a time on internal streams that fork from and join the
+ * handle's stream inside the call (the same happens for the periodic refresh inside br_step, which
+ * also stores the call's gradients through an internal stream that joins before it returns).  The
+ * launch chain of a basis is captured into a CUDA graph the first time its (order, form) occurs and
+ * replayed afterwards; if the handle's stream is itself being captured at that moment the capture
+ * is refused and the library falls back to plain launches for the rest of the handle's life. */
 BR_API br_status br_refresh_basis(br_handle* h, int layer);
 
 /* Wait for the stream and return the device status word (BR_OK, BR_WARN_RANK_DEFICIENT,

@@ -176,8 +176,9 @@ BR_API br_status br_set_lr(br_handle* h, float lr);
  * handle's stream inside the call (the same happens for the periodic refresh inside br_step, which
  * also stores the call's gradients through an internal stream that joins before it returns).  The
  * launch chain of a basis is captured into a CUDA graph the first time its (order, form) occurs and
- * replayed afterwards; if the handle's stream is itself being captured at that moment the capture
- * is refused and the library falls back to plain launches for the rest of the handle's life. */
+ * replayed afterwards (plain launches if that capture fails).  Neither this call nor br_step may be
+ * issued while the handle's stream is being captured by the caller: both read conditioning notes of
+ * the previous refresh back from the device. */
 BR_API br_status br_refresh_basis(br_handle* h, int layer);
 
 /* Wait for the stream and return the device status word (BR_OK, BR_WARN_RANK_DEFICIENT,

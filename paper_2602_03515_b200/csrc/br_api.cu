@@ -350,7 +350,9 @@ br_status deflated_power(br_handle* h, br_handle::Lane& ln, QrTc* tcq, int64_t k
 
 // A <- qr(A).Q for the product in the lane's buffer; the conditioning note goes to d_cond[ci].
 br_status orthonormalise(br_handle* h, br_handle::Lane& ln, int64_t k, QrTc* tcq, int ci, cudaStream_t s) {
-  if (h->use_graphs) {
+  cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(s, &capturing) != cudaSuccess) { cudaGetLastError(); capturing = cudaStreamCaptureStatusActive; }
+  if (h->use_graphs && capturing == cudaStreamCaptureStatusNone) {
     const int64_t key = 2 * k + (tcq ? 1 : 0);
     auto it = ln.qr_graphs.find(key);
     if (it == ln.qr_graphs.end()) {

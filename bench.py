@@ -25,9 +25,9 @@ sys.path.insert(0, ROOT)
 from workloads import get_workload  # noqa: E402
 from workloads.configs import GEOM_BI, GEOM_NONE, GEOM_UNI, SRC_SECOND  # noqa: E402
 
-# profiles/k_tc_gemm_c5_4layers.md: 45.5e9 B of DRAM traffic for the five launches of one step, which
+# profiles/k_tc_gemm_c5_4layers.md: 40.1e9 B of DRAM traffic for the ten launches of one step, which
 # execute 2.111e13 flop
-NCU_DRAM_BYTES_PER_EXECUTED_FLOP = 45.5e9 / 2.111e13
+NCU_DRAM_BYTES_PER_EXECUTED_FLOP = 40.1e9 / 2.111e13
 
 METRIC = "rotated_adam_params_per_sec"
 UNIT = "params/s"

@@ -278,7 +278,7 @@ BR_API br_status br_gemm_bf16(void* cuda_stream, int64_t Md, int64_t Nd, int64_t
  * F is k x k fp32, DEVICE, read only.  The caller owns F and Q.  device_flag, if not NULL, is a
  * DEVICE int that receives 0 or BR_WARN_RANK_DEFICIENT.
  *
- * Scratch lives in a fixed array inside the library's device image (about 3.4 MB on every GPU
+ * Scratch lives in a fixed array inside the library's device image (about 2.9 MB on every GPU
  * that loads the library, held until the process exits), so k is limited to 512: larger orders
  * return BR_ERR_SHAPE and must use br_create / br_refresh_basis.  The call itself, and everything
  * it calls, performs no cudaMalloc, cudaFree or other allocating routine.  The first call on a

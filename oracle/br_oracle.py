@@ -92,31 +92,69 @@ def qr_pos(A: np.ndarray):
     return Q, R, deficient
 
 
+def qr_pos_lapack(A: np.ndarray):
+    """The same factorisation with the library's Householder QR (numpy.linalg.qr, i.e. LAPACK) as the
+    step, followed by the same sign fix.  For a full-column-rank A the factorisation with
+    diag(R) > 0 is unique, so this and `qr_pos` compute one definition (Sec. 3.2 only says "QR
+    decomposition"); `qr_pos` is the written-out form that can be checked by eye, this one is what
+    makes orders in the thousands affordable (`Hyper.qr = "lapack"`).  Pinned against `qr_pos` and
+    against the defining properties (Q^T Q = I, Q R = A, R upper triangular with a positive
+    diagonal) in tests/test_oracle_pins.py.  Returns (Q, R, deficient) like `qr_pos`."""
+    A = np.asarray(A, dtype=np.float64)
+    rows, cols = A.shape
+    assert rows >= cols
+    Q, R = np.linalg.qr(A, mode="reduced")
+    d = np.diag(R).copy()
+    sgn = np.where(d < 0.0, -1.0, 1.0)
+    Q = Q * sgn[None, :]
+    R = R * sgn[:, None]
+    dmax = np.max(np.abs(d)) if cols else 0.0
+    deficient = bool(dmax == 0.0 or np.any(np.abs(d) <= RANK_TOL * dmax))
+    return Q, R, deficient
+
+
+QR_IMPLS = {"householder": qr_pos, "lapack": qr_pos_lapack}
+
 COMPLETION = 1e-6
 
 
-def qr_completed(A: np.ndarray, Qprev: np.ndarray):
+def qr_completed(A: np.ndarray, Qprev: np.ndarray, qr=qr_pos):
     """Q factor of A with a positive diagonal of R.  The paper does not say what Power() returns
     when F Q is rank-deficient (S = 1st on the larger side of a bilateral layer: M M^T has rank
     <= min(m, n)).  Reading taken here: whenever the plain factorisation meets a negligible pivot,
     the directions outside the range of A are completed from the current basis, by factorising
     A with COMPLETION * ||A_j|| * Qprev_j added to every column j (a zero column becomes Qprev_j),
     which has full rank when Qprev has.  The rule is invariant to a rescaling of A or of its columns."""
-    Q, R, d = qr_pos(A)
+    Q, R, d = qr(A)
     if d:
         cn = np.linalg.norm(A, axis=0)
         w = np.where(cn > 0.0, COMPLETION * cn, 1.0)
-        Q, R, _ = qr_pos(A + Qprev * w[None, :])
+        Q, R, _ = qr(A + Qprev * w[None, :])
     return Q, R, d
 
 
-def power(F: np.ndarray, Q: np.ndarray, iters: int = 1):
+def power(F: np.ndarray, Q: np.ndarray, iters: int = 1, qr=qr_pos):
     """Power(F, Q): `iters` times Q <- qr(F Q).Q (Sec. 3.2; the paper uses 1)."""
     deficient = False
     for _ in range(iters):
-        Q, _, d = qr_completed(F @ Q, Q)
+        Q, _, d = qr_completed(F @ Q, Q, qr)
         deficient |= d
     return Q, deficient
+
+
+def power_sensitivity(F: np.ndarray, Q: np.ndarray, rel: float = 2.0 ** -24, seed: int = 0, qr=qr_pos) -> float:
+    """Diagnostic of how well posed one Power(F, Q) is: the largest entry by which the sign-normalised
+    result moves when every entry of F is perturbed by a relative `rel` (symmetric Gaussian pattern;
+    the default is one fp32 rounding of the stored factor).  The unique Q factor can be numerically
+    fragile (trailing columns come out of a cancellation against the leading eigen-directions): a
+    basis mismatch of this size against an implementation that keeps F in fp32 says nothing about
+    its arithmetic.  Not a step of the method."""
+    F = np.asarray(F, dtype=np.float64)
+    Z = np.random.default_rng(seed).standard_normal(F.shape)
+    Z = (Z + Z.T) / np.sqrt(2.0)
+    Q0, _ = power(F, Q, 1, qr)
+    Q1, _ = power(F * (1.0 + rel * Z), Q, 1, qr)
+    return float(np.max(np.abs(sign_normalise(Q0) - sign_normalise(Q1))))
 
 
 def sign_normalise(Q: np.ndarray) -> np.ndarray:
@@ -177,6 +215,7 @@ class Hyper:
     power_iters: int = 1
     accum: str = "every_step"      # or "on_refresh" (literal Algorithm 2)
     clip_norm: float = 0.0         # global-norm gradient clipping (App. D.2 uses 1.0); 0 = off
+    qr: str = "householder"        # QR step of Power(): "householder" (written out) or "lapack" (library routine)
 
 
 class OracleLayer:
@@ -229,18 +268,18 @@ class OracleLayer:
         if self.R is not None:
             self.R = beta * self.R + (1.0 - beta) * (G.T @ G)
 
-    def refresh(self, power_iters=1):
+    def refresh(self, power_iters=1, qr=qr_pos):
         """The Power part of Algorithm 2 on the current L, R (S=2nd) or M (S=1st)."""
         deficient = False
         piv = []
         if self.left:
             F = self.L if self.src == SRC_SECOND else self.M @ self.M.T
-            self.U, d, p = _power_with_pivot(F, self.U, power_iters)
+            self.U, d, p = _power_with_pivot(F, self.U, power_iters, qr)
             deficient |= d
             piv.append(p)
         if self.right:
             F = self.R if self.src == SRC_SECOND else self.M.T @ self.M
-            self.V, d, p = _power_with_pivot(F, self.V, power_iters)
+            self.V, d, p = _power_with_pivot(F, self.V, power_iters, qr)
             deficient |= d
             piv.append(p)
         self.refresh_count += 1
@@ -248,11 +287,11 @@ class OracleLayer:
         return deficient
 
 
-def _power_with_pivot(F, Q, iters):
+def _power_with_pivot(F, Q, iters, qr=qr_pos):
     deficient, piv = False, np.inf
     for _ in range(iters):
         A = F @ Q
-        Q, R, d = qr_completed(A, Q)
+        Q, R, d = qr_completed(A, Q, qr)
         deficient |= d
         cn = np.linalg.norm(A, axis=0)
         cn[cn == 0] = 1.0
@@ -329,7 +368,7 @@ class Oracle:
         if lay.t % freq == 0:
             if second and hp.accum == "on_refresh":
                 lay.accumulate_factors(G, self._beta_factor())
-            deficient = lay.refresh(hp.power_iters)
+            deficient = lay.refresh(hp.power_iters, QR_IMPLS[hp.qr])
         # Alg. 1 lines 8-11
         Gt = lay.rotate(G)
         Mt = lay.rotate(lay.M)
@@ -351,7 +390,7 @@ class Oracle:
                 continue
             if lay.t == 0:
                 raise ValueError("refresh before the first update: the factor is all zero")
-            deficient |= lay.refresh(self.hp.power_iters)
+            deficient |= lay.refresh(self.hp.power_iters, QR_IMPLS[self.hp.qr])
         return STATUS_RANK_DEFICIENT if deficient else STATUS_OK
 
     def counters(self, layer: int):

@@ -173,7 +173,7 @@ k_dgemm(int ta, int tb, int64_t M, int64_t N, int64_t K, double alpha, const TA*
   const bool split = gridDim.z > 1;
   double* out = split ? partial + (int64_t)blockIdx.z * M * N : C;
   const int64_t ldo = split ? N : ldc;
-  const bool vec_o = split ? ((N & 1) == 0) : (vec_c != 0);
+  const bool vec_o = split ? (((N & 1) == 0) && ((reinterpret_cast<uintptr_t>(partial) & 15) == 0)) : (vec_c != 0);
 #pragma unroll
   for (int mi = 0; mi < 4; ++mi) {
     const int64_t row = m0 + 32 * wm + 8 * mi + g;

@@ -10,7 +10,7 @@
 // its scratch in a fixed array that lives in the library's device image.
 //
 // The array is loaded on every GPU that loads the library and stays there until the process
-// exits (3.4 MB per GPU), which is why the supported order is capped at kMaxOrder.
+// exits (2.9 MB per GPU), which is why the supported order is capped at kMaxOrder.
 //
 // `g_power_scratch` is a device symbol: in host code its name is only a stand-in, never a device
 // address, so the host obtains the real address with cudaGetSymbolAddress -- once per device,
@@ -22,9 +22,11 @@
 namespace {
 
 constexpr int64_t kMaxOrder = 512;
-// k*k doubles for the product F*Q, the QR work area for order kMaxOrder (152,576 doubles), and
-// 64 doubles holding the rank-deficiency flag.
-constexpr size_t kScratchDoubles = (size_t)kMaxOrder * kMaxOrder + 160000 + 64;
+// k*k doubles for the product F*Q (rounded up to a 256-byte boundary), the QR work area (90,688
+// doubles at order kMaxOrder, the largest over all orders up to it), and 64 doubles holding the
+// rank-deficiency flag.
+constexpr size_t kWorkDoubles = 98304;
+constexpr size_t kScratchDoubles = (size_t)kMaxOrder * kMaxOrder + kWorkDoubles + 64;
 
 static __device__ __align__(256) double g_power_scratch[kScratchDoubles];
 
@@ -56,13 +58,15 @@ extern "C" br_status br_power_static(void* cuda_stream, const float* F, float* Q
   using namespace br;
   if (!F || !Q || k < 1) return BR_ERR_INVALID;
   if (k > kMaxOrder) return BR_ERR_SHAPE;   // beyond the fixed scratch: use the handle-based path
-  const size_t need = (size_t)k * k + qr_work_doubles(k) + 64;
-  if (need > kScratchDoubles) return BR_ERR_SHAPE;
+  // the work area starts on a 256-byte boundary whatever the parity of k: its sub-buffers are
+  // accessed with 16-byte vector loads and stores
+  const size_t work_off = ((size_t)k * k + 31) / 32 * 32;
+  if (work_off + qr_work_doubles(k) + 64 > kScratchDoubles) return BR_ERR_SHAPE;
   cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
   double* scratch = nullptr;
   if (scratch_for_current_device(&scratch) != cudaSuccess) { (void)cudaGetLastError(); return BR_ERR_CUDA; }
   double* A = scratch;                                   // k x k product, overwritten by its Q factor
-  double* work = scratch + (size_t)k * k;
+  double* work = scratch + work_off;
   int* flag = device_flag ? device_flag : reinterpret_cast<int*>(scratch + (kScratchDoubles - 64));
   // The array keeps whatever the previous call left.  Only the flag has to start at zero; every
   // other word is written by this call before it is read.

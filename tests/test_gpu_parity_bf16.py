@@ -1,7 +1,7 @@
 """GPU parity of the tensor-core (bf16 operands, fp32 accumulation) path against the float64
-oracle through the C-ABI.  Tolerances: per-step parameter update relative L2 <= 2e-2; bases
-(sign-normalised) max-abs <= 1e-3 where the refresh is fed identical factors (teacher-forced);
-integer state bit-exact."""
+oracle through the C-ABI, free-running (nothing is copied from one side to the other).
+Tolerances: per-step parameter update relative L2 <= 2e-2; after every refresh the bases
+(sign-normalised) max-abs <= 1e-3 and V~ relative L2 <= 2e-2; integer state bit-exact."""
 from dataclasses import replace
 
 import numpy as np
@@ -12,17 +12,21 @@ from workloads.configs import GEOM_BI, GEOM_UNI, SRC_FIRST, SRC_SECOND, scaled
 
 pytestmark = pytest.mark.gpu
 
-TOL_DW = 2e-2
+TOL_DW, TOL_BASIS, TOL_V2 = 2e-2, 1e-3, 2e-2
 
 
-def _run(w, calls, tau=-1, tol=TOL_DW, **kw):
+def _run(w, calls, tau=-1, tol=TOL_DW, tol_basis=TOL_BASIS, **kw):
+    """tol_basis: a number, or a function of the refresh count of the layer (the bases of a long
+    free-running trajectory drift apart at the rate the fp32 storage of L and R allows)."""
     from tests.parity_util import SideBySide, rel_l2
     import paper_2602_03515_b200 as br
     sbs = SideBySide(w, gemm_prec=br.BR_GEMM_BF16, **kw)
     worst = 0.0
     deficient = False
+    worst_q = {}
     try:
         for c in range(calls):
+            before = [lay.refresh_count for lay in sbs.oracle.layers]
             st_g, st_o, dg, do = sbs.step(tau)
             # (a rank-deficient refresh is reported by the oracle's step at once, by the library through
             # the status word that br_sync_status reads)
@@ -35,9 +39,16 @@ def _run(w, calls, tau=-1, tol=TOL_DW, **kw):
                 e = rel_l2(a, b)
                 worst = max(worst, e)
                 assert e <= tol, (c, li, e)
-            for li in range(len(w.layers)):
+            for li, lay in enumerate(sbs.oracle.layers):
                 assert sbs.opt.counters(li) == sbs.oracle.counters(li)
+                if lay.refresh_count != before[li]:
+                    # a refresh happened inside this call: bases and V~ against the oracle's, now
+                    tb = tol_basis(lay.refresh_count) if callable(tol_basis) else tol_basis
+                    errs = sbs.check_bases(li, tb, TOL_V2, where=f"call {c + 1}, refresh {lay.refresh_count},")
+                    for k_, e_ in errs.items():
+                        worst_q[k_] = max(worst_q.get(k_, 0.0), e_)
         assert sbs.opt.sync_status() == (br.BR_WARN_RANK_DEFICIENT if deficient else br.BR_OK)
+        print(f"{w.name}: worst dW {worst:.2e}, worst after-refresh errors {worst_q}")
         for li, lay in enumerate(sbs.oracle.layers):
             # the tensor-core path keeps M~ = U^T M V (accumulated from bf16-pair products); M is U M~ V^T
             assert rel_l2(sbs.state(li, br.BR_BUF_M), lay.M) < 1e-4

@@ -202,6 +202,56 @@ def test_p6_qr_pos_hand_example():
                                     [-2 / 7, 6 / 35, -33 / 35]]), atol=1e-12)
 
 
+@pytest.mark.parametrize("shape", [(3, 3), (40, 40), (257, 257), (64, 20)])
+def test_p6_library_qr_variant_equals_the_written_out_one(shape):
+    """`qr_pos_lapack` (what `Hyper.qr = "lapack"` selects for orders in the thousands) against the
+    written-out Householder `qr_pos`, and against what defines the result whatever computes it:
+    Q^T Q = I, Q R = A, R upper triangular with a positive diagonal (unique for full column rank)."""
+    A = rng(17).standard_normal(shape)
+    Q0, R0, d0 = O.qr_pos(A)
+    Q1, R1, d1 = O.qr_pos_lapack(A)
+    assert not d0 and not d1
+    assert np.max(np.abs(Q0 - Q1)) < 1e-11 and np.max(np.abs(R0 - R1)) < 1e-11 * np.max(np.abs(R0))
+    assert np.max(np.abs(Q1.T @ Q1 - np.eye(shape[1]))) < 1e-12
+    assert np.max(np.abs(Q1 @ R1 - A)) < 1e-12 * np.max(np.abs(A)) * shape[0]
+    assert np.all(np.diag(R1) > 0) and np.array_equal(R1, np.triu(R1))
+
+
+def test_p6_library_qr_variant_hand_example_flag_and_trajectory():
+    A = np.array([[12.0, -51, 4], [6, 167, -68], [-4, 24, -41]])
+    Q, R, _ = O.qr_pos_lapack(A)
+    assert np.allclose(R, [[14, 21, -14], [0, 175, -70], [0, 0, 35]], atol=1e-10)
+    B = rng(8).standard_normal((6, 2)) @ rng(9).standard_normal((2, 6))   # rank 2
+    assert O.qr_pos_lapack(B)[2] and O.qr_pos(B)[2]
+    assert O.qr_pos_lapack(np.zeros((4, 4)))[2]
+    # a whole trajectory through three refreshes: the two variants agree to rounding
+    out = []
+    for impl in ("householder", "lapack"):
+        lay = O.OracleLayer(rng(3).standard_normal((24, 40)) * 0.02, O.GEOM_BI, O.SRC_SECOND, 0)
+        orc = O.Oracle([lay], O.Hyper(freq=4, qr=impl))
+        g = rng(4)
+        for _ in range(13):
+            orc.step([g.standard_normal((24, 40)) * 0.01], 0)
+        out.append((lay.W.copy(), lay.U.copy(), lay.V.copy()))
+    for a, b in zip(*out):
+        assert np.max(np.abs(a - b)) < 1e-9
+
+
+def test_p6_power_sensitivity_diagnostic():
+    """The conditioning diagnostic: zero for a diagonal factor (a relative perturbation keeps it diagonal,
+    so Power(F, I) stays I), first order in the size of the perturbation, and far larger for a
+    low-rank-plus-noise factor started from the identity than for a well-separated one."""
+    assert O.power_sensitivity(np.diag(np.logspace(0, -3, 16)), np.eye(16)) == 0.0
+    Qe, _ = np.linalg.qr(rng(31).standard_normal((24, 24)))
+    F = (Qe * (0.5 ** np.arange(24))) @ Qe.T
+    s1, s2 = O.power_sensitivity(F, np.eye(24), rel=1e-9), O.power_sensitivity(F, np.eye(24), rel=2e-9)
+    assert 0.0 < s1 < 1e-3 and abs(s2 / s1 - 2.0) < 1e-3
+    B = rng(32).standard_normal((64, 4))
+    noisy = 1e4 * B @ B.T + np.cov(rng(33).standard_normal((64, 640)))
+    easy = (Qe * np.linspace(2.0, 1.0, 24)) @ Qe.T
+    assert O.power_sensitivity(noisy, np.eye(64)) > 1e3 * O.power_sensitivity(easy, np.eye(24))
+
+
 def test_p6_rank_deficient_flag_and_orthonormality():
     A = rng(8).standard_normal((6, 2)) @ rng(9).standard_normal((2, 6))   # rank 2
     Q, R, deficient = O.qr_pos(A)

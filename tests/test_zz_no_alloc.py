@@ -6,7 +6,9 @@ device image instead of the handle's slab.
 Checked here, through the C-ABI, on two calls in a row (the second one finds the first one's
 leftovers in the shared array): the result equals what the handle-based path (br_set_state +
 br_refresh_basis) produces from the same factor and basis, within the basis tolerance of the other
-tests (sign-normalised max-abs 1e-3).  Orders beyond the fixed scratch are rejected."""
+tests (sign-normalised max-abs 1e-3), and equals the float64 oracle's Power(F, Q) within the same
+tolerance.  Odd orders are covered as well (the work area behind the k x k product must stay on a
+vector-access boundary for them).  Orders beyond the fixed scratch are rejected."""
 import numpy as np
 import pytest
 
@@ -24,12 +26,13 @@ def _factor(k, seed):
     return F, Q0.astype(np.float32)
 
 
-def test_static_scratch_power_matches_handle_path_twice():
+@pytest.mark.parametrize("k", [200, 129, 201])      # several panels, the last one ragged; odd orders
+def test_static_scratch_power_matches_handle_path_twice(k):
     import torch
     import paper_2602_03515_b200 as br
+    from oracle import br_oracle as O
     from workloads import LayerSpec
     from tests.parity_util import basis_err
-    k = 200                                    # several panels, the last one ragged
     w = torch.zeros(k, 16, device="cuda")
     opt = br.BasisRotation([LayerSpec("W", k, 16, br.BR_GEOM_BILATERAL, br.BR_SRC_SECOND, 0)], [w],
                            grad_dtype="f32", gemm_prec=br.BR_GEMM_FP32, freq=10 ** 6)
@@ -55,6 +58,9 @@ def test_static_scratch_power_matches_handle_path_twice():
             assert int(flag.item()) == 0
             assert np.all(np.isfinite(got))
             assert basis_err(got, want) <= TOL_BASIS, (call, basis_err(got, want))
+            ref, deficient = O.power(F.astype(np.float64), Q0.astype(np.float64))
+            assert not deficient
+            assert basis_err(got, ref) <= TOL_BASIS, (call, basis_err(got, ref))
             assert np.max(np.abs(got.T @ got - np.eye(k))) < 1e-5
     finally:
         opt.close()

@@ -168,6 +168,32 @@ def fit_tau(w_name, n_layers, tau_req, gemm_prec, free_bytes, margin, br):
 
 
 # ---------------------------------------------------------------------------------------------
+def cpu_oracle_refresh(w, shapes):
+    """Seconds the oracle's Power() takes for the bases of the given layer shapes, per refresh.  One
+    Power(F, Q) (float64 product + QR, the library QR routine as its step: the written-out Householder
+    form takes about a minute at order 2560) is timed at the smallest distinct order; larger orders are
+    composed by k^3.  Returns (seconds, description)."""
+    import numpy as np
+    from oracle import br_oracle as O
+    orders = []
+    for (m, n, geom, src) in shapes:
+        if geom == GEOM_BI or (geom == GEOM_UNI and m <= n):
+            orders.append(m)
+        if geom == GEOM_BI or (geom == GEOM_UNI and m > n):
+            orders.append(n)
+    if not orders:
+        return 0.0, "no rotated side"
+    k0 = min(orders)
+    rng = np.random.default_rng(1)
+    X = rng.standard_normal((k0, 2 * k0))
+    F = X @ X.T / (2 * k0)
+    t0 = time.perf_counter()
+    O.power(F, np.eye(k0), qr=O.qr_pos_lapack)
+    t_k0 = time.perf_counter() - t0
+    total = sum(t_k0 * (k / k0) ** 3 for k in orders)
+    return total, f"Power() timed at order {k0} ({t_k0:.2f} s), orders {sorted(set(orders))} composed by k^3"
+
+
 def cpu_oracle_sample(w, shapes, reps=1):
     """Time the float64 oracle (as it stands) on one steady step of each given layer shape."""
     import numpy as np
@@ -193,7 +219,9 @@ def cpu_oracle_sample(w, shapes, reps=1):
         threads = max(p["num_threads"] for p in threadpoolctl.threadpool_info() if p.get("user_api") == "blas")
     except Exception:
         threads = len(os.sched_getaffinity(0))
-    return total_params / total_t, total_t, threads
+    t_refresh, how = cpu_oracle_refresh(w, shapes)
+    amortised = total_t + t_refresh / w.freq
+    return total_params / amortised, amortised, threads, dict(step_seconds=total_t, refresh_seconds=t_refresh, refresh=how)
 
 
 def sample_shapes(w, small: bool):
@@ -217,13 +245,14 @@ def run_reference(args):
     shapes = sample_shapes(w, small=True)
     times = []
     for i in range(args.warmup + args.steps):
-        v, t, threads = cpu_oracle_sample(w, shapes)
+        v, t, threads, parts = cpu_oracle_sample(w, shapes)
         if i >= args.warmup:
             times.append(t)
     ms = 1e3 * sum(times) / len(times)
     params = sum(m * n for m, n, _, _ in shapes)
     value = params / (ms / 1e3)
-    sample = "one steady (refresh-free) oracle step of a %dx%d matrix of %s per step" % (shapes[0][0], shapes[0][1], w.name)
+    sample = ("one oracle step of a %dx%d matrix of %s + (one Power() of each of its bases)/freq per step; %s; the %s is left out of the sample"
+              % (shapes[0][0], shapes[0][1], w.name, parts["refresh"], "embedding" if w.name in ("c4", "c5") else "rest of the layer set"))
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f64", "data": "synthetic", "config": {"workload": w.name, "sample": sample},
@@ -231,6 +260,54 @@ def run_reference(args):
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line), flush=True)
+
+
+def deep_ring_check(args, br, torch, dev, stream, tau_req, gemm_prec, main_steady_ms, main_params, main_tau):
+    """The steady step with the ring depth the workload asks for, on the largest decoder depth whose state
+    fits it: the work of a step (one ring write, one ring read per parameter) should not depend on the
+    depth of the ring, only memory does.  Reported as time per parameter beside the main run's."""
+    free0, _ = torch.cuda.mem_get_info(dev)
+    n_fit = None
+    for n_layers in range((args.layers or 32), 0, -1):
+        wt = get_workload(args.workload, n_layers=n_layers, tau=tau_req)
+        descs = [br.BrLayerDesc(m=l.m, n=l.n, geom=l.geom, src=l.src, grad_dtype=br.BR_BF16, tau_max=l.tau_max, freq=0,
+                                reserved=0, weight=0) for l in wt.layers]
+        hp = br.BrHparams(lr=wt.lr, beta1=wt.beta1, beta2=wt.beta2, eps=wt.eps, weight_decay=0.0, beta_factor=-1.0, freq=wt.freq,
+                          power_iters=1, accum=0, gemm_prec=gemm_prec, flags=0, clip_norm=0.0, scratch_limit_bytes=0)
+        need = br.br_state_bytes(descs, hp)[0] + wt.n_params * (4 + 2 + 4) + (6 << 30)
+        if need <= free0:
+            n_fit = n_layers
+            break
+    if n_fit is None:
+        return {"error": "no depth fits"}
+    wt = get_workload(args.workload, n_layers=n_fit, tau=tau_req)
+    weights = [torch.empty(l.m, l.n, device=dev).normal_(0.0, 0.02) for l in wt.layers]
+    with torch.cuda.stream(stream):
+        gen = DeviceGradients(wt, dev, torch)
+        opt = br.BasisRotation.from_workload(wt, weights, stream=stream)
+        for _ in range(tau_req + 8):
+            opt.step(gen.fresh(), tau_req)
+        for _ in range(3):
+            opt.refresh_basis(-1)
+            for _ in range(4):
+                opt.step(gen.fresh(), tau_req)
+        steps = 10
+        ev0 = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+        ev1 = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+        for k in range(steps):
+            gen.fresh()
+            ev0[k].record(stream)
+            opt.step(gen.grads, tau_req)
+            ev1[k].record(stream)
+        torch.cuda.synchronize(dev)
+        assert opt.sync_status() >= 0
+        ms = sum(a.elapsed_time(b) for a, b in zip(ev0, ev1)) / steps
+        slot = opt.counters(0)["ring_slot"]
+    opt.close()
+    return {"decoder_layers": n_fit, "params": wt.n_params, "tau": tau_req, "ms_steady_step": ms, "steps": steps,
+            "ps_per_param": 1e9 * ms / wt.n_params, "main_run_ps_per_param": 1e9 * main_steady_ms / main_params,
+            "main_run_tau": main_tau, "ring_slot_after": slot,
+            "note": "same command, same process: the largest decoder depth whose state fits a uniform ring of the requested depth"}
 
 
 # ---------------------------------------------------------------------------------------------
@@ -246,6 +323,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=12)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--scratch-gib", type=float, default=0.0)
+    ap.add_argument("--no-tau-check", action="store_true",
+                    help="skip the second, shallower run at the requested ring depth (config.tau32_check)")
     ap.add_argument("--no-refresh", action="store_true",
                     help="profiling captures only: skip the basis refresh (priming and timing); the line is then not a bench value")
     args = ap.parse_args()
@@ -262,6 +341,11 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.gpus != world:
+        # one process per GPU: N > 1 needs a launcher that sets WORLD_SIZE / RANK / LOCAL_RANK
+        sys.exit(f"bench.py: --gpus {args.gpus} but WORLD_SIZE is {world}; launch N > 1 as "
+                 f"`python -m torch.distributed.run --nnodes=1 --nproc-per-node {args.gpus} --master-addr 127.0.0.1 "
+                 f"--master-port P bench.py --gpus {args.gpus} ...`")
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
@@ -438,7 +522,10 @@ def main():
         e2e_ms = 1e3 * (time.perf_counter() - t0) / args.e2e_steps + refresh_ms / w.freq
         e2e_ms = max_over_ranks([e2e_ms], world, dev, torch)[0]
         e2e = {"value": replica_value(n_params, world, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
-               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": args.e2e_steps}
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": args.e2e_steps,
+               "note": "the step's inputs (every layer's gradient) are uploaded from pinned host memory every step; its result, the updated "
+                       "weights, stays on the device where the caller's model owns it -- read back per step are one updated weight "
+                       "matrix (%d x %d fp32) and, at the end, the status word" % tuple(weights[0].shape)}
         del host, grads2
 
     # ---- rooflines -------------------------------------------------------------------------------
@@ -452,13 +539,37 @@ def main():
         # DRAM bytes per launch: dram__bytes_read+write of an ncu capture of a small case of this
         # workload (profiles/), scaled to this run's launches by executed flop per launch
         traffic = NCU_DRAM_BYTES_PER_EXECUTED_FLOP * prof["tc_flops"] / prof["tc_launches"]
-        roofline = {"bound": "tensor", "kernel": "k_tc_gemm", "achieved": achieved, "peak": peaks["tf_sustained"],
-                    "unit": "TFLOP/s", "frac": achieved / peaks["tf_sustained"], "traffic": traffic,
+        # achieved / frac: what the tensor pipe executed (9 one-sided products per bilateral matrix, the factor
+        # products on upper-triangle tiles only); effective_*: the method's own 8 m n (m + n) over the same time
+        roofline = {"bound": "tensor", "kernel": "k_tc_gemm", "achieved": executed, "peak": peaks["tf_sustained"],
+                    "unit": "TFLOP/s", "frac": executed / peaks["tf_sustained"], "traffic": traffic,
                     "traffic_source": "ncu capture of the 4-layer case, scaled by executed flop per launch",
-                    "executed_tflops": executed, "executed_frac": executed / peaks["tf_sustained"],
+                    "effective_tflops": achieved, "effective_frac": achieved / peaks["tf_sustained"],
+                    "flops_counted": "executed by the tensor pipe (effective_* counts the algorithmic 8mn(m+n))",
                     "launches_per_step": prof["tc_launches"] / prof_steps, "ms_per_step_in_kernel": tc_ms_step,
                     "avg_launch_ms": prof["tc_ms"] / prof["tc_launches"],
                     "peak_source": peaks["source"] + ", bf16 sustained"}
+
+    # ---- the refresh against its own rooflines ------------------------------------------------------
+    roofline_refresh = None
+    if not args.no_refresh:
+        orders = []
+        for l in w.layers:
+            if l.geom == GEOM_BI or (l.geom == GEOM_UNI and l.m <= l.n):
+                orders.append(l.m)
+            if l.geom == GEOM_BI or (l.geom == GEOM_UNI and l.m > l.n):
+                orders.append(l.n)
+        # per basis of order k: 2 k^3 (the product F Q) + 8/3 k^3 (QR with Q formed); S = 1st adds the factor itself
+        ref_flops = sum((2.0 + 8.0 / 3.0) * float(k) ** 3 for k in orders)
+        ref_tflops = ref_flops / (refresh_ms / 1e3) / 1e12
+        fp64_peak = 148 * 64 * 2 * 1.965e9 / 1e12       # 148 SMs x 64 fp64 FMA per clock (mma.sync.m8n8k4.f64) x 2 x 1.965 GHz
+        roofline_refresh = {"bound": "fp64 matrix unit / tensor", "kernel": "k_dgemm + k_chol_inverse + k_tc_gemm (three-term bf16 splits)",
+                            "bases": len(orders), "algorithmic_flops": ref_flops, "achieved": ref_tflops, "unit": "TFLOP/s",
+                            "peak_fp64_unit": fp64_peak, "frac_of_fp64_unit": ref_tflops / fp64_peak,
+                            "peak_bf16_split6": peaks["tf_sustained"] / 6.0, "frac_of_bf16_split6": ref_tflops / (peaks["tf_sustained"] / 6.0),
+                            "ms": refresh_ms, "share_of_amortised_step": (refresh_ms / w.freq) / amortised_ms,
+                            "peak_source": "fp64: 148 SMs x 64 FMA/clk x 2 x 1.965 GHz (a register-only loop of the instruction reaches 99 % of it); "
+                                           "bf16: " + peaks["source"] + " sustained / 6 (six bf16 products per fp32-accurate product)"}
 
     # ---- element-wise kernel of the path (Eq. (adam) for parameters that are not rotated) ---------------
     # The steady step of a fully rotated layer set runs no element-wise kernel (the moment updates are
@@ -496,10 +607,11 @@ def main():
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         shapes = sample_shapes(w, small=False)
-        v, t, threads = cpu_oracle_sample(w, shapes, reps=3)
-        cpu = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "seconds": t,
-               "sample": "best of 3 steady (refresh-free) float64 oracle steps of each of " +
-                         ", ".join(f"{m}x{n}" for m, n, _, _ in shapes) + f" from {w.name}"}
+        v, t, threads, parts = cpu_oracle_sample(w, shapes, reps=3)
+        cpu = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "seconds": t, **parts,
+               "sample": "best of 3 float64 oracle steps of each of " +
+                         ", ".join(f"{m}x{n}" for m, n, _, _ in shapes) + f" from {w.name}, plus (one Power() of each of their bases)/freq, "
+                         "as the GPU value charges it; the 32000-row embedding is left out of the sample (one float64 step of it is beyond the sample's budget)"}
 
     if rank == 0:
         line = {
@@ -514,11 +626,20 @@ def main():
                        "l2": "inputs larger than L2 (no flush needed)" if n_params * 2 > (126 << 20) else "inputs smaller than L2",
                        "replicas": world, "refresh_skipped_not_a_bench_value": bool(args.no_refresh), "gradients": "device-generated; signal factors fixed per layer, noise drawn afresh before every step (untimed)"},
             "clocks": clocks, "clocks_during_refresh": clocks_refresh, "e2e": e2e, "gpu_launches": int(l1 - l0),
-            "roofline": roofline, "roofline_elementwise": roofline_elem, "cpu_baseline": cpu,
+            "roofline": roofline, "roofline_refresh": roofline_refresh, "roofline_elementwise": roofline_elem, "cpu_baseline": cpu,
             "algorithmic_flops_per_step": alg_flops,
         }
-        print(json.dumps(line), flush=True)
     opt.close()
+    # ---- the requested ring depth on as many layers as fit it (the full set runs with a shallower ring) ----
+    if rank == 0 and world == 1 and args.workload in ("c4", "c5") and tau < tau_req and not args.no_tau_check and not args.no_refresh:
+        try:
+            del opt, weights, grads, gen
+            torch.cuda.empty_cache()
+            line["config"]["tau32_check"] = deep_ring_check(args, br, torch, dev, stream, tau_req, gemm_prec, steady_ms, n_params, tau)
+        except Exception as ex:                  # the side measurement must not take the bench line down
+            line["config"]["tau32_check"] = {"error": str(ex)}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
 

@@ -25,7 +25,9 @@
  * All pointers named DEVICE are CUDA device pointers on the handle's device; all
  * others are host pointers.  Matrices are row-major and contiguous.  Every entry
  * point returns a br_status: 0 = ok, > 0 informational (state is valid), < 0
- * error.  An error detected on the host leaves the handle unchanged.  Work is
+ * error.  An error detected on the host leaves the handle unchanged; BR_ERR_CUDA from br_step or
+ * br_refresh_basis (a failed enqueue) leaves the integer state as it was before the call, but device
+ * buffers may be partly updated: the handle is then good for the accessors and br_destroy only.  Work is
  * enqueued on the handle's stream; only the calls documented as synchronising
  * wait for it.  There is no CPU fallback: every step of the path runs in CUDA
  * kernels, and the calls fail with BR_ERR_CUDA when no device is usable.
@@ -249,6 +251,28 @@ BR_API br_status br_effective_delay(const double* C, const int* tau, int n, doub
  */
 BR_API br_status br_lr_warmup_cosine(int64_t step, int64_t total_steps, double warmup_fraction, double base_lr,
                                      double min_lr, double* out_lr);
+
+/*
+ * Failure-path diagnostics (every device-side wait is bounded and reports through the status word;
+ * host errors leave the integer state untouched).  Neither call faults,
+ * traps or hangs the GPU.
+ *
+ * br_debug_inject: host-side fault injection.  With kind = BR_INJECT_LAUNCH_FAILURE the library counts
+ * the CUDA calls (launches, copies, event operations) it is about to issue for this handle; the one
+ * that finds `countdown` at 0 is not issued and reports a launch failure instead, so the entry point
+ * that was running returns BR_ERR_CUDA.  BR_INJECT_NONE disarms it.  After an injected failure inside
+ * br_step the integer state (calls, t, refresh_count, ring slot) reads as before the call; device
+ * buffers may have been touched by the launches that went out before it.
+ *
+ * br_debug_wait_timeout: enqueues a one-warp kernel that waits, with the contraction kernel's own bounded
+ * wait, on a barrier that nothing will ever arrive on, for limit_ns (1 us .. 2 s).  The wait gives up,
+ * the kernel returns, and the status word holds BR_ERR_TIMEOUT from then on: br_sync_status returns it,
+ * later contraction launches of the handle return at once without touching their outputs, and the
+ * handle can still be read and destroyed.
+ */
+typedef enum { BR_INJECT_NONE = 0, BR_INJECT_LAUNCH_FAILURE = 1 } br_inject_kind;
+BR_API br_status br_debug_inject(br_handle* h, int kind, int64_t countdown);
+BR_API br_status br_debug_wait_timeout(br_handle* h, uint64_t limit_ns);
 
 BR_API const char* br_strerror(int status);
 /* Message of the last error on this handle (or of the last failed br_create when h is NULL). */

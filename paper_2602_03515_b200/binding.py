@@ -99,6 +99,8 @@ def load_library():
         "br_effective_delay": ([C.POINTER(C.c_double), C.POINTER(C.c_int), C.c_int, C.POINTER(C.c_double)], C.c_int),
         "br_lr_warmup_cosine": ([C.c_int64, C.c_int64, C.c_double, C.c_double, C.c_double, C.POINTER(C.c_double)], C.c_int),
         "br_destroy": ([H], C.c_int),
+        "br_debug_inject": ([H, C.c_int, C.c_int64], C.c_int),
+        "br_debug_wait_timeout": ([H, C.c_uint64], C.c_int),
         "br_power_static": ([C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p], C.c_int),
         "br_strerror": ([C.c_int], C.c_char_p),
         "br_last_error": ([H], C.c_char_p),
@@ -228,6 +230,17 @@ def br_lr_warmup_cosine(step: int, total_steps: int, warmup_fraction: float, bas
     _check(load_library().br_lr_warmup_cosine(int(step), int(total_steps), float(warmup_fraction), float(base_lr),
                                               float(min_lr), C.byref(out)))
     return float(out.value)
+
+
+BR_INJECT_NONE, BR_INJECT_LAUNCH_FAILURE = 0, 1
+
+
+def br_debug_inject(handle, kind: int, countdown: int = 0) -> int:
+    return _check(load_library().br_debug_inject(handle, int(kind), int(countdown)), handle)
+
+
+def br_debug_wait_timeout(handle, limit_ns: int) -> int:
+    return _check(load_library().br_debug_wait_timeout(handle, int(limit_ns)), handle)
 
 
 def br_destroy(handle) -> int:

@@ -149,6 +149,9 @@ struct br_handle {
 
 namespace {
 
+br_status step_enqueue(br_handle* h, const void* const* grads, int tau);
+void release(br_handle* h);
+
 struct Bump {
   size_t off = 0;
   char* base = nullptr;
@@ -284,7 +287,7 @@ void init_layers(br_handle* h, const br_layer_desc* layers, int n_layers) {
 
 #define BR_CUDA(h, expr)                                                              \
   do {                                                                                \
-    cudaError_t e__ = (expr);                                                         \
+    cudaError_t e__ = (h)->stats.inject() ? cudaErrorLaunchFailure : (expr);          \
     if (e__ != cudaSuccess) {                                                         \
       (h)->err = format("%s failed: %s", #expr, cudaGetErrorString(e__));             \
       return BR_ERR_CUDA;                                                             \
@@ -500,17 +503,24 @@ br_status refresh_layers(br_handle* h, const int* ids, int n_ids) {
   // interleave the enqueueing so that every lane has work early
   size_t longest = 0;
   for (auto& v : per_lane) longest = std::max(longest, v.size());
-  for (size_t r = 0; r < longest; ++r)
-    for (int i = 0; i < nl; ++i) {
+  br_status failed = BR_OK;
+  for (size_t r = 0; r < longest && failed == BR_OK; ++r)
+    for (int i = 0; i < nl && failed == BR_OK; ++i) {
       if (r >= per_lane[i].size()) continue;
       const Job& jb = per_lane[i][r];
-      br_status st = refresh_side(h, h->layers[jb.layer], jb.left, h->lanes[i]);
-      if (st != BR_OK) return st;
+      failed = refresh_side(h, h->layers[jb.layer], jb.left, h->lanes[i]);
     }
+  // the lanes forked from the handle's stream: join them again whatever happened above, so that
+  // nothing of this call is still running on an internal stream once the handle's stream has passed it
   for (int i = 1; i < nl; ++i) {
-    BR_CUDA(h, cudaEventRecord(h->lanes[i].done, h->lanes[i].stream));
-    BR_CUDA(h, cudaStreamWaitEvent(h->stream, h->lanes[i].done, 0));
+    cudaError_t je = cudaEventRecord(h->lanes[i].done, h->lanes[i].stream);
+    if (je == cudaSuccess) je = cudaStreamWaitEvent(h->stream, h->lanes[i].done, 0);
+    if (je != cudaSuccess && failed == BR_OK) {
+      h->err = format("joining a refresh lane failed: %s", cudaGetErrorString(je));
+      failed = BR_ERR_CUDA;
+    }
   }
+  if (failed != BR_OK) return failed;
   h->stats.prof.end(span, h->stream, h->stats.gemm_flops - f0);
   BR_CUDA(h, cudaMemcpyAsync(h->h_cond, h->d_cond, sizeof(int) * h->cond_known.size(), cudaMemcpyDeviceToHost, h->stream));
   BR_CUDA(h, cudaEventRecord(h->ev_cond, h->stream));
@@ -657,6 +667,35 @@ size_t buf_bytes(const Layer& L, int which, void** ptr) {
   }
 }
 
+// Frees everything a handle owns; also the teardown of a br_create that failed half-way (every
+// member is null or empty until it has been created).
+void release(br_handle* h) {
+  cudaSetDevice(h->device);
+  cudaStreamSynchronize(h->stream);
+  if (h->tc) tc_step_destroy(h->tc);
+  for (int i = 1; i < br_handle::kMaxLanes; ++i) {
+    if (h->lanes[i].stream) { cudaStreamSynchronize(h->lanes[i].stream); cudaStreamDestroy(h->lanes[i].stream); }
+    if (h->lanes[i].done) cudaEventDestroy(h->lanes[i].done);
+  }
+  if (h->ev_begin) cudaEventDestroy(h->ev_begin);
+  if (h->ev_cond) cudaEventDestroy(h->ev_cond);
+  if (h->copy_stream) { cudaStreamSynchronize(h->copy_stream); cudaStreamDestroy(h->copy_stream); }
+  if (h->ev_consumed) cudaEventDestroy(h->ev_consumed);
+  if (h->ev_copied) cudaEventDestroy(h->ev_copied);
+  if (h->h_cond) cudaFreeHost(h->h_cond);
+  for (int i = 0; i < br_handle::kMaxLanes; ++i) {
+    for (auto& kv : h->lanes[i].qr_graphs) if (kv.second.exec) cudaGraphExecDestroy(kv.second.exec);
+    for (QrTc* t : h->lanes[i].tcq) qr_tc_destroy(t);
+  }
+  for (auto& sp : h->stats.prof.spans) { cudaEventDestroy(sp.a); cudaEventDestroy(sp.b); }
+  for (auto e : h->stats.prof.free_events) cudaEventDestroy(e);
+  if (h->slab) {
+    if (h->alloc.alloc) h->alloc.free(h->slab, h->alloc.ctx); else cudaFree(h->slab);
+  }
+  (void)cudaGetLastError();
+  delete h;
+}
+
 }  // namespace
 
 // ---------------------------------------------------------------------------------------------
@@ -737,8 +776,7 @@ br_status br_create(br_handle** out, const br_layer_desc* layers, int n_layers, 
   cudaStream_t s = h->stream;
   auto fail = [&](const char* what, cudaError_t ce) {
     g_create_error = format("%s: %s", what, cudaGetErrorString(ce));
-    if (h->alloc.alloc) h->alloc.free(h->slab, h->alloc.ctx); else cudaFree(h->slab);
-    delete h;
+    release(h);
     return BR_ERR_CUDA;
   };
   if ((e = cudaMemsetAsync(h->slab, 0, sz.total, s)) != cudaSuccess) return fail("cudaMemsetAsync", e);
@@ -778,8 +816,7 @@ br_status br_create(br_handle** out, const br_layer_desc* layers, int n_layers, 
         QrTc* t = qr_tc_create(k, h->lanes[i].tcq_scratch, device, s, &qerr);
         if (!t) {
           g_create_error = qerr ? qerr : "tensor-core projection plans could not be created";
-          if (h->alloc.alloc) h->alloc.free(h->slab, h->alloc.ctx); else cudaFree(h->slab);
-          delete h;
+          release(h);
           return BR_ERR_CUDA;
         }
         h->lanes[i].tcq.push_back(t);
@@ -789,8 +826,7 @@ br_status br_create(br_handle** out, const br_layer_desc* layers, int n_layers, 
   h->tc = tc_step_create(h->layers, h->hp, h->slab + sz.total, tc_bytes, h->d_clip, h->clip_slots, device, s, &tc_err);
   if (!h->tc && tc_err) {
     g_create_error = tc_err;
-    if (h->alloc.alloc) h->alloc.free(h->slab, h->alloc.ctx); else cudaFree(h->slab);
-    delete h;
+    release(h);
     return BR_ERR_CUDA;
   }
   if ((e = cudaStreamSynchronize(s)) != cudaSuccess) return fail("cudaStreamSynchronize", e);
@@ -814,6 +850,31 @@ br_status br_step(br_handle* h, const void* const* grads, int tau) {
       return BR_ERR_TAU;
     }
   }
+  // The integer state moves while the work is enqueued (the launches need the new values); when an
+  // enqueue fails it is put back, so that calls, t, the refresh schedule and the ring slot read as
+  // they did before the call.  Device buffers may already have been touched by the launches that
+  // did go out: after BR_ERR_CUDA the handle is good for the accessors and br_destroy only.
+  struct Snapshot { int64_t t, refresh_count, n_accum; };
+  const int64_t calls_before = h->calls;
+  std::vector<Snapshot> before(nl);
+  for (int i = 0; i < nl; ++i) before[i] = {h->layers[i].t, h->layers[i].refresh_count, h->layers[i].n_accum};
+  st = step_enqueue(h, grads, tau);
+  if (st < 0) {
+    h->calls = calls_before;
+    for (int i = 0; i < nl; ++i) {
+      h->layers[i].t = before[i].t; h->layers[i].refresh_count = before[i].refresh_count; h->layers[i].n_accum = before[i].n_accum;
+    }
+  }
+  return st;
+}
+
+}  // extern "C"
+
+namespace {
+
+br_status step_enqueue(br_handle* h, const void* const* grads, int tau) {
+  const int nl = (int)h->layers.size();
+  br_status st = BR_OK;
   // ---- integer state (host) ---------------------------------------------------------------
   h->calls += 1;
   if (h->d_clip) {
@@ -894,7 +955,10 @@ br_status br_step(br_handle* h, const void* const* grads, int tau) {
       cudaEventRecord(h->ev_copied, h->copy_stream);
       cudaStreamWaitEvent(h->stream, h->ev_copied, 0);
     }
-    if (rc != 0) { h->err = terr ? terr : "tensor-core step failed"; return rc < 0 ? (br_status)rc : BR_ERR_CUDA; }
+    if (rc != 0) {
+      if (terr) h->err = terr; else if (h->err.empty()) h->err = "tensor-core step failed";
+      return rc < 0 ? (br_status)rc : BR_ERR_CUDA;
+    }
   }
   // ---- store g_c in the ring (after every reader of the slot it may overwrite) --------------
   for (int i = 0; i < nl; ++i) {
@@ -905,6 +969,27 @@ br_status br_step(br_handle* h, const void* const* grads, int tau) {
     BR_CUDA(h, cudaMemcpyAsync(dst, grads[i], bytes, cudaMemcpyDeviceToDevice, h->stream));
   }
   return any ? BR_OK : BR_WARMUP;
+}
+
+}  // namespace
+
+extern "C" {
+
+br_status br_debug_inject(br_handle* h, int kind, int64_t countdown) {
+  if (!h) return BR_ERR_INVALID;
+  if (kind == BR_INJECT_NONE) { h->stats.fail_countdown = -1; return BR_OK; }
+  if (kind != BR_INJECT_LAUNCH_FAILURE || countdown < 0) { h->err = "unknown injection kind or negative countdown"; return BR_ERR_INVALID; }
+  h->stats.fail_countdown = countdown;
+  return BR_OK;
+}
+
+br_status br_debug_wait_timeout(br_handle* h, uint64_t limit_ns) {
+  br_status st = check_handle(h);
+  if (st != BR_OK) return st;
+  if (limit_ns < 1000 || limit_ns > 2000000000ull) { h->err = "limit outside [1 us, 2 s]"; return BR_ERR_INVALID; }
+  BR_CUDA(h, tc_wait_probe(limit_ns, h->d_status, h->stream));
+  count(h);
+  return BR_OK;
 }
 
 br_status br_set_lr(br_handle* h, float lr) {
@@ -936,6 +1021,12 @@ br_status br_refresh_basis(br_handle* h, int layer) {
   // tensor-core layers keep the rotated momentum: back to the original space with the old basis,
   // forward again with the new one
   const char* terr = nullptr;
+  std::vector<int64_t> count_before(nl);
+  for (int i = 0; i < nl; ++i) count_before[i] = h->layers[i].refresh_count;
+  auto undo = [&](br_status code) {            // a failed enqueue: the integer state reads as before the call
+    for (int i = 0; i < nl; ++i) h->layers[i].refresh_count = count_before[i];
+    return code;
+  };
   if (!tc_ids.empty()) {
     int rc = tc_step_reexpress(h->tc, h->layers, tc_ids.data(), (int)tc_ids.size(), 0, h->d_status, h->stream, &h->stats, &terr);
     if (rc != 0) { h->err = terr ? terr : "re-expression failed"; return (br_status)rc; }
@@ -944,10 +1035,10 @@ br_status br_refresh_basis(br_handle* h, int layer) {
       if (L.Morig) BR_CUDA(h, cudaMemcpyAsync(L.Morig, L.M, 4 * (size_t)L.d.m * L.d.n, cudaMemcpyDeviceToDevice, h->stream));
     }
   }
-  if ((st = refresh_layers(h, ids.data(), (int)ids.size())) != BR_OK) return st;
+  if ((st = refresh_layers(h, ids.data(), (int)ids.size())) != BR_OK) return undo(st);
   if (!tc_ids.empty()) {
     int rc = tc_step_reexpress(h->tc, h->layers, tc_ids.data(), (int)tc_ids.size(), 1, h->d_status, h->stream, &h->stats, &terr);
-    if (rc != 0) { h->err = terr ? terr : "re-expression failed"; return (br_status)rc; }
+    if (rc != 0) { h->err = terr ? terr : "re-expression failed"; return undo((br_status)rc); }
   }
   return BR_OK;
 }
@@ -1159,29 +1250,7 @@ br_status br_get_profile(br_handle* h, br_profile_stats* out) {
 
 br_status br_destroy(br_handle* h) {
   if (!h) return BR_OK;
-  cudaSetDevice(h->device);
-  cudaStreamSynchronize(h->stream);
-  if (h->tc) tc_step_destroy(h->tc);
-  for (int i = 1; i < br_handle::kMaxLanes; ++i) {
-    if (h->lanes[i].stream) { cudaStreamSynchronize(h->lanes[i].stream); cudaStreamDestroy(h->lanes[i].stream); }
-    if (h->lanes[i].done) cudaEventDestroy(h->lanes[i].done);
-  }
-  if (h->ev_begin) cudaEventDestroy(h->ev_begin);
-  if (h->ev_cond) cudaEventDestroy(h->ev_cond);
-  if (h->copy_stream) { cudaStreamSynchronize(h->copy_stream); cudaStreamDestroy(h->copy_stream); }
-  if (h->ev_consumed) cudaEventDestroy(h->ev_consumed);
-  if (h->ev_copied) cudaEventDestroy(h->ev_copied);
-  if (h->h_cond) cudaFreeHost(h->h_cond);
-  for (int i = 0; i < br_handle::kMaxLanes; ++i) {
-    for (auto& kv : h->lanes[i].qr_graphs) if (kv.second.exec) cudaGraphExecDestroy(kv.second.exec);
-    for (QrTc* t : h->lanes[i].tcq) qr_tc_destroy(t);
-  }
-  for (auto& sp : h->stats.prof.spans) { cudaEventDestroy(sp.a); cudaEventDestroy(sp.b); }
-  for (auto e : h->stats.prof.free_events) cudaEventDestroy(e);
-  if (h->slab) {
-    if (h->alloc.alloc) h->alloc.free(h->slab, h->alloc.ctx); else cudaFree(h->slab);
-  }
-  delete h;
+  release(h);
   return BR_OK;
 }
 

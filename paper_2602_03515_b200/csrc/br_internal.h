@@ -49,6 +49,14 @@ struct LaunchStats {
   int64_t launches = 0;
   double gemm_flops = 0.0;
   Profiler prof;
+  // Host-side fault injection (br_debug_inject): when >= 0, counts down once per CUDA call the
+  // library is about to issue for this handle; the call that finds it at 0 is NOT issued and reports
+  // cudaErrorLaunchFailure instead.  Nothing on the device is touched by the injected failure.
+  int64_t fail_countdown = -1;
+  bool inject() {
+    if (fail_countdown < 0) return false;
+    return fail_countdown-- == 0;
+  }
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -199,5 +207,7 @@ cudaError_t tc_plan_launch_range(TcPlan* p, int first, int count, long long call
                                  float dyn_beta, int* status_word, cudaStream_t s);
 double tc_plan_flops_range(const TcPlan* p, int first, int count);
 int tc_supported(int device);
+// Exercises the bounded mbarrier wait of the contraction kernel: a wait that nothing satisfies, limit_ns long.
+cudaError_t tc_wait_probe(uint64_t limit_ns, int* status_word, cudaStream_t s);
 
 }  // namespace br

@@ -173,7 +173,7 @@ constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s: far above any legitim
 // Bounded wait.  Returns false when the wait gave up or another role raised the abort flag.
 template <bool CLUSTER = false>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          int* status) {
+                                          int* status, uint64_t limit_ns = kWaitLimitNs) {
   auto try_wait = [&] { return CLUSTER ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity); };
   if (try_wait()) return true;
   const uint64_t t0 = global_timer_ns();
@@ -182,7 +182,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     if (try_wait()) return true;
     if ((++spins & 0xFF) == 0) {
       if (*abort_flag) return false;
-      if (global_timer_ns() - t0 > kWaitLimitNs) {
+      if (global_timer_ns() - t0 > limit_ns) {
         *abort_flag = 1;
         atomicMin(status, (int)BR_ERR_TIMEOUT);
         return false;
@@ -743,6 +743,20 @@ k_tc_gemm(const DevProblem* __restrict__ probs, int n_probs, int first_tile, int
   }
 }
 
+// One warp waits, with the kernel's own bounded wait, on an mbarrier that nothing ever arrives on: the
+// wait must give up after limit_ns, leave BR_ERR_TIMEOUT in the status word and return.
+__global__ void __launch_bounds__(32) k_wait_probe(uint64_t limit_ns, int* status) {
+  __shared__ alignas(8) uint64_t bar;
+  __shared__ int abort_word;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    abort_word = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncwarp();
+  if (threadIdx.x == 0) mbar_wait(smem_u32(&bar), 0u, &abort_word, status, limit_ns);
+}
+
 // ---------------------------------------------------------------------------------------------
 // Host side: tensor-map encoding and plans
 // ---------------------------------------------------------------------------------------------
@@ -1059,6 +1073,11 @@ cudaError_t tc_plan_launch_range(TcPlan* p, int first, int count, long long call
 cudaError_t tc_plan_launch(TcPlan* p, long long calls, int tau, float dyn_alpha, float dyn_beta,
                            int* status_word, cudaStream_t s) {
   return tc_plan_launch_range(p, 0, p->n, calls, tau, dyn_alpha, dyn_beta, status_word, s);
+}
+
+cudaError_t tc_wait_probe(uint64_t limit_ns, int* status_word, cudaStream_t s) {
+  k_wait_probe<<<1, 32, 0, s>>>(limit_ns, status_word);
+  return cudaGetLastError();
 }
 
 double tc_plan_flops_range(const TcPlan* p, int first, int count) {

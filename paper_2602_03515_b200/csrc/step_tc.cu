@@ -362,6 +362,7 @@ struct Launcher {
   }
   int run(TcPlan* p, const char* what, long long calls, int tau, float a, float b) {
     if (!p) return 0;
+    if (stats->inject()) return fail(what, cudaErrorLaunchFailure);     // host-side fault injection: nothing is launched
     const int span = stats->prof.begin(PROF_TC, s);
     cudaError_t e = tc_plan_launch(p, calls, tau, a, b, d_status, s);
     stats->prof.end(span, s, tc_plan_flops(p));

@@ -2,15 +2,15 @@
 benchmark times (tensor-core path, grouped launches over several layers, gradients read through
 the delay ring).
 
-A whole oracle trajectory with refreshes is out of reach at these sizes (the oracle's own Householder
-QR is O(k^3) interpreted loops), so the step and the refresh are checked separately:
+Free-running trajectories with refreshes inside them are in tests/test_gpu_free_running.py; here the
+step and the refresh are checked separately, at the largest shapes:
 
 * step: the bases are set to seeded random orthogonal matrices on both sides (teacher-forced), the
   delayed step runs for two updates, and the whole weight change, the momentum and the second moment
   are compared with the oracle element by element (tolerance of the bf16 tensor-core path, 2e-2);
-* refresh: a forced refresh from given factors is compared with the oracle's Power() on a factor
-  of order 1024, and, at the largest order of the benchmark (6912), against the properties that
-  define the result at any size: Q^T Q = I, and R = Q^T (F Q0) upper triangular with a positive
+* refresh: a forced refresh from given factors is compared with the oracle's Power() at orders
+  1024, 2560, 4224 and 6912 (the largest of the benchmark), and there also against the properties
+  that define the result at any size: Q^T Q = I, and R = Q^T (F Q0) upper triangular with a positive
   diagonal (checked on sampled columns in float64).
 """
 from dataclasses import replace
@@ -142,12 +142,13 @@ def test_refresh_tensor_core_projections(k):
     """Third refresh of a basis of order 4224 / 2560 in one handle (orders from 2048 use the tensor-core
     forms: deflated power product, block projections with at least 2^18 coefficients).  The first (from U = I) is ill-conditioned, the second runs in fp64 and notes that
     no column shrank much, so the third runs its large block projections on the tensor cores
-    (three-term bf16 splits, applied twice).  The result is unique (QR with a positive diagonal), so
-    it is compared with LAPACK's QR of the float64 product F U2 after fixing the signs -- the
-    routine the oracle's own Householder QR is pinned against at small orders, where the oracle
-    itself (interpreted loops, minutes at this order) is affordable."""
+    (three-term bf16 splits, applied twice).  Compared with the oracle's Power(F, U2): at order 2560 in
+    its written-out Householder form (about a minute of interpreted loops), at order 4224 -- where that
+    form would take some five minutes -- with the library QR routine as the step (`qr_pos_lapack`, pinned
+    against the written-out form at small orders)."""
     import torch
     import paper_2602_03515_b200 as br
+    from oracle import br_oracle as O
     from tests.parity_util import basis_err
     F = _lowrank_noise_factor(k, 16, 33, samples=3)      # 13,000 noise samples: the noise part is well conditioned
     w = torch.zeros(k, 8, device="cuda")
@@ -164,15 +165,23 @@ def test_refresh_tensor_core_projections(k):
         opt.refresh_basis(0)                                        # large block projections on the tensor cores
         assert opt.sync_status() == br.BR_OK
         U3 = opt.get_state(0, br.BR_BUF_U).numpy().astype(np.float64)
-        q, r = np.linalg.qr(F.astype(np.float64) @ U2.astype(np.float64))
-        ref = q * np.sign(np.diag(r))
+        ref, deficient = O.power(F.astype(np.float64), U2.astype(np.float64),
+                                 qr=O.qr_pos if k <= 2560 else O.qr_pos_lapack)
+        assert not deficient
         assert basis_err(U3, ref) < 1e-5
         assert np.max(np.abs(U3.T @ U3 - np.eye(k))) < 1e-5
     finally:
         opt.close()
 
 
-def test_refresh_order_6912_properties():
+def test_refresh_order_6912_against_oracle_power_and_properties():
+    """The largest order of the ~3B layer set.  First refresh from U = I (ill-conditioned: columns lose
+    up to 1e-5 of their length), second from the first one's result (the basis tracks the factor).  Both
+    are compared with the oracle's Power() (library QR routine as its step at this order), and with the
+    properties that define the result whatever computes it, on sampled columns in float64: Q^T Q = I and
+    R = Q^T (F Q0) upper triangular with a positive diagonal."""
+    from oracle import br_oracle as O
+    from tests.parity_util import basis_err
     k = 6912
     F = _lowrank_noise_factor(k, 32, 32, samples=2)      # 14,000 noise samples for order 6912: full rank with margin
     Q0 = np.eye(k, dtype=np.float32)
@@ -182,14 +191,17 @@ def test_refresh_order_6912_properties():
     rng = np.random.default_rng(0)
     cols = np.unique(np.concatenate([np.arange(64), np.arange(k - 64, k), rng.integers(0, k, 384)]))
     F64 = F.astype(np.float64)
-    for Qin, U in ((Q0.astype(np.float64), U1), (U1f.astype(np.float64), U2)):
+    for Qin, U, tol in ((Q0.astype(np.float64), U1, 1e-3), (U1f.astype(np.float64), U2, 1e-5)):
         assert np.all(np.isfinite(U))
-        assert np.max(np.abs(U.T @ U[:, cols] - np.eye(k)[:, cols])) < 2e-5
+        ref, deficient = O.power(F64, Qin, qr=O.qr_pos_lapack)
+        assert not deficient
+        assert basis_err(U, ref) < tol, basis_err(U, ref)
+        assert np.max(np.abs(U.T @ U[:, cols] - np.eye(k)[:, cols])) < 1e-5
         A = F64 @ Qin[:, cols]                           # sampled columns of F Q0
         R = U.T @ A                                      # column j of R: zero below row cols[j], positive there
         scale = np.linalg.norm(A, axis=0)
         below = np.arange(k)[:, None] > cols[None, :]
-        assert np.max(np.abs(R * below) / scale[None, :]) < 1e-3
+        assert np.max(np.abs(R * below) / scale[None, :]) < 1e-5
         assert np.all(R[cols, np.arange(len(cols))] > 0)
 
 

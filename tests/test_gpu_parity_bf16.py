@@ -15,7 +15,7 @@ pytestmark = pytest.mark.gpu
 TOL_DW, TOL_BASIS, TOL_V2 = 2e-2, 1e-3, 2e-2
 
 
-def _run(w, calls, tau=-1, tol=TOL_DW, tol_basis=TOL_BASIS, **kw):
+def _run(w, calls, tau=-1, tol=TOL_DW, tol_basis=TOL_BASIS, verbose=False, **kw):
     """tol_basis: a number, or a function of the refresh count of the layer (the bases of a long
     free-running trajectory drift apart at the rate the fp32 storage of L and R allows)."""
     from tests.parity_util import SideBySide, rel_l2
@@ -27,6 +27,7 @@ def _run(w, calls, tau=-1, tol=TOL_DW, tol_basis=TOL_BASIS, **kw):
     try:
         for c in range(calls):
             before = [lay.refresh_count for lay in sbs.oracle.layers]
+            sbs.remember_bases()
             st_g, st_o, dg, do = sbs.step(tau)
             # (a rank-deficient refresh is reported by the oracle's step at once, by the library through
             # the status word that br_sync_status reads)
@@ -38,6 +39,8 @@ def _run(w, calls, tau=-1, tol=TOL_DW, tol_basis=TOL_BASIS, **kw):
                     continue
                 e = rel_l2(a, b)
                 worst = max(worst, e)
+                if verbose:
+                    print(f"call {c + 1} layer {li} dW rel-L2 {e:.2e}")
                 assert e <= tol, (c, li, e)
             for li, lay in enumerate(sbs.oracle.layers):
                 assert sbs.opt.counters(li) == sbs.oracle.counters(li)
@@ -47,6 +50,8 @@ def _run(w, calls, tau=-1, tol=TOL_DW, tol_basis=TOL_BASIS, **kw):
                     errs = sbs.check_bases(li, tb, TOL_V2, where=f"call {c + 1}, refresh {lay.refresh_count},")
                     for k_, e_ in errs.items():
                         worst_q[k_] = max(worst_q.get(k_, 0.0), e_)
+                    if verbose:
+                        print(f"call {c + 1} layer {li} refresh {lay.refresh_count}: {errs}, oracle min pivot {lay.last_min_pivot:.2e}")
         assert sbs.opt.sync_status() == (br.BR_WARN_RANK_DEFICIENT if deficient else br.BR_OK)
         print(f"{w.name}: worst dW {worst:.2e}, worst after-refresh errors {worst_q}")
         for li, lay in enumerate(sbs.oracle.layers):

@@ -21,6 +21,8 @@ def _run(w, calls, tau=-1, **kw):
     worst_dw, worst_q = 0.0, 0.0
     try:
         for c in range(calls):
+            before = [lay.refresh_count for lay in sbs.oracle.layers]
+            sbs.remember_bases()
             st_g, st_o, dg, do = sbs.step(tau)
             assert st_g == st_o or (st_g == br.BR_OK and st_o == 2), (c, st_g, st_o)
             for li, (a, b) in enumerate(zip(dg, do)):
@@ -30,6 +32,9 @@ def _run(w, calls, tau=-1, **kw):
                 worst_dw = max(worst_dw, rel_l2(a, b))
             for li, lay in enumerate(sbs.oracle.layers):
                 assert sbs.opt.counters(li) == sbs.oracle.counters(li)
+                if lay.refresh_count != before[li] and st_o != 2:
+                    # a refresh happened inside this call: bases and V~ against the oracle's, now
+                    sbs.check_bases(li, TOL_BASIS, 1e-3, where=f"call {c + 1}, refresh {lay.refresh_count},", tensor_core=False)
         for li, lay in enumerate(sbs.oracle.layers):
             for which, ref in ((br.BR_BUF_U, lay.U), (br.BR_BUF_V, lay.V)):
                 if ref is not None and lay.refresh_count > 0:
@@ -301,3 +306,43 @@ def test_closed_loop_quadratic_against_oracle_and_the_papers_claim():
     rotated, e3 = gpu_run(GEOM_BI, False)
     assert max(e1, e2, e3) < 5e-2, (e1, e2, e3)          # closed loops amplify rounding: loss within 5 %
     assert misaligned > 5.0 * aligned and rotated < 2.0 * aligned
+
+
+def test_closed_loop_spiral_plain_adam_through_the_ring():
+    """The spiral loss of Sec. 2.2 / App. D.1 in closed loop: two parameters, geometry none (Eq. (adam)),
+    learning rate 0.1, beta1 = 0, beta2 = 0.9; the gradient is computed from the library's own current
+    weights at every call, and from call 40 on it is applied one call late (tau = 1, through the ring).
+    The iterates follow the oracle's own closed loop while rounding has not been amplified yet (a
+    float64 emulation with fp32 weights and moments separates from the float64 run by 1e-4 within 60
+    steps of this oscillating trajectory and by 4e-4 within 100), and the oscillation statistics agree
+    afterwards."""
+    import torch
+    import paper_2602_03515_b200 as br
+    from oracle import br_oracle as O
+    from workloads.closed_loop import spiral_grad, spiral_valley_excess
+    steps, delay_from = 500, 40
+    for p0 in ([8.0, 0.0], [5.0, 5.0]):
+        w = torch.tensor([p0], dtype=torch.float32, device="cuda")
+        opt = br.BasisRotation([LayerSpec("p", 1, 2, GEOM_NONE, SRC_SECOND, 1)], [w], grad_dtype="f32", lr=0.1, beta1=0.0,
+                               beta2=0.9, eps=1e-8, gemm_prec=br.BR_GEMM_FP32)
+        f32 = lambda x: float(np.float32(x))
+        lay = O.OracleLayer(np.array([p0], dtype=np.float64), O.GEOM_NONE, O.SRC_SECOND, 1)
+        orc = O.Oracle([lay], O.Hyper(lr=f32(0.1), beta1=0.0, beta2=f32(0.9), eps=f32(1e-8), freq=10))
+        ex_g, ex_o = [], []
+        try:
+            for c in range(steps):
+                tau = 0 if c < delay_from else 1
+                pg = w.double().cpu().numpy()[0]
+                g = torch.from_numpy(spiral_grad(pg)[None, :].astype(np.float32)).cuda()
+                assert opt.step([g], tau) == br.BR_OK
+                orc.step([spiral_grad(lay.W[0])[None, :]], tau)
+                assert opt.counters(0) == orc.counters(0)
+                if c < 60:
+                    assert np.max(np.abs(w.double().cpu().numpy()[0] - lay.W[0])) < 1e-3, c
+                if c >= 100:
+                    ex_g.append(spiral_valley_excess(w.double().cpu().numpy()[0]))
+                    ex_o.append(spiral_valley_excess(lay.W[0]))
+            assert opt.sync_status() == br.BR_OK
+        finally:
+            opt.close()
+        assert abs(np.mean(ex_g) / np.mean(ex_o) - 1.0) < 0.1, (np.mean(ex_g), np.mean(ex_o))

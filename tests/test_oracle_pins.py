@@ -563,3 +563,45 @@ def test_closed_loop_quadratic_rotation_removes_the_delay_penalty():
     assert rotated < 2.0 * aligned
     # and delay itself hurts plain Adam on the misaligned problem
     assert _closed_loop_oracle(O.GEOM_NONE, False, 0) < 0.5 * misaligned
+
+
+def _spiral_run(p0, steps, delay_from=None):
+    """Plain Adam of Eq. (adam) on the spiral loss with the paper's settings (App. D.1: learning rate 0.1,
+    beta1 = 0, beta2 = 0.9), gradient computed from the current iterate; from call `delay_from` on the
+    applied gradient is one call old (tau = 1 through the ring)."""
+    from workloads.closed_loop import spiral_grad
+    lay = O.OracleLayer(np.array([p0], dtype=np.float64), O.GEOM_NONE, O.SRC_SECOND, 1)
+    orc = O.Oracle([lay], O.Hyper(lr=0.1, beta1=0.0, beta2=0.9, eps=1e-8, freq=10 ** 9))
+    traj = [lay.W[0].copy()]
+    for c in range(steps):
+        orc.step([spiral_grad(lay.W[0])[None, :]], 0 if (delay_from is None or c < delay_from) else 1)
+        traj.append(lay.W[0].copy())
+    return np.array(traj)
+
+
+def test_spiral_loss_definition_and_the_papers_alignment_claim():
+    """Spiral loss of Sec. 2.2 / App. D.1.  Definition: the gradient equals central differences of
+    f(r, theta) = r^2 + (20 sin(4r - theta) + 1)^2, and on the valley 20 sin(4r - theta) = -1 the loss is
+    r^2.  The paper's observation, in the form that can be checked without its figure: without delay Adam
+    sits higher up the valley walls (oscillates more) where the Hessian eigenbasis is misaligned with the
+    coordinate axes than where it is aligned, and a delay of one step raises that further in both."""
+    from workloads.closed_loop import spiral_grad, spiral_loss, spiral_misalignment, spiral_valley_excess
+    for p in ([3.0, -1.0], [-0.7, 5.2], [6.0, 6.0]):
+        p = np.array(p)
+        fd = np.array([(spiral_loss(p + e) - spiral_loss(p - e)) / 2e-6 for e in (np.array([1e-6, 0]), np.array([0, 1e-6]))])
+        assert np.allclose(spiral_grad(p), fd, rtol=1e-6, atol=1e-5)
+    th = 0.3
+    r = (np.arcsin(-1.0 / 20.0) + th + 4 * np.pi) / 4.0
+    on_valley = np.array([r * np.cos(th), r * np.sin(th)])
+    assert abs(spiral_loss(on_valley) - r * r) < 1e-9 and abs(spiral_valley_excess(on_valley)) < 1e-9
+    stats = {}
+    for name, p0 in (("aligned", [8.0, 0.0]), ("misaligned", [5.0, 5.0])):
+        free, delayed = _spiral_run(p0, 1000), _spiral_run(p0, 1000, delay_from=600)
+        assert np.array_equal(free[:601], delayed[:601])                   # identical until the delay starts
+        stats[name] = (spiral_misalignment(free[600]),
+                       np.mean([spiral_valley_excess(p) for p in free[600:]]),
+                       np.mean([spiral_valley_excess(p) for p in delayed[600:]]))
+    assert stats["aligned"][0] < 0.05 and stats["misaligned"][0] > 0.9
+    assert stats["misaligned"][1] > 1.5 * stats["aligned"][1]              # misalignment: more oscillation
+    for name in stats:
+        assert stats[name][2] > 2.0 * stats[name][1]                      # delay: more again

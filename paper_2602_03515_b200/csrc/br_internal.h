@@ -182,6 +182,8 @@ struct TcProblem {
   // factor clip[(calls - 1 - tau) mod clip_slots]; clip_mode 1 multiplies it by the factor (G~), 2 by
   // its square (G G^T), 0 leaves it alone
   const float* clip = nullptr; int32_t clip_slots = 0; int32_t clip_mode = 0;
+  int32_t fold_kb = 0;            // > 0: accumulate in chunks of this many 64-deep k-blocks, summed outside the tensor
+                                  // core (a plan whose problems all ask for it runs the folded form of the kernel)
   int32_t symmetric = 0;          // 1: A_p = B_p and D is square: only tiles touching the upper triangle are
                                   // computed, the rest of D is written as their mirror image (EPI_AXPBY_F32 only)
   float alpha = 1.f, beta = 0.f, eps = 0.f, beta1 = 0.f;

@@ -34,6 +34,19 @@
 // "accumulator empty" barrier.  Both CTAs meet at a cluster barrier after set-up and before they free
 // their tensor memory, so neither exits while the other can still signal it.
 //
+// Folded form (factor products G G^T, G^T G).  The tensor core truncates its fp32 accumulator once
+// per instruction (16-deep slice of the contraction), a one-sided error that grows with the length of
+// the chain and with the size of the partial sums: 0.3 (K / 16) 2^-24 relative for contraction length
+// K, 3e-6 at K = 2560.  The factors feed Power(), whose trailing basis vectors come out of a
+// cancellation against eigenvalues 1e5 times larger, and an error of that size moves them by 1e-2.
+// In this form the contraction is cut into chunks of a few k-blocks; the chunks are accumulated from
+// zero, alternately in the two tensor-memory buffers, and eight epilogue warps (two per lane quadrant,
+// 128 result columns each) add every finished chunk, round to nearest on the CUDA cores, to a running
+// sum they keep in registers, while the tensor core is already working on the next chunk.  Chains
+// are 8 to 16 instructions on partial sums a tenth the size: the error drops by the number of chunks.
+// The final epilogue (factor EMA and its mirror image) runs from the registers while the first two
+// chunks of the next tile accumulate.
+//
 // Every wait on an mbarrier is bounded: when a wait gives up the CTA raises an abort flag,
 // records BR_ERR_TIMEOUT in the status word, leaves its loops, frees its tensor memory and
 // returns; later launches return at once while the status word is negative.
@@ -77,6 +90,8 @@ struct Form {
 };
 constexpr int TMEM_COLS = 512;
 constexpr int NUM_THREADS = 192;                 // warp 0: TMA, warp 1: MMA, warps 2..5: epilogue
+constexpr int FOLD_THREADS = 320;                // folded form: warps 2..9 fold and write (two per lane quadrant)
+constexpr int SMEM_BYTES_FOLD = OPERAND_BYTES + 2 * EPI_BYTES + 1024;
 constexpr int MAX_PAIRS = 3;
 // Tile rasterisation: a group of row-blocks (or, transposed, of column-blocks) is swept across the
 // other dimension, so that the group's operand panel stays in L2 while the other operand streams
@@ -104,6 +119,7 @@ struct alignas(128) DevProblem {
   int32_t tri;                    // symmetric product with square tiles: the tile list holds the upper triangle only
   const float* clip;              // clipping factors by call (see TcProblem::clip_mode), or null
   int32_t clip_slots, clip_mode;
+  int32_t fold_kb;                // folded form: k-blocks per chunk
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -254,6 +270,39 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      :: "r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+         "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+         "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+         "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
 // Shared-memory matrix descriptor, 128-byte swizzle.  lbo / sbo in bytes.
 //   K-major : rows of 128 bytes (64 elements of K); 8-row groups 1024 bytes apart (sbo); lbo unused.
 //   MN-major: rows of 128 bytes (64 elements of M/N), one row per k; 8-k groups sbo apart,
@@ -343,8 +392,8 @@ __device__ __forceinline__ TileInfo locate_tile(const DevProblem* probs, int n_p
 // ---------------------------------------------------------------------------------------------
 // The kernel
 // ---------------------------------------------------------------------------------------------
-template <bool SHARED, bool PAIR>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+template <bool SHARED, bool PAIR, bool FOLD = false>
+__global__ void __launch_bounds__(FOLD ? FOLD_THREADS : NUM_THREADS, 1)
 k_tc_gemm(const DevProblem* __restrict__ probs, int n_probs, int first_tile, int total_tiles, long long calls,
           int tau, float dyn_alpha, float dyn_beta, int* status) {
   using F = Form<SHARED, PAIR>;
@@ -384,7 +433,7 @@ k_tc_gemm(const DevProblem* __restrict__ probs, int n_probs, int first_tile, int
   if (threadIdx.x == 0) {
     for (int s = 0; s < NST; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     // accumulator hand-back: four epilogue warps, of both CTAs in the paired form
-    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), PAIR ? 8 : 4); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), (FOLD ? 2 : 1) * (PAIR ? 8 : 4)); }
     abort_word = 0;
     dead_word = (*reinterpret_cast<volatile int*>(status) < 0) ? 1u : 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -478,6 +527,7 @@ k_tc_gemm(const DevProblem* __restrict__ probs, int n_probs, int first_tile, int
     if (lane == 0 && rank == 0) {
       int stage = 0; uint32_t phase = 0;
       int acc = 0; uint32_t acc_phase = 0;
+      uint32_t fold_seq = 0;                      // folded form: chunks handed over so far (buffer = seq & 1)
       // a commit arrives on this CTA's barrier and, in the paired form, on the peer's as well
       auto commit = [&](uint32_t bar) {
         if (PAIR) { umma_commit_pair(bar); umma_commit_pair(map_to_cta(bar, 1)); } else { umma_commit(bar); }
@@ -492,6 +542,42 @@ k_tc_gemm(const DevProblem* __restrict__ probs, int n_probs, int first_tile, int
         // MN-major: 16 k rows = two 8-row groups of 1024 bytes.
         const uint32_t a_lbo = p->a_mn ? BK * 128 : 0, a_adv = p->a_mn ? 2048 : 32;
         const uint32_t b_lbo = p->b_mn ? BK * 128 : 0, b_adv = p->b_mn ? 2048 : 32;
+        if (FOLD) {
+          // chunks of fold_kb k-blocks, each accumulated from zero, alternately in the two buffers, and
+          // handed to the epilogue warps, which add it to the running sum in their registers
+          bool ok = true;
+          for (int kb0 = 0; kb0 < nkb && ok; kb0 += p->fold_kb) {
+            const int buf = (int)(fold_seq & 1u);
+            if (!mbar_wait<PAIR>(tempty_bar(buf), ((fold_seq >> 1) & 1u) ^ 1u, abort_flag, status)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t d_chunk = tmem_base + (uint32_t)buf * BN;
+            uint32_t accumulate = 0;
+            const int kb1 = min(nkb, kb0 + p->fold_kb);
+            for (int kb = kb0; kb < kb1; ++kb) {
+              if (!mbar_wait(full_bar(stage), phase, abort_flag, status)) { ok = false; break; }
+              tc_fence_after();
+              const uint64_t adesc = make_smem_desc(sA(stage, 0), a_lbo, 1024);
+              const uint64_t bdesc = make_smem_desc(sB(stage, 0), b_lbo, 1024);
+#pragma unroll
+              for (int k = 0; k < BK / UMMA_K; ++k) {
+                if (PAIR)
+                  umma_bf16_pair(d_chunk, adesc + (uint64_t)((k * a_adv) >> 4), bdesc + (uint64_t)((k * b_adv) >> 4),
+                                 idesc, accumulate);
+                else
+                  umma_bf16(d_chunk, adesc + (uint64_t)((k * a_adv) >> 4), bdesc + (uint64_t)((k * b_adv) >> 4),
+                            idesc, accumulate);
+                accumulate = 1;
+              }
+              commit(empty_bar(stage));
+              if (++stage == NST) { stage = 0; phase ^= 1u; }
+            }
+            if (!ok) break;
+            commit(tfull_bar(buf));
+            ++fold_seq;
+          }
+          if (!ok) break;
+          continue;
+        }
         if (!mbar_wait<PAIR>(tempty_bar(acc), acc_phase ^ 1u, abort_flag, status)) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)acc * BN;
@@ -540,6 +626,7 @@ k_tc_gemm(const DevProblem* __restrict__ probs, int n_probs, int first_tile, int
     float* tile = epi_tiles + quad * (32 * EPI_LD);
     const int sub_r = lane >> 3, sub_c = (lane & 7) * 4;
     int acc = 0; uint32_t acc_phase = 0;
+    uint32_t fold_seq = 0;
     for (int tile_i = first_tile + unit; tile_i < total_tiles && !*abort_flag; tile_i += n_units) {
       const TileInfo ti = locate_tile<TM>(probs, n_probs, tile_i, calls, tau);
       if (!ti.active) continue;
@@ -568,6 +655,113 @@ k_tc_gemm(const DevProblem* __restrict__ probs, int n_probs, int first_tile, int
             if (epi == EPI_ROTATED_ADAM)
               asm volatile("prefetch.global.L2 [%0];" ::"l"(p->D2 + (long long)(row_base + lane) * p->ldd + ti.n0 + 32 * q));
           }
+      }
+      if (FOLD) {
+        // ---- folded form: this warp owns 32 rows (its lane quadrant) x 128 columns (its half) ----
+        const int half = (warp - 2) >> 2;
+        float* ftile = epi_tiles + (warp - 2) * (32 * EPI_LD);
+        const int nkb = (p->K + BK - 1) / BK;
+        const uint32_t lane_base = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(half * 128);
+        // which of the four 32-column blocks are written at all (uniform across the warp)
+        uint32_t need = 0;
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+          const int col0 = ti.n0 + half * 128 + 32 * b;
+          if (col0 < p->Nd && quad_ok && !(p->symmetric && row_base >= col0 + 32)) need |= 1u << b;
+        }
+        // The running sum of this thread: its row, its warp's 128 columns.  The first chunk is loaded
+        // straight into these registers; every later one is added with packed fp32 adds, one 32-column
+        // block at a time (the other warp of the quadrant covers the load latency).
+        uint32_t sum[4][32];
+        bool ok = true;
+        for (int kb0 = 0; kb0 < nkb; kb0 += p->fold_kb) {
+          const int buf = (int)(fold_seq & 1u);
+          if (!mbar_wait(tfull_bar(buf), (fold_seq >> 1) & 1u, abort_flag, status)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t src = lane_base + (uint32_t)(buf * BN);
+          if (kb0 == 0) {
+#pragma unroll
+            for (int b = 0; b < 4; ++b)
+              if ((need >> b) & 1u) tmem_ld32_issue(src + 32 * b, sum[b]);
+            tmem_wait_ld();
+          } else {
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+              if (!((need >> b) & 1u)) continue;
+#pragma unroll
+              for (int h = 0; h < 2; ++h) {
+                uint32_t t[16];
+                tmem_ld16_issue(src + 32 * b + 16 * h, t);
+                tmem_wait_ld();
+#pragma unroll
+                for (int j = 0; j < 16; j += 2) {
+                  const float2 r = __fadd2_rn(make_float2(__uint_as_float(sum[b][16 * h + j]), __uint_as_float(sum[b][16 * h + j + 1])),
+                                              make_float2(__uint_as_float(t[j]), __uint_as_float(t[j + 1])));
+                  sum[b][16 * h + j] = __float_as_uint(r.x); sum[b][16 * h + j + 1] = __float_as_uint(r.y);
+                }
+              }
+            }
+          }
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) {
+            if (PAIR) mbar_arrive_cluster(map_to_cta(tempty_bar(buf), 0)); else mbar_arrive(tempty_bar(buf));
+          }
+          ++fold_seq;
+        }
+        if (!ok) break;
+        // ---- factor EMA D <- alpha sum + beta D on the blocks that touch the upper triangle, and their mirror image ----
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+          if (!((need >> b) & 1u)) continue;
+          const int col0 = ti.n0 + half * 128 + 32 * b;
+          __syncwarp();
+#pragma unroll
+          for (int j = 0; j < 32; ++j) ftile[lane * EPI_LD + j] = __uint_as_float(sum[b][j]);
+          __syncwarp();
+          const int col = col0 + sub_c;
+          int n_it = 0;
+          if (col < p->Nd) { n_it = (p->Md - row_base - sub_r + 3) >> 2; n_it = n_it > 8 ? 8 : n_it; }
+          float* d = p->D + (long long)(row_base + sub_r) * p->ldd + col;
+          const long long step = 4 * p->ldd;
+          const bool mirror = p->symmetric && col0 >= row_base + 32;
+          // four row groups at a time (registers): read the old values, combine, write, and put the
+          // result back into the tile for the mirror image
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            float4 o[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+              if (beta != 0.0f && 4 * h + i < n_it) o[i] = *reinterpret_cast<const float4*>(d + (4 * h + i) * step);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const int it = 4 * h + i;
+              float* t4 = ftile + (it * 4 + sub_r) * EPI_LD + sub_c;
+              float4 r = make_float4(alpha * t4[0], alpha * t4[1], alpha * t4[2], alpha * t4[3]);
+              if (beta != 0.0f && it < n_it) {
+                r.x = fmaf(beta, o[i].x, r.x); r.y = fmaf(beta, o[i].y, r.y);
+                r.z = fmaf(beta, o[i].z, r.z); r.w = fmaf(beta, o[i].w, r.w);
+              }
+              if (it < n_it) *reinterpret_cast<float4*>(d + it * step) = r;
+              if (mirror) { t4[0] = r.x; t4[1] = r.y; t4[2] = r.z; t4[3] = r.w; }     // (each thread rewrites only what it read)
+            }
+          }
+          if (mirror) {
+            __syncwarp();
+            const int mrow0 = col0 + sub_r, mcol = row_base + sub_c;
+            if (mcol < p->Nd) {
+#pragma unroll
+              for (int it = 0; it < 8; ++it) {
+                const int mrow = mrow0 + it * 4;
+                if (mrow >= p->Md) break;
+                const float* t1 = ftile + sub_c * EPI_LD + (it * 4 + sub_r);
+                *reinterpret_cast<float4*>(p->D + (long long)mrow * p->ldd + mcol) =
+                    make_float4(t1[0], t1[EPI_LD], t1[2 * EPI_LD], t1[3 * EPI_LD]);
+              }
+            }
+          }
+        }
+        continue;
       }
       if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag, status)) break;
       tc_fence_after();
@@ -807,7 +1001,8 @@ bool encode_operand(CUtensorMap* map, const TcOperand& op, int64_t rows, int64_t
 }
 
 typedef void (*TcKernel)(const DevProblem*, int, int, int, long long, int, float, float, int*);
-TcKernel kernel_of(bool shared, bool pair) {
+TcKernel kernel_of(bool shared, bool pair, bool fold = false) {
+  if (fold) return pair ? k_tc_gemm<false, true, true> : k_tc_gemm<false, false, true>;
   if (pair) return shared ? k_tc_gemm<true, true> : k_tc_gemm<false, true>;
   return shared ? k_tc_gemm<true, false> : k_tc_gemm<false, false>;
 }
@@ -848,6 +1043,7 @@ int pair_capacity(bool shared) {
 }  // namespace
 
 struct TcPlan {
+  bool fold = false;            // launches the folded form (chunked accumulation, running sum in tensor memory)
   bool shared = false;          // launches the shared-operand form of the kernel
   bool pair = false;            // launches the paired form (clusters of two CTAs, 256-row tiles)
   int max_pairs = 0;            // CTA pairs that can be resident at once
@@ -894,6 +1090,12 @@ TcPlan* tc_plan_create(const TcProblem* problems, int n, int device, cudaStream_
     if (nA > 2 || nB > 2) eligible = false;
   }
   shared = shared && eligible;
+  // the folded form: every problem asks for it, and none sums several operand pairs
+  bool fold = !shared;
+  for (int i = 0; i < n; ++i) fold = fold && problems[i].fold_kb > 0 && problems[i].n_pairs == 1;
+  if (const char* env = std::getenv("BR_TC_FOLD")) { if (env[0] == '0') fold = false; }      // tuning aid
+  int fold_override = 0;
+  if (const char* env = std::getenv("BR_TC_FOLD_KB")) { const int v = std::atoi(env); if (v >= 1 && v <= 1024) fold_override = v; }
   const int pairs = pair_capacity(shared);
   const bool pair = pairs > 0;
   const int TM = pair ? 2 * BM : BM;            // rows of a tile
@@ -985,6 +1187,7 @@ TcPlan* tc_plan_create(const TcProblem* problems, int n, int device, cudaStream_
     d.alpha = q.alpha; d.beta = q.beta; d.eps = q.eps; d.beta1 = q.beta1;
     d.symmetric = q.symmetric ? 1 : 0;
     d.clip = q.clip_mode ? q.clip : nullptr; d.clip_slots = q.clip_slots; d.clip_mode = q.clip_mode;
+    d.fold_kb = fold ? (fold_override ? fold_override : q.fold_kb) : 0;
     if (d.clip && (q.clip_slots < 1 || (q.clip_mode == 1 && q.epilogue != EPI_ROTATED_ADAM) ||
                    (q.clip_mode == 2 && q.epilogue != EPI_AXPBY_F32)))
       return fail("tensor-core problem: clipping applies to the rotated-Adam and factor epilogues");
@@ -1013,6 +1216,7 @@ TcPlan* tc_plan_create(const TcProblem* problems, int n, int device, cudaStream_
     prob_flops.push_back(flops - flops_before);
   }
   TcPlan* plan = new TcPlan();
+  plan->fold = fold;
   plan->shared = shared;
   plan->pair = pair;
   plan->max_pairs = pairs;
@@ -1049,9 +1253,10 @@ cudaError_t tc_plan_launch_range(TcPlan* p, int first, int count, long long call
   if (first < 0 || count < 1 || first + count > p->n) return cudaErrorInvalidValue;
   const int t0 = p->tile_begin[first], t1 = p->tile_begin[first + count];
   const int tiles = t1 - t0;
-  TcKernel kernel = kernel_of(p->shared, p->pair);
+  TcKernel kernel = kernel_of(p->shared, p->pair, p->fold);
   // per-device attribute: set again when another device is current (cheap, idempotent)
-  cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+  const int smem_bytes = p->fold ? SMEM_BYTES_FOLD : SMEM_BYTES;
+  cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
   cudaLaunchConfig_t cfg = {};
   cudaLaunchAttribute attr[1];
   if (p->pair) {
@@ -1063,8 +1268,8 @@ cudaError_t tc_plan_launch_range(TcPlan* p, int first, int count, long long call
   } else {
     cfg.gridDim = dim3((unsigned)(tiles < p->sm_count ? tiles : p->sm_count));
   }
-  cfg.blockDim = dim3(NUM_THREADS);
-  cfg.dynamicSmemBytes = SMEM_BYTES;
+  cfg.blockDim = dim3(p->fold ? FOLD_THREADS : NUM_THREADS);
+  cfg.dynamicSmemBytes = smem_bytes;
   cfg.stream = s;
   return cudaLaunchKernelEx(&cfg, kernel, (const DevProblem*)p->d_probs, p->n, t0, t1, calls, tau, dyn_alpha,
                             dyn_beta, status_word);

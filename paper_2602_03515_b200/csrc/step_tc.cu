@@ -38,6 +38,11 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 // phase writes (first-side products, X, Y) still be in L2 when the next phase reads it: on the ~3B layer
 // set a step takes 158 ms with 8 GiB (3 chunks), 150 with 4, 147 with 2, 148 with 1, 150.5 with 0.5.
 constexpr size_t kDefaultScratch = 2ull << 30;
+// Factor products are accumulated in chunks of a few 64-deep k-blocks (see gemm_tc.cu, folded form): at
+// least ten chunks per contraction where it is long enough, at most four k-blocks per chunk (the epilogue
+// warps keep up with the tensor core from four k-blocks on; with two they are the limit: a step of the
+// ~3B layer set takes 4 % longer with four than without the folding, 12 % longer with two).
+inline int fold_kb(int64_t K) { return (int)std::max<int64_t>(1, std::min<int64_t>(4, (K + 63) / 64 / 10)); }
 
 struct LayerScratch {
   __nv_bfloat16* B[4] = {nullptr, nullptr, nullptr, nullptr};
@@ -100,14 +105,14 @@ void factor_problems(const Layer& L, float beta, std::vector<TcProblem>* out) {
     TcProblem q; q.Md = m; q.Nd = m; q.K = n; q.n_pairs = 1;
     q.A[0] = ring_op(L, 0); q.B[0] = ring_op(L, 0);
     q.epilogue = EPI_AXPBY_F32; q.alpha = 1.f - beta; q.beta = beta; q.D = L.L; q.ldd = m; q.tau_max = L.d.tau_max;
-    q.symmetric = 1;
+    q.symmetric = 1; q.fold_kb = fold_kb(n);
     out->push_back(q);
   }
   if (L.R) {      // R <- beta R + (1-beta) G^T G : both operands MN-major views of G
     TcProblem q; q.Md = n; q.Nd = n; q.K = m; q.n_pairs = 1;
     q.A[0] = ring_op(L, 1); q.B[0] = ring_op(L, 1);
     q.epilogue = EPI_AXPBY_F32; q.alpha = 1.f - beta; q.beta = beta; q.D = L.R; q.ldd = n; q.tau_max = L.d.tau_max;
-    q.symmetric = 1;
+    q.symmetric = 1; q.fold_kb = fold_kb(m);
     out->push_back(q);
   }
 }

@@ -121,10 +121,10 @@ typedef struct {
    * the last refresh of this layer's bases.  Bit 0 (left) and bit 1 (right): no column of F Q shrank
    * below 1e-3 of its length under orthonormalisation; the next refresh of a tensor-core layer runs
    * its block projections on the tensor cores only for a basis whose bit is set.  Bit 2 (left) and
-   * bit 3 (right): the factorisation had to clamp a pivot (a numerically rank-deficient product; the
-   * status word then holds BR_WARN_RANK_DEFICIENT and the affected columns of that refresh are not
-   * orthonormal); the next refresh of that basis completes it from the current one.  Saved and
-   * restored with the other counters so that a resumed run takes the same decisions. */
+   * bit 3 (right): the last refresh met a numerically rank-deficient product (some |R_jj| <= 1e-12 of
+   * the largest); the status word then holds BR_WARN_RANK_DEFICIENT and the basis was completed from the
+   * previous one in that same refresh, so it is orthonormal.  Saved and restored with the other
+   * counters so that a resumed run takes the same decisions. */
   int64_t basis_flags;
 } br_counters;
 

@@ -363,7 +363,7 @@ br_status orthonormalise(br_handle* h, br_handle::Lane& ln, int64_t k, QrTc* tcq
       cudaGraph_t graph = nullptr;
       cudaError_t e = cudaStreamBeginCapture(s, cudaStreamCaptureModeRelaxed);
       if (e == cudaSuccess) {
-        const cudaError_t qe = qr_pos_inplace(ln.rA, k, ln.rWork, h->d_status, s, &g.launches, &g.flops, tcq, ln.cond);
+        const cudaError_t qe = qr_pos_inplace(ln.rA, k, ln.rWork, h->d_status, s, &g.launches, &g.flops, tcq, ln.cond, ln.rF, ln.rQ);
         e = cudaStreamEndCapture(s, &graph);          // always ends the capture, also after a failed launch
         if (e == cudaSuccess && qe != cudaSuccess) e = qe;
         if (e == cudaSuccess && graph) e = cudaGraphInstantiate(&g.exec, graph, 0);
@@ -385,7 +385,7 @@ br_status orthonormalise(br_handle* h, br_handle::Lane& ln, int64_t k, QrTc* tcq
     }
   }
   BR_CUDA(h, qr_pos_inplace(ln.rA, k, ln.rWork, h->d_status, s, &h->stats.launches, &h->stats.gemm_flops, tcq,
-                            h->d_cond + ci));
+                            h->d_cond + ci, ln.rF, ln.rQ));
   return BR_OK;
 }
 
@@ -404,7 +404,7 @@ br_status refresh_side(br_handle* h, Layer& L, bool left_side, br_handle::Lane& 
   const int64_t other = left_side ? n : m;
   const bool short_of_rank = (L.d.src == BR_SRC_FIRST) ? (k > other)
                                                        : (L.n_accum < (k + other - 1) / other);
-  const bool complete = short_of_rank || (h->cond_known[ci] & 2);
+  const bool complete = short_of_rank;
   QrTc* tcq = nullptr;
   if (L.use_tc && (h->cond_known[ci] & 1) && !complete)
     for (QrTc* t : ln.tcq) if (qr_tc_order(t) == k) tcq = t;
@@ -424,26 +424,33 @@ br_status refresh_side(br_handle* h, Layer& L, bool left_side, br_handle::Lane& 
       }
     } else if (left_side) {
       // (M M^T) U = M (M^T U)
+      BR_CUDA(h, f32_to_f64(Q, ln.rQ, k * k, s));          // the current basis, for the completion of a deficient product
+      count(h);
       BR_CUDA(h, sdgemm(1, 0, n, m, m, 1.0, Mo, n, Q, m, 0.0, ln.rZ, m, s));
       BR_CUDA(h, fdgemm(0, 0, m, m, n, 1.0, Mo, n, ln.rZ, m, 0.0, ln.rA, m, s));
       count(h, 2); h->stats.gemm_flops += 4.0 * m * m * n;
     } else {
       // (M^T M) V = M^T (M V)
+      BR_CUDA(h, f32_to_f64(Q, ln.rQ, k * k, s));
+      count(h);
       BR_CUDA(h, sdgemm(0, 0, m, n, n, 1.0, Mo, n, Q, n, 0.0, ln.rZ, n, s));
       BR_CUDA(h, fdgemm(1, 0, n, n, m, 1.0, Mo, n, ln.rZ, n, 0.0, ln.rA, n, s));
       count(h, 2); h->stats.gemm_flops += 4.0 * n * n * m;
     }
     // A rank-deficient product has no unique Q factor.  Which products are is known on the host: with
     // S = 1st, M M^T (M^T M) has rank <= min(m, n), short of the larger side; with S = 2nd, a factor that
-    // has accumulated a gradients has rank <= a * (the other dimension); and a basis whose previous
-    // refresh had to clamp a pivot sits on a factor that is rank-deficient numerically (gradients
-    // confined to a subspace).  The directions outside the range of F Q are then completed from the
-    // current basis: what is orthonormalised is F Q with 1e-6 ||(F Q)_j|| Q_j added to every column j
-    // (full rank whenever Q is).
+    // has accumulated a gradients has rank <= a * (the other dimension).  The directions outside the
+    // range of F Q are then completed from the current basis: what is orthonormalised is F Q with
+    // 1e-6 ||(F Q)_j|| Q_j added to every column j (full rank whenever Q is).
     if (complete) {
       BR_CUDA(h, qr_complete_columns(ln.rA, Q, k, ln.rWork, h->d_status, s));
       count(h, 3);
     }
+    // A product that is rank-deficient only numerically (gradients confined to a subspace) shows in the
+    // factorisation itself: the orthonormalisation then repeats it, in the same call, on the completed
+    // product, for which it needs the product once more (the factor's buffer is free by now) and the
+    // current basis (ln.rQ).
+    BR_CUDA(h, cudaMemcpyAsync(ln.rF, ln.rA, sizeof(double) * (size_t)k * (size_t)k, cudaMemcpyDeviceToDevice, s));
     {
       br_status st = orthonormalise(h, ln, k, tcq, ci, s);
       if (st != BR_OK) return st;

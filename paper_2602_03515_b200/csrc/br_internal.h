@@ -147,8 +147,15 @@ cudaError_t qr_tc_project(QrTc* t, int node, double* A, int64_t k, int64_t jp, i
 // tc: null, or the plans for this order: the first sweep then projects on the tensor cores (ask for it
 // only when the previous refresh of this basis left *cond_out == 1).  cond_out: DEVICE int that
 // receives 1 when no column shrank below 1e-3 of its length during this factorisation, else 0.
+// Acopy / Qprev (both k x k fp64, or both null): a second copy of A and the basis the product was formed
+// from.  With them, a product that turns out rank-deficient -- some |R_jj| <= 1e-12 max |R_kk| -- is
+// factorised again in the same call with 1e-6 ||A_j|| Qprev_j added to every column (the completion rule
+// for rank-deficient products), so that the result is orthonormal either way; BR_WARN_RANK_DEFICIENT is
+// raised.  The launches of that second factorisation are always enqueued and return at once when the
+// product has full rank.
 cudaError_t qr_pos_inplace(double* A, int64_t k, double* work, int* status, cudaStream_t s,
-                           int64_t* launches, double* flops, QrTc* tc = nullptr, int* cond_out = nullptr);
+                           int64_t* launches, double* flops, QrTc* tc = nullptr, int* cond_out = nullptr,
+                           const double* Acopy = nullptr, const double* Qprev = nullptr);
 
 // ---------------------------------------------------------------------------------------------
 // tcgen05 grouped contraction (gemm_tc.cu)

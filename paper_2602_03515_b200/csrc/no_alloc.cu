@@ -22,7 +22,7 @@
 namespace {
 
 constexpr int64_t kMaxOrder = 512;
-// k*k doubles for the product F*Q (rounded up to a 256-byte boundary), the QR work area (90,688
+// k*k doubles for the product F*Q (rounded up to a 256-byte boundary), the QR work area (91,200
 // doubles at order kMaxOrder, the largest over all orders up to it), and 64 doubles holding the
 // rank-deficiency flag.
 constexpr size_t kWorkDoubles = 98304;

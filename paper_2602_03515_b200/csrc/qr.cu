@@ -88,7 +88,7 @@ __global__ void __launch_bounds__(512)
 k_chol_inverse(const double* __restrict__ S, int bw, double* __restrict__ Rinv, int* __restrict__ status,
                int* __restrict__ skip_next, const int* __restrict__ skip_self,
                const double* __restrict__ norm0, int* __restrict__ ill_clear, double ill_ratio,
-               int* __restrict__ tc_ok_clear) {
+               int* __restrict__ tc_ok_clear, double* __restrict__ rdiag) {
   if (skip_self && *skip_self) {
     if (skip_next && threadIdx.x == 0) *skip_next = 1;
     return;
@@ -132,6 +132,8 @@ k_chol_inverse(const double* __restrict__ S, int bw, double* __restrict__ Rinv, 
     if (t == 0) {
       if (clamped) { atomicMax(status, (int)BR_WARN_RANK_DEFICIENT); any_clamped = true; }
       min_ratio = fmin(min_ratio, piv * diag0_inv[c]);
+      // R_cc^2 of the whole factorisation is the product of this column's pivots over every pass and sweep
+      if (rdiag) rdiag[c] *= piv;
       if (orig < nrm_floor[c]) ill = true;
       if (orig < tc_floor[c]) tc_bad = true;
     }
@@ -198,7 +200,9 @@ __global__ void k_store_flag(int* dst, const int* src) { *dst = (src[0] ? 1 : 0)
 // part[z][j] = sum over the row chunk z of A[i][j]^2 (rows in order)
 constexpr int kNormChunks = 32;
 __global__ void __launch_bounds__(256)
-k_column_norms_partial(const double* __restrict__ A, int64_t k, int64_t rows_per_chunk, double* __restrict__ part) {
+k_column_norms_partial(const double* __restrict__ A, int64_t k, int64_t rows_per_chunk, double* __restrict__ part,
+                       const int* __restrict__ skip) {
+  if (skip && *skip) return;
   const int64_t j = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
   if (j >= k) return;
   const int64_t r0 = (int64_t)blockIdx.y * rows_per_chunk;
@@ -215,14 +219,56 @@ k_column_norms_partial(const double* __restrict__ A, int64_t k, int64_t rows_per
 // norm0[j] = sum_z part[z][j] in chunk order; *flag = 1
 __global__ void __launch_bounds__(256)
 k_column_norms_sum(const double* __restrict__ part, int64_t k, int nchunks, double* __restrict__ norm0,
-                   int* __restrict__ flag) {
+                   int* __restrict__ flag, double* __restrict__ rdiag, const int* __restrict__ skip) {
   const int64_t j = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
   // sweep-2 cancelled, tensor-core projections allowed next time, no pivot clamped so far
-  if (j == 0) { flag[0] = 1; flag[1] = 1; flag[2] = 0; }
-  if (j >= k) return;
+  // (a cancelled factorisation leaves only "sweep 2 cancelled" behind)
+  const bool off = skip && *skip;
+  if (j == 0) { flag[0] = 1; if (!off) { flag[1] = 1; flag[2] = 0; } }
+  if (off || j >= k) return;
   double s = 0.0;
   for (int z = 0; z < nchunks; ++z) s += part[(int64_t)z * k + j];
   norm0[j] = s;
+  if (rdiag) rdiag[j] = 1.0;
+}
+
+// The rank decision of the oracle's QR, on the squared diagonal of R: the product is rank-deficient when
+// some R_jj^2 is at most 1e-24 of the largest (|R_jj| <= 1e-12 max_k |R_kk|), or is not a positive number.
+// *run_fix = 0 then lets the completion that is enqueued behind this kernel run (it returns at once
+// otherwise), the status word gets BR_WARN_RANK_DEFICIENT, and note[2] tells the next refresh of this
+// basis to complete its product up front.
+__global__ void __launch_bounds__(256)
+k_rank_decide(const double* __restrict__ rdiag, int64_t k, int* __restrict__ skip_fix, int* __restrict__ status,
+              int* __restrict__ note) {
+  __shared__ double smin[256], smax[256];
+  double lo = 1e300, hi = 0.0;
+  bool bad = false;
+  for (int64_t j = threadIdx.x; j < k; j += blockDim.x) {
+    const double v = rdiag[j];
+    if (!(v > 0.0)) bad = true;
+    lo = fmin(lo, v); hi = fmax(hi, v);
+  }
+  smin[threadIdx.x] = bad ? 0.0 : lo; smax[threadIdx.x] = hi;
+  __syncthreads();
+  for (int w = 128; w > 0; w >>= 1) {
+    if (threadIdx.x < w) {
+      smin[threadIdx.x] = fmin(smin[threadIdx.x], smin[threadIdx.x + w]);
+      smax[threadIdx.x] = fmax(smax[threadIdx.x], smax[threadIdx.x + w]);
+    }
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    const bool deficient = !(smin[0] > 1e-24 * smax[0]);
+    *skip_fix = deficient ? 0 : 1;
+    if (deficient) { atomicMax(status, (int)BR_WARN_RANK_DEFICIENT); if (note) note[2] = 1; }
+  }
+}
+
+// A <- B (k x k doubles) unless *skip
+__global__ void __launch_bounds__(256)
+k_copy_unless(double* __restrict__ A, const double* __restrict__ B, int64_t n, const int* __restrict__ skip) {
+  if (skip && *skip) return;
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) A[i] = B[i];
 }
 
 struct ProjNode { int64_t jp, wp, jt, wt; };
@@ -404,6 +450,7 @@ namespace {
 struct Sweep {
   double* A; int64_t k; int b, sg, sp_max;
   double *gram_part, *S, *Rinv, *norm0, *C, *proj_part;
+  double* rdiag = nullptr;    // squared diagonal of R, accumulated over passes and sweeps
   int *skip2, *sweep2_skip;   // sweep2_skip[1] is the "tensor cores allowed next time" flag
   QrTc* tc = nullptr;         // non-null: block projections of the first sweep on the tensor cores
   int node = 0;               // running index of the projection in recursion order
@@ -427,7 +474,7 @@ void leaf(Sweep& q, int64_t j0, int bw) {
     if (e != cudaSuccess) { q.err = e; return; }
     k_chol_inverse<<<1, 512, 0, q.s>>>(q.S, bw, q.Rinv, q.status, pass ? nullptr : q.skip2, skip,
                                        (q.first && !pass) ? q.norm0 + j0 : nullptr, q.sweep2_skip, q.ill_ratio,
-                                       q.sweep2_skip + 1);
+                                       q.sweep2_skip + 1, q.rdiag ? q.rdiag + j0 : nullptr);
     // P <- P R^-1 (in place: a CTA reads only the rows it writes, and writes after its last read)
     e = dgemm_ex(0, 0, k, bw, bw, 1.0, P, k, q.Rinv, bw, 0.0, P, k, 1, nullptr, skip, q.s);
     if (e != cudaSuccess) { q.err = e; return; }
@@ -476,9 +523,11 @@ inline int64_t proj_part_doubles(int64_t k) {
 
 namespace {
 constexpr double kCompletion = 1e-6;
+template <typename TQ>
 __global__ void __launch_bounds__(256)
-k_complete_columns(double* __restrict__ A, const float* __restrict__ Q, int64_t k, const double* __restrict__ norm2,
-                   int* __restrict__ status) {
+k_complete_columns(double* __restrict__ A, const TQ* __restrict__ Q, int64_t k, const double* __restrict__ norm2,
+                   int* __restrict__ status, const int* __restrict__ skip) {
+  if (skip && *skip) return;
   const int64_t total = k * k;
   if (blockIdx.x == 0 && threadIdx.x == 0) atomicMax(status, (int)BR_WARN_RANK_DEFICIENT);
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
@@ -490,7 +539,9 @@ k_complete_columns(double* __restrict__ A, const float* __restrict__ Q, int64_t 
 }
 }  // namespace
 
-cudaError_t qr_complete_columns(double* A, const float* Q, int64_t k, double* work, int* status, cudaStream_t s) {
+namespace {
+template <typename TQ>
+cudaError_t complete_columns(double* A, const TQ* Q, int64_t k, double* work, int* status, const int* skip, cudaStream_t s) {
   // column norms exactly as the factorisation computes them (same kernels, same order)
   double* part = work;                                   // kNormChunks * k doubles at most (see qr_work_doubles)
   const int nchunks = (int)std::min<int64_t>(kNormChunks, std::max<int64_t>(1, k / 4));
@@ -499,21 +550,30 @@ cudaError_t qr_complete_columns(double* A, const float* Q, int64_t k, double* wo
   double* norm2 = part + (int64_t)used * k;
   int* dummy = reinterpret_cast<int*>(norm2 + k);
   dim3 grid((unsigned)cdiv(k, 256), (unsigned)used);
-  k_column_norms_partial<<<grid, 256, 0, s>>>(A, k, rows_per_chunk, part);
-  k_column_norms_sum<<<(unsigned)cdiv(k, 256), 256, 0, s>>>(part, k, used, norm2, dummy);
+  k_column_norms_partial<<<grid, 256, 0, s>>>(A, k, rows_per_chunk, part, skip);
+  k_column_norms_sum<<<(unsigned)cdiv(k, 256), 256, 0, s>>>(part, k, used, norm2, dummy, nullptr, skip);
   const int64_t blocks = cdiv(k * k, 256);
-  k_complete_columns<<<(unsigned)(blocks < 1184 ? blocks : 1184), 256, 0, s>>>(A, Q, k, norm2, status);
+  k_complete_columns<TQ><<<(unsigned)(blocks < 1184 ? blocks : 1184), 256, 0, s>>>(A, Q, k, norm2, status, skip);
   return cudaGetLastError();
+}
+}  // namespace
+
+cudaError_t qr_complete_columns(double* A, const float* Q, int64_t k, double* work, int* status, cudaStream_t s) {
+  return complete_columns<float>(A, Q, k, work, status, nullptr, s);
 }
 
 size_t qr_work_doubles(int64_t k) {
   const int64_t b = std::min<int64_t>(panel_width(k), k);
   return (size_t)(pad32((int64_t)gram_splits(k) * b * b) + 2 * pad32(b * b) + 64 + pad32(k) +
-                  pad32(((k + 1) / 2) * ((k + 1) / 2)) + pad32(proj_part_doubles(k)));
+                  pad32(((k + 1) / 2) * ((k + 1) / 2)) + pad32(proj_part_doubles(k)) + pad32(k));
 }
 
-cudaError_t qr_pos_inplace(double* A, int64_t k, double* work, int* status, cudaStream_t s,
-                           int64_t* launches, double* flops, QrTc* tc, int* cond_out) {
+namespace {
+// One factorisation (two sweeps, the second cancelled on the device unless the first met an ill-conditioned
+// input).  flag_base: which of the flag words of the work area this run uses; skip_all: a DEVICE flag that
+// turns the whole run into launches that return at once; rdiag: receives the squared diagonal of R.
+cudaError_t run_qr(double* A, int64_t k, double* work, int flag_base, int* status, cudaStream_t s, const int* skip_all,
+                   QrTc* tc, bool track_rdiag, int64_t* launches, double* flops) {
   Sweep q;
   if (tc && tc->k == k) { q.tc = tc; q.ill_ratio = kTcRatio; }
   q.A = A; q.k = k; q.s = s; q.status = status;
@@ -524,12 +584,13 @@ cudaError_t qr_pos_inplace(double* A, int64_t k, double* work, int* status, cuda
   q.gram_part = work;
   q.S = q.gram_part + pad32((int64_t)q.sg * b * b);
   q.Rinv = q.S + pad32(b * b);
-  int* flags = reinterpret_cast<int*>(q.Rinv + pad32(b * b));      // 64 doubles reserved for flags
+  int* flags = reinterpret_cast<int*>(q.Rinv + pad32(b * b)) + flag_base;      // 64 doubles reserved for flags
   q.skip2 = flags;
   q.sweep2_skip = flags + 1;
   q.norm0 = q.Rinv + pad32(b * b) + 64;
   q.C = q.norm0 + pad32(k);
   q.proj_part = q.C + pad32(((k + 1) / 2) * ((k + 1) / 2));
+  q.rdiag = track_rdiag ? q.proj_part + pad32(proj_part_doubles(k)) : nullptr;
   // first sweep, watching how much of its norm each column keeps
   {
     // the partial sums borrow the (still unused) projection buffer: kNormChunks * k <= (k + 1)^2 / 4 for k >= 128
@@ -537,22 +598,45 @@ cudaError_t qr_pos_inplace(double* A, int64_t k, double* work, int* status, cuda
     const int64_t rows_per_chunk = cdiv(k, nchunks);
     const int used = (int)cdiv(k, rows_per_chunk);
     dim3 grid((unsigned)cdiv(k, 256), (unsigned)used);
-    k_column_norms_partial<<<grid, 256, 0, s>>>(A, k, rows_per_chunk, q.C);
-    k_column_norms_sum<<<(unsigned)cdiv(k, 256), 256, 0, s>>>(q.C, k, used, q.norm0, q.sweep2_skip);
+    k_column_norms_partial<<<grid, 256, 0, s>>>(A, k, rows_per_chunk, q.C, skip_all);
+    k_column_norms_sum<<<(unsigned)cdiv(k, 256), 256, 0, s>>>(q.C, k, used, q.norm0, q.sweep2_skip, q.rdiag, skip_all);
   }
-  q.skip = nullptr; q.first = true;
+  q.skip = skip_all; q.first = true;
   orth(q, 0, k);
   if (q.err != cudaSuccess) return q.err;
   // second sweep, cancelled on the device unless the first one met an ill-conditioned input
   q.skip = q.sweep2_skip; q.first = false;
   orth(q, 0, k);
   if (q.err != cudaSuccess) return q.err;
-  if (cond_out) k_store_flag<<<1, 1, 0, s>>>(cond_out, q.sweep2_skip + 1);
-  cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess) return e;
-  if (launches) *launches += q.launches + 2 + (cond_out ? 1 : 0);
+  if (launches) *launches += q.launches + 2;
   if (flops) *flops += q.flops;
-  return cudaSuccess;
+  return cudaGetLastError();
+}
+}  // namespace
+
+cudaError_t qr_pos_inplace(double* A, int64_t k, double* work, int* status, cudaStream_t s,
+                           int64_t* launches, double* flops, QrTc* tc, int* cond_out, const double* Acopy,
+                           const double* Qprev) {
+  const bool fix = Acopy != nullptr && Qprev != nullptr;
+  cudaError_t e = run_qr(A, k, work, 0, status, s, nullptr, tc, fix, launches, flops);
+  if (e != cudaSuccess) return e;
+  const int64_t b = std::min<int64_t>(panel_width(k), k);
+  int* flags = reinterpret_cast<int*>(work + pad32((int64_t)gram_splits(k) * b * b) + 2 * pad32(b * b));
+  if (fix) {
+    // The oracle's rule for a rank-deficient product (decided on the diagonal of R, as the oracle decides
+    // it): factorise A with 1e-6 ||A_j|| Qprev_j added to every column instead.  Everything is enqueued
+    // here and returns at once unless the decision kernel finds the product deficient.
+    double* rdiag = work + qr_work_doubles(k) - pad32(k);
+    int* skip_fix = flags + 16;
+    k_rank_decide<<<1, 256, 0, s>>>(rdiag, k, skip_fix, status, flags + 1);
+    const int64_t n = k * k, blocks = cdiv(n, 256);
+    k_copy_unless<<<(unsigned)(blocks < 1184 ? blocks : 1184), 256, 0, s>>>(A, Acopy, n, skip_fix);
+    if ((e = complete_columns<double>(A, Qprev, k, work, status, skip_fix, s)) != cudaSuccess) return e;
+    if ((e = run_qr(A, k, work, 8, status, s, skip_fix, nullptr, false, launches, nullptr)) != cudaSuccess) return e;
+    if (launches) *launches += 5;
+  }
+  if (cond_out) { k_store_flag<<<1, 1, 0, s>>>(cond_out, flags + 2); if (launches) *launches += 1; }
+  return cudaGetLastError();
 }
 
 }  // namespace br

@@ -68,7 +68,7 @@ class SideBySide:
     """Steps a workload through libbr (GPU) and the oracle (CPU float64) together."""
 
     def __init__(self, w, *, gemm_prec=None, accum="every_step", power_iters=1, clip_norm=0.0, device="cuda:0",
-                 oracle_qr="householder", twin=False, **kw):
+                 oracle_qr="householder", twin=False, beta_factor=-1.0, **kw):
         import torch
         import paper_2602_03515_b200 as br
         self.torch, self.br, self.w = torch, br, w
@@ -80,7 +80,8 @@ class SideBySide:
         f32 = lambda x: float(np.float32(x))
         self.oracle = O.make_oracle(w, w0, accum=accum, power_iters=power_iters, lr=f32(w.lr),
                                     beta1=f32(w.beta1), beta2=f32(w.beta2), eps=f32(w.eps),
-                                    weight_decay=f32(w.weight_decay), clip_norm=f32(clip_norm), qr=oracle_qr)
+                                    weight_decay=f32(w.weight_decay), clip_norm=f32(clip_norm), qr=oracle_qr,
+                                    beta_factor=f32(beta_factor))
         # optional twin of the oracle whose factor products carry the library's documented accuracy
         self.twin = None
         if twin:
@@ -92,7 +93,7 @@ class SideBySide:
                 lay.set_noise(factor_accuracy(lay, "U", True), factor_accuracy(lay, "V", True), 1000 + i)
         gp = gemm_prec if gemm_prec is not None else (br.BR_GEMM_FP32 if w.gemm_prec == "f32" else br.BR_GEMM_BF16)
         self.opt = br.BasisRotation.from_workload(
-            w, self.weights, gemm_prec=gp, power_iters=power_iters, clip_norm=clip_norm,
+            w, self.weights, gemm_prec=gp, power_iters=power_iters, clip_norm=clip_norm, beta_factor=beta_factor,
             accum=br.BR_ACCUM_ON_REFRESH if accum == "on_refresh" else br.BR_ACCUM_EVERY_STEP, **kw)
         self.call = 0
 

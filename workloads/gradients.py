@@ -51,6 +51,12 @@ class GradientStream:
             # Signal factors drawn once per layer: a persistent signal subspace.
             self._A = _rng(w.seed, layer, 0, _TAG_FACTOR_A).standard_normal((self.m, w.grad_rank))
             self._B = _rng(w.seed, layer, 0, _TAG_FACTOR_B).standard_normal((self.n, w.grad_rank))
+        if w.grad_kind == "integer_subspace":
+            # Gradients confined to fixed rank-r row and column spaces, with entries that are small integers
+            # times grad_scale (a power of two): exactly representable in bf16, so that products and short
+            # sums of them are exact in fp32 and the factors G G^T, G^T G have exactly rank r on both sides.
+            self._A = _rng(w.seed, layer, 0, _TAG_FACTOR_A).integers(-1, 2, (self.m, w.grad_rank)).astype(np.float64)
+            self._B = _rng(w.seed, layer, 0, _TAG_FACTOR_B).integers(-1, 2, (self.n, w.grad_rank)).astype(np.float64)
 
     def f64(self, call: int) -> np.ndarray:
         w = self.w
@@ -59,6 +65,9 @@ class GradientStream:
             return w.grad_scale * r.standard_normal((self.m, self.n))
         if w.grad_kind == "lowrank_noise":
             return self._A @ self._B.T + w.grad_scale * r.standard_normal((self.m, self.n))
+        if w.grad_kind == "integer_subspace":
+            C = r.integers(-1, 2, (w.grad_rank, w.grad_rank)).astype(np.float64)
+            return w.grad_scale * (self._A @ C @ self._B.T)
         if w.grad_kind == "student_t":
             return w.grad_scale * r.standard_t(3.0, size=(self.m, self.n))
         raise ValueError(w.grad_kind)

@@ -363,6 +363,9 @@ br_status orthonormalise(br_handle* h, br_handle::Lane& ln, int64_t k, QrTc* tcq
       cudaGraph_t graph = nullptr;
       cudaError_t e = cudaStreamBeginCapture(s, cudaStreamCaptureModeRelaxed);
       if (e == cudaSuccess) {
+        // (the completion of a rank-deficient product is part of the chain as launches that a device flag
+        // cancels; as the body of a conditional graph node it made a refresh of 57 bases slower, 354 ms
+        // against 324, although a full-rank product then launches nothing of it)
         const cudaError_t qe = qr_pos_inplace(ln.rA, k, ln.rWork, h->d_status, s, &g.launches, &g.flops, tcq, ln.cond, ln.rF, ln.rQ);
         e = cudaStreamEndCapture(s, &graph);          // always ends the capture, also after a failed launch
         if (e == cudaSuccess && qe != cudaSuccess) e = qe;

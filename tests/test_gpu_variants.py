@@ -30,4 +30,5 @@ def test_refresh_without_graphs_and_small_lanes():
     _run({"BR_REFRESH_GRAPHS": "0", "BR_REFRESH_SMALL_LANES": "0", "BR_REFRESH_LANES": "1"},
          ["tests/test_gpu_full_size.py::test_refresh_order_1024_against_oracle_power",
           "tests/test_gpu_full_size.py::test_refresh_tensor_core_projections",
+          "tests/test_gpu_parity_fp32.py::test_numerically_rank_deficient_refresh_is_completed_in_the_same_call",
           "tests/test_gpu_parity_bf16.py", "-k", "not checkpoint"])

@@ -11,7 +11,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libbr.so")
-SOURCES = ["br_api.cu", "elem.cu", "gemm_simt.cu", "dgemm.cu", "qr.cu", "gemm_tc.cu", "step_tc.cu", "no_alloc.cu"]
+SOURCES = ["br_api.cu", "elem.cu", "gemm_simt.cu", "dgemm.cu", "qr.cu", "gemm_tc.cu", "step_tc.cu", "no_alloc.cu", "small_step.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC,-fvisibility=hidden", "--expt-relaxed-constexpr",
               "-I", os.path.join(ROOT, "include"), "-I", CSRC]

@@ -930,7 +930,21 @@ br_status step_enqueue(br_handle* h, const void* const* grads, int tau) {
                             hp.lr, hp.beta1, hp.beta2, hp.eps, hp.weight_decay, GS[i], h->stream));
       count(h);
     } else if (!L.use_tc) {
-      if ((st = update_layer_simt(h, L, G[i], GS[i])) != BR_OK) return st;
+      // a small matrix is bound by launch latency: its whole update is one launch, unless a refresh is due
+      static const bool small_on = !(std::getenv("BR_SMALL_STEP") && std::getenv("BR_SMALL_STEP")[0] == '0');
+      if (small_on && L.t % L.freq != 0 && small_step_eligible(L.d.m, L.d.n, L.left, L.right)) {
+        const bool acc = L.d.src == BR_SRC_SECOND && hp.accum == BR_ACCUM_EVERY_STEP;
+        const int64_t m = L.d.m, n = L.d.n;
+        BR_CUDA(h, small_step(m, n, L.left, L.right, G[i], L.d.grad_dtype == BR_BF16, GS[i], L.M, L.V2, L.U, L.V, L.L, L.R,
+                              L.d.weight, acc ? 1 : 0, hp.lr, hp.beta1, hp.beta2, hp.eps, hp.weight_decay,
+                              hp.beta_factor < 0.f ? hp.beta2 : hp.beta_factor, h->stream));
+        count(h);
+        h->stats.gemm_flops += (acc ? 2.0 : 0.0) * ((L.L ? m * m * n : 0) + (L.R ? n * n * m : 0)) +
+                               6.0 * m * n * ((L.left ? m : 0) + (L.right ? n : 0));
+        if (acc) L.n_accum += 1;
+      } else if ((st = update_layer_simt(h, L, G[i], GS[i])) != BR_OK) {
+        return st;
+      }
     }
   }
   if (h->tc) {

@@ -101,6 +101,13 @@ cudaError_t sub_f32_from_f64(double* A, int64_t ld, int64_t rows, int64_t cols, 
 cudaError_t ema_out(float* out, const float* M, const void* G, int g_is_bf16, int64_t numel, float beta1,
                     const float* gscale, cudaStream_t s);
 
+// One whole update (Alg. 1 lines 4, 8-11 and the factor EMAs of Alg. 2, no refresh) of a matrix with both
+// dimensions <= 128 in a single one-CTA launch (small_step.cu).  accumulate: update L and R as well.
+bool small_step_eligible(int64_t m, int64_t n, bool left, bool right);
+cudaError_t small_step(int64_t m, int64_t n, bool left, bool right, const void* G, int g_is_bf16, const float* gscale,
+                       float* M, float* V2, float* U, float* V, float* L, float* R, float* W, int accumulate, float lr,
+                       float beta1, float beta2, float eps, float weight_decay, float beta_factor, cudaStream_t s);
+
 // ---------------------------------------------------------------------------------------------
 // SIMT contractions (gemm_simt.cu):  C = alpha * op(A) op(B) + beta * C, row-major.
 // op(X) = X or X^T (ta / tb).  M, N, K are the dimensions of the product.

@@ -60,6 +60,30 @@ def test_c1_full_trajectory():
     _run(w, w.calls, tau=2)
 
 
+def test_small_matrix_update_is_a_single_launch():
+    """A matrix with both dimensions <= 128 on the fp32 path is bound by launch latency: an update on which
+    no refresh is due is one launch of the library (the refresh calls of C1, every fifth update, take the
+    general path); parity of that kernel is what test_c1_full_trajectory and the strategy grid assert."""
+    import torch
+    import paper_2602_03515_b200 as br
+    from workloads import GradientStream, initial_weight
+    w = get_workload("c1")
+    wt = torch.from_numpy(initial_weight(w, 0).copy()).cuda()
+    opt = br.BasisRotation.from_workload(w, [wt])
+    gs = GradientStream(w, 0)
+    try:
+        per_call = []
+        for c in range(1, 9):
+            n0, _ = opt.launch_stats()
+            opt.step([torch.from_numpy(gs(c)).cuda()], 2)
+            per_call.append(opt.launch_stats()[0] - n0)
+        # calls 1-2: warm-up (no update); updates t = 1..6 at calls 3..8; t = 5 (call 7) refreshes
+        assert per_call[:2] == [0, 0] and per_call[2:6] == [1, 1, 1, 1] and per_call[6] > 10 and per_call[7] == 1
+        assert opt.sync_status() == br.BR_OK
+    finally:
+        opt.close()
+
+
 def _small(geom, src, m, n, dtype="f32", kind="iid_normal", tau=1, freq=3, scale=0.05, **kw):
     return Workload("small", [LayerSpec("W", m, n, geom, src, tau)], dtype, kind, scale, 4, tau=tau,
                     freq=freq, calls=10, gemm_prec="f32", seed=3, **kw)

@@ -95,13 +95,18 @@ typedef struct {
   int32_t power_iters; /* Power() applications per refresh, >= 1 (the paper uses 1)         */
   int32_t accum;       /* br_accum_mode                                                    */
   int32_t gemm_prec;   /* br_gemm_prec                                                     */
-  uint32_t flags;      /* reserved, 0                                                      */
+  uint32_t flags;      /* BR_FLAG_* bits, 0 by default                                     */
   /* Global-norm gradient clipping (App. D.2 of the paper uses 1.0); 0 = off.  The gradients of one
    * call, over all layers of the handle, are scaled by min(1, clip_norm / their joint L2 norm); the
    * factor belongs to the call and goes with its gradients through the delay ring. */
   float clip_norm;
   uint64_t scratch_limit_bytes; /* cap on per-step transient scratch; 0 -> library default */
 } br_hparams;
+
+/* br_hparams.flags.  BR_FLAG_DEBUG_CANARY: a debugging layout of the handle's memory, with 256 bytes of
+ * guard words behind every piece of state and scratch (a few hundred KB for a large layer set);
+ * br_debug_check_canaries tells whether any kernel wrote past the piece in front of a guard. */
+#define BR_FLAG_DEBUG_CANARY 1u
 
 /* Device-memory allocator.  NULL (or NULL members) -> cudaMalloc / cudaFree.  alloc returns a
  * DEVICE pointer aligned to at least 256 bytes, or NULL. */
@@ -273,6 +278,9 @@ BR_API br_status br_lr_warmup_cosine(int64_t step, int64_t total_steps, double w
 typedef enum { BR_INJECT_NONE = 0, BR_INJECT_LAUNCH_FAILURE = 1 } br_inject_kind;
 BR_API br_status br_debug_inject(br_handle* h, int kind, int64_t countdown);
 BR_API br_status br_debug_wait_timeout(br_handle* h, uint64_t limit_ns);
+/* Waits for the stream and checks the guard words of a handle created with BR_FLAG_DEBUG_CANARY: BR_OK, or
+ * BR_ERR_STATE with the first overwritten guard in br_last_error (also when the handle has no guards). */
+BR_API br_status br_debug_check_canaries(br_handle* h);
 
 BR_API const char* br_strerror(int status);
 /* Message of the last error on this handle (or of the last failed br_create when h is NULL). */

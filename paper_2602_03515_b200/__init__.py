@@ -13,6 +13,6 @@ from .binding import (  # noqa: F401
     br_state_bytes, br_create, br_step, br_set_lr, br_refresh_basis, br_sync_status,
     br_get_counters, br_get_basis_flags, br_set_counters, br_get_state, br_set_state, br_get_launch_stats,
     br_profile, br_get_profile, br_stage_aware_freq, br_effective_delay, br_lr_warmup_cosine, br_destroy, br_strerror, br_last_error, br_gemm_bf16, br_power_static,
-    BR_INJECT_NONE, BR_INJECT_LAUNCH_FAILURE, br_debug_inject, br_debug_wait_timeout,
+    BR_INJECT_NONE, BR_INJECT_LAUNCH_FAILURE, br_debug_inject, br_debug_wait_timeout, BR_FLAG_DEBUG_CANARY, br_debug_check_canaries,
     BasisRotation,
 )

@@ -101,6 +101,7 @@ def load_library():
         "br_destroy": ([H], C.c_int),
         "br_debug_inject": ([H, C.c_int, C.c_int64], C.c_int),
         "br_debug_wait_timeout": ([H, C.c_uint64], C.c_int),
+        "br_debug_check_canaries": ([H], C.c_int),
         "br_power_static": ([C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p], C.c_int),
         "br_strerror": ([C.c_int], C.c_char_p),
         "br_last_error": ([H], C.c_char_p),
@@ -239,6 +240,13 @@ def br_debug_inject(handle, kind: int, countdown: int = 0) -> int:
     return _check(load_library().br_debug_inject(handle, int(kind), int(countdown)), handle)
 
 
+BR_FLAG_DEBUG_CANARY = 1
+
+
+def br_debug_check_canaries(handle) -> int:
+    return _check(load_library().br_debug_check_canaries(handle), handle)
+
+
 def br_debug_wait_timeout(handle, limit_ns: int) -> int:
     return _check(load_library().br_debug_wait_timeout(handle, int(limit_ns)), handle)
 
@@ -273,7 +281,7 @@ class BasisRotation:
     def __init__(self, specs, weights, *, grad_dtype: str = "bf16", lr=1e-3, beta1=0.9, beta2=0.999,
                  eps=1e-8, weight_decay=0.0, beta_factor=-1.0, freq=10, power_iters=1,
                  accum=BR_ACCUM_EVERY_STEP, gemm_prec=BR_GEMM_BF16, scratch_limit_bytes=0, clip_norm=0.0,
-                 device=None, stream=None, use_torch_allocator=True):
+                 flags=0, device=None, stream=None, use_torch_allocator=True):
         import torch
         self._torch = torch
         assert len(specs) == len(weights)
@@ -292,7 +300,7 @@ class BasisRotation:
                                            weight=w.data_ptr()))
         self.hp = BrHparams(lr=lr, beta1=beta1, beta2=beta2, eps=eps, weight_decay=weight_decay,
                             beta_factor=beta_factor, freq=freq, power_iters=power_iters, accum=accum,
-                            gemm_prec=gemm_prec, flags=0, clip_norm=clip_norm, scratch_limit_bytes=scratch_limit_bytes)
+                            gemm_prec=gemm_prec, flags=flags, clip_norm=clip_norm, scratch_limit_bytes=scratch_limit_bytes)
         self._blocks = {}
         self._alloc = None
         if use_torch_allocator:

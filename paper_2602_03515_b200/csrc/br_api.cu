@@ -62,6 +62,7 @@ br_status validate(const br_layer_desc* layers, int n_layers, const br_hparams* 
   if (hp->freq < 1 || hp->power_iters < 1) { *err = "freq and power_iters must be >= 1"; return BR_ERR_INVALID; }
   if (hp->accum != BR_ACCUM_EVERY_STEP && hp->accum != BR_ACCUM_ON_REFRESH) { *err = "bad accum mode"; return BR_ERR_INVALID; }
   if (hp->gemm_prec != BR_GEMM_FP32 && hp->gemm_prec != BR_GEMM_BF16) { *err = "bad gemm_prec"; return BR_ERR_INVALID; }
+  if (hp->flags & ~(uint32_t)BR_FLAG_DEBUG_CANARY) { *err = "unknown bit in flags"; return BR_ERR_INVALID; }
   for (int i = 0; i < n_layers; ++i) {
     const br_layer_desc& d = layers[i];
     if (d.m < 1 || d.n < 1 || d.m > (1 << 20) || d.n > (1 << 20)) { *err = format("layer %d: bad shape %lld x %lld", i, (long long)d.m, (long long)d.n); return BR_ERR_SHAPE; }
@@ -143,6 +144,9 @@ struct br_handle {
   size_t tcq_bytes = 0;
   // tensor-core path
   TcStep* tc = nullptr;
+  // debug canaries (BR_FLAG_DEBUG_CANARY): offsets of the guards in the slab, on the host and on the device
+  std::vector<unsigned long long> guard_offsets;
+  unsigned long long* d_guard_offsets = nullptr;
   LaunchStats stats;
   std::string err;
 };
@@ -155,9 +159,15 @@ void release(br_handle* h);
 struct Bump {
   size_t off = 0;
   char* base = nullptr;
+  size_t guard = 0;                                   // debug canaries: bytes of guard behind every piece
+  std::vector<unsigned long long>* guards = nullptr;  // their offsets (collected in the pass that has a base)
   template <typename T> T* take(size_t count) {
     size_t o = off;
     off = align_up(off + count * sizeof(T));
+    if (guard) {
+      if (guards && base) guards->push_back((unsigned long long)off);
+      off += guard;
+    }
     return base ? reinterpret_cast<T*>(base + o) : nullptr;
   }
 };
@@ -165,6 +175,7 @@ struct Bump {
 // Lays out every buffer of the handle in one slab.  With base == nullptr only sizes are computed.
 void layout(br_handle* h, Bump& b, Sizes* sz) {
   const br_hparams& hp = h->hp;
+  if (hp.flags & BR_FLAG_DEBUG_CANARY) { b.guard = kAlign; b.guards = &h->guard_offsets; h->guard_offsets.clear(); }
   size_t max_numel = 0, max_k = 0, max_z = 0, n_sides = 0;
   bool any_simt = false;
   for (Layer& L : h->layers) {
@@ -693,6 +704,7 @@ void release(br_handle* h) {
   if (h->ev_consumed) cudaEventDestroy(h->ev_consumed);
   if (h->ev_copied) cudaEventDestroy(h->ev_copied);
   if (h->h_cond) cudaFreeHost(h->h_cond);
+  if (h->d_guard_offsets) cudaFree(h->d_guard_offsets);
   for (int i = 0; i < br_handle::kMaxLanes; ++i) {
     for (auto& kv : h->lanes[i].qr_graphs) if (kv.second.exec) cudaGraphExecDestroy(kv.second.exec);
     for (QrTc* t : h->lanes[i].tcq) qr_tc_destroy(t);
@@ -790,6 +802,12 @@ br_status br_create(br_handle** out, const br_layer_desc* layers, int n_layers, 
     return BR_ERR_CUDA;
   };
   if ((e = cudaMemsetAsync(h->slab, 0, sz.total, s)) != cudaSuccess) return fail("cudaMemsetAsync", e);
+  if (!h->guard_offsets.empty()) {
+    const size_t gb = sizeof(unsigned long long) * h->guard_offsets.size();
+    if ((e = cudaMalloc(reinterpret_cast<void**>(&h->d_guard_offsets), gb)) != cudaSuccess) return fail("cudaMalloc (canary table)", e);
+    if ((e = cudaMemcpyAsync(h->d_guard_offsets, h->guard_offsets.data(), gb, cudaMemcpyHostToDevice, s)) != cudaSuccess) return fail("cudaMemcpyAsync", e);
+    if ((e = guard_fill(h->slab, h->d_guard_offsets, (int)h->guard_offsets.size(), s)) != cudaSuccess) return fail("guard_fill", e);
+  }
   for (Layer& L : h->layers) {
     if (L.U && (e = set_identity(L.U, L.d.m, s)) != cudaSuccess) return fail("set_identity", e);
     if (L.V && (e = set_identity(L.V, L.d.n, s)) != cudaSuccess) return fail("set_identity", e);
@@ -1004,6 +1022,26 @@ br_status br_debug_inject(br_handle* h, int kind, int64_t countdown) {
   if (kind == BR_INJECT_NONE) { h->stats.fail_countdown = -1; return BR_OK; }
   if (kind != BR_INJECT_LAUNCH_FAILURE || countdown < 0) { h->err = "unknown injection kind or negative countdown"; return BR_ERR_INVALID; }
   h->stats.fail_countdown = countdown;
+  return BR_OK;
+}
+
+br_status br_debug_check_canaries(br_handle* h) {
+  br_status st = check_handle(h);
+  if (st != BR_OK) return st;
+  if (h->guard_offsets.empty()) { h->err = "the handle was created without BR_FLAG_DEBUG_CANARY"; return BR_ERR_STATE; }
+  int* first_bad = h->d_status + 8;                   // a spare word of the status area
+  const int none = 0x7fffffff;
+  BR_CUDA(h, cudaStreamSynchronize(h->stream));
+  BR_CUDA(h, cudaMemcpy(first_bad, &none, sizeof(int), cudaMemcpyHostToDevice));
+  BR_CUDA(h, guard_check(h->slab, h->d_guard_offsets, (int)h->guard_offsets.size(), first_bad, h->stream));
+  BR_CUDA(h, cudaStreamSynchronize(h->stream));
+  int bad = none;
+  BR_CUDA(h, cudaMemcpy(&bad, first_bad, sizeof(int), cudaMemcpyDeviceToHost));
+  if (bad != none) {
+    h->err = format("canary %d of %zu (slab offset %llu) was overwritten: the piece in front of it was overrun", bad,
+                    h->guard_offsets.size(), h->guard_offsets[(size_t)bad]);
+    return BR_ERR_STATE;
+  }
   return BR_OK;
 }
 

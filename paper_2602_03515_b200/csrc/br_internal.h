@@ -108,6 +108,10 @@ cudaError_t small_step(int64_t m, int64_t n, bool left, bool right, const void* 
                        float* M, float* V2, float* U, float* V, float* L, float* R, float* W, int accumulate, float lr,
                        float beta1, float beta2, float eps, float weight_decay, float beta_factor, cudaStream_t s);
 
+// Debug canaries (BR_FLAG_DEBUG_CANARY): n guards of 256 bytes at byte offsets offs[] (DEVICE array) of the slab.
+cudaError_t guard_fill(char* slab, const unsigned long long* offs, int n, cudaStream_t s);
+cudaError_t guard_check(const char* slab, const unsigned long long* offs, int n, int* first_bad, cudaStream_t s);
+
 // ---------------------------------------------------------------------------------------------
 // SIMT contractions (gemm_simt.cu):  C = alpha * op(A) op(B) + beta * C, row-major.
 // op(X) = X or X^T (ta / tb).  M, N, K are the dimensions of the product.

@@ -417,4 +417,28 @@ cudaError_t f64_to_f32(const double* X, float* out, int64_t numel, cudaStream_t 
   return cudaGetLastError();
 }
 
+// ---- debug canaries: 256-byte guard words behind every piece of the handle's slab ----
+namespace {
+constexpr unsigned int kGuardWord = 0xC5C5C5C5u;
+__global__ void k_guard_fill(char* slab, const unsigned long long* offs, int n) {
+  const int g = blockIdx.x;
+  if (g < n) reinterpret_cast<unsigned int*>(slab + offs[g])[threadIdx.x] = kGuardWord;
+}
+__global__ void k_guard_check(const char* slab, const unsigned long long* offs, int n, int* first_bad) {
+  const int g = blockIdx.x;
+  if (g < n && reinterpret_cast<const unsigned int*>(slab + offs[g])[threadIdx.x] != kGuardWord) atomicMin(first_bad, g);
+}
+}  // namespace
+
+cudaError_t guard_fill(char* slab, const unsigned long long* offs, int n, cudaStream_t s) {
+  if (n <= 0) return cudaSuccess;
+  k_guard_fill<<<n, 64, 0, s>>>(slab, offs, n);
+  return cudaGetLastError();
+}
+cudaError_t guard_check(const char* slab, const unsigned long long* offs, int n, int* first_bad, cudaStream_t s) {
+  if (n <= 0) return cudaSuccess;
+  k_guard_check<<<n, 64, 0, s>>>(slab, offs, n, first_bad);
+  return cudaGetLastError();
+}
+
 }  // namespace br

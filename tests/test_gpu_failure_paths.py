@@ -178,3 +178,46 @@ def test_failed_enqueue_inside_forced_refresh():
         finally:
             opt.close()
     torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("prec", ["fp32", "bf16"])
+def test_debug_canaries_stay_intact_and_catch_an_overrun(prec):
+    """BR_FLAG_DEBUG_CANARY puts guard words behind every piece of the handle's memory.  A run through
+    steps and refreshes (factor products, rotations, refresh lanes, tensor-core scratch) leaves all of
+    them intact; a word overwritten from the host side, inside the test's own allocation, is reported
+    with its position.  A handle without the flag has no guards to check."""
+    import torch
+    import paper_2602_03515_b200 as br
+    gp = br.BR_GEMM_BF16 if prec == "bf16" else br.BR_GEMM_FP32
+    specs = [LayerSpec("a", 128, 136, GEOM_BI, SRC_SECOND, 2), LayerSpec("b", 72, 264, GEOM_UNI, SRC_FIRST, 1),
+             LayerSpec("c", 40, 24, GEOM_BI, SRC_SECOND, 0)]
+    ws = [torch.randn(s.m, s.n, device="cuda") * 0.02 for s in specs]
+    dt = "bf16" if prec == "bf16" else "f32"
+    tdt = torch.bfloat16 if prec == "bf16" else torch.float32
+    opt = br.BasisRotation(specs, ws, grad_dtype=dt, gemm_prec=gp, freq=3, flags=br.BR_FLAG_DEBUG_CANARY)
+    try:
+        for _ in range(9):
+            opt.step([(torch.randn(s.m, s.n, device="cuda") * 0.01).to(tdt) for s in specs], -1)
+        opt.refresh_basis(-1)
+        assert opt.sync_status() == br.BR_OK
+        assert br.br_debug_check_canaries(opt.handle) == br.BR_OK
+        # the slab is the one block the torch-backed allocator handed out: find a guard in it and damage it
+        (slab,) = opt._blocks.values()
+        host = slab.cpu().numpy()
+        word = np.frombuffer(host.tobytes(), dtype=np.uint32)
+        runs = np.flatnonzero(word == 0xC5C5C5C5)
+        assert len(runs) >= 64 * 10                       # dozens of guards of 64 words each
+        slab[int(runs[100]) * 4] = 0                      # one byte of one guard
+        torch.cuda.synchronize()
+        with pytest.raises(br.BrError) as e:
+            br.br_debug_check_canaries(opt.handle)
+        assert e.value.status == br.BR_ERR_STATE and "canary" in str(e.value)
+    finally:
+        opt.close()
+    plain = br.BasisRotation(specs[2:], ws[2:], grad_dtype=dt, gemm_prec=gp)
+    try:
+        with pytest.raises(br.BrError) as e:
+            br.br_debug_check_canaries(plain.handle)
+        assert e.value.status == br.BR_ERR_STATE
+    finally:
+        plain.close()

@@ -64,6 +64,13 @@ def test_host_validation(br):
     with pytest.raises(br.BrError) as e:
         br.br_state_bytes([_desc(br, 4, 4, 7, 2)], _hp(br))
     assert e.value.status == br.BR_ERR_INVALID
+    with pytest.raises(br.BrError) as e:
+        br.br_state_bytes([_desc(br, 4, 4, 2, 2)], _hp(br, flags=2))
+    assert e.value.status == br.BR_ERR_INVALID
+    # the debugging layout adds one 256-byte guard per piece of memory
+    plain, _ = br.br_state_bytes([_desc(br, 64, 32, 2, 2, tau=2)], _hp(br))
+    guarded, _ = br.br_state_bytes([_desc(br, 64, 32, 2, 2, tau=2)], _hp(br, flags=br.BR_FLAG_DEBUG_CANARY))
+    assert guarded > plain and (guarded - plain) % 256 == 0
     assert br.br_strerror(br.BR_ERR_TAU) == "tau out of range"
     assert br.br_destroy(None) == br.BR_OK
 

@@ -605,3 +605,23 @@ def test_spiral_loss_definition_and_the_papers_alignment_claim():
     assert stats["misaligned"][1] > 1.5 * stats["aligned"][1]              # misalignment: more oscillation
     for name in stats:
         assert stats[name][2] > 2.0 * stats[name][1]                      # delay: more again
+
+
+def test_golden_c1_trajectory_is_reproduced():
+    """tests/golden/c1_trajectory.txt (written by tests/golden/make_c1_trajectory.py from the oracle alone):
+    the oracle of today reproduces the stored C1 trajectory -- counters exactly, values to 1e-9 relative (the host BLAS may order its sums differently).
+    Not a pin to the paper (it prints no worked example); a guard against accidental changes of the
+    oracle's arithmetic, e.g. while a faster QR step is added beside the written-out one."""
+    import importlib.util
+    import os
+    here = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
+    spec = importlib.util.spec_from_file_location("make_c1_trajectory", os.path.join(here, "make_c1_trajectory.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    stored = [l.split() for l in open(os.path.join(here, "c1_trajectory.txt")) if not l.startswith("#")]
+    now = list(mod.rows())
+    assert len(stored) == len(now) == 20
+    for line, (c, st, t, rc, vals) in zip(stored, now):
+        assert [int(x) for x in line[:4]] == [c, st, t, rc]
+        ref = np.array([float(x) for x in line[4:]])
+        assert np.all(np.abs(np.array(vals) - ref) <= 1e-9 * np.abs(ref) + 1e-300)

@@ -35,7 +35,7 @@ UNIT = "params/s"
 
 # ---------------------------------------------------------------------------------------------
 def algorithmic_flops_per_step(w) -> float:
-    """Contraction work the method itself prescribes per step (Alg. 1 lines 8-11 and the factor
+    """Contraction work the method itself prescribes per step (Alg. 1 (rotation, second moment, weight update) and the factor
     EMAs of Alg. 2): bilateral/2nd 8mn(m+n); one-sided on side s: 8 s^2 max (2nd) or 6 s^2 max (1st)."""
     f = 0.0
     for l in w.layers:

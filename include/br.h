@@ -143,7 +143,7 @@ typedef enum {
   BR_BUF_R = 6,   /* n*n fp32 (S=2nd, right side rotated)             */
   BR_BUF_RING = 7, /* tau_max * m*n gradients in grad_dtype, slot-major */
   /* m*n fp32: the momentum in rotated coordinates, M~ = U^T M V.  Between two refreshes
-   * M~_t = beta1 M~_{t-1} + (1-beta1) U^T G_t V holds exactly (Alg. 1 line 4 is linear), and this is
+   * M~_t = beta1 M~_{t-1} + (1-beta1) U^T G_t V holds exactly (Alg. 1 (momentum update) is linear), and this is
    * what layers on the tensor-core path store; BR_BUF_M converts on the way in and out with fp32
    * products.  A checkpoint that must resume bit-identically saves and restores this buffer (after
    * U and V) instead of BR_BUF_M.  Absent for layers on the fp32 path. */
@@ -214,7 +214,7 @@ typedef struct {
   double tc_ms;          /* tensor-core contraction launches                                  */
   double tc_flops;       /* floating-point operations those launches issued                   */
   int64_t tc_launches;
-  double ema_ms;         /* momentum EMA launches (Alg. 1 line 4, with the bf16 hi/lo of M)    */
+  double ema_ms;         /* momentum EMA launches (Alg. 1 (momentum update), with the bf16 hi/lo of M)    */
   double ema_bytes;      /* bytes those launches must move (gradient, M in and out, hi/lo)    */
   int64_t ema_launches;
   double refresh_ms;     /* Power() spans: power product + QR + conversions                   */

@@ -244,7 +244,7 @@ class OracleLayer:
 
     # -- pieces of Algorithm 1 / 2 -------------------------------------------------
     def rotate(self, X):
-        """U^T X V with the identity on an unrotated side (Alg. 1, lines 8-9)."""
+        """U^T X V with the identity on an unrotated side (Alg. 1 (rotation of G and M))."""
         Y = X
         if self.left:
             Y = self.U.T @ Y
@@ -253,7 +253,7 @@ class OracleLayer:
         return Y
 
     def rotate_back(self, X):
-        """U X V^T (Alg. 1, line 11)."""
+        """U X V^T (Alg. 1 (weight update))."""
         Y = X
         if self.left:
             Y = self.U @ Y
@@ -358,18 +358,18 @@ class Oracle:
             lay.W, lay.M, lay.V2, lay.last_dW = plain_adam_update(
                 lay.W, lay.M, lay.V2, G, hp.lr, hp.beta1, hp.beta2, hp.eps, hp.weight_decay)
             return False
-        # Alg. 1 line 4
+        # Alg. 1 (momentum update)
         lay.M = hp.beta1 * lay.M + (1.0 - hp.beta1) * G
         second = lay.src == SRC_SECOND
         if second and hp.accum == "every_step":
             lay.accumulate_factors(G, self._beta_factor())
-        # Alg. 1 lines 5-6
+        # Alg. 1 (periodic refresh)
         freq = lay.freq if lay.freq > 0 else hp.freq
         if lay.t % freq == 0:
             if second and hp.accum == "on_refresh":
                 lay.accumulate_factors(G, self._beta_factor())
             deficient = lay.refresh(hp.power_iters, QR_IMPLS[hp.qr])
-        # Alg. 1 lines 8-11
+        # Alg. 1 (rotation, second moment, weight update)
         Gt = lay.rotate(G)
         Mt = lay.rotate(lay.M)
         lay.V2 = hp.beta2 * lay.V2 + (1.0 - hp.beta2) * Gt * Gt

@@ -629,7 +629,7 @@ br_status update_layer_simt(br_handle* h, Layer& L, const void* G, const float* 
   const int64_t m = L.d.m, n = L.d.n, mn = m * n;
   const int bf = L.d.grad_dtype == BR_BF16;
   br_status st;
-  // Alg. 1 line 4 (and widen a bf16 gradient once)
+  // Alg. 1 (momentum update) (and widen a bf16 gradient once)
   // (a clipped gradient is materialised in fp32 too: everything below works on the scaled values)
   const bool copy = bf || gscale != nullptr;
   BR_CUDA(h, ema_momentum(L.M, G, bf, mn, hp.beta1, copy ? h->sG : nullptr, nullptr, nullptr, gscale, s));
@@ -637,18 +637,18 @@ br_status update_layer_simt(br_handle* h, Layer& L, const void* G, const float* 
   const float* G32 = copy ? h->sG : reinterpret_cast<const float*>(G);
   const bool second = L.d.src == BR_SRC_SECOND;
   if (second && hp.accum == BR_ACCUM_EVERY_STEP && (st = accumulate_factors_simt(h, L, G32)) != BR_OK) return st;
-  // Alg. 1 lines 5-6
+  // Alg. 1 (periodic refresh)
   if (L.t % L.freq == 0) {
     if (second && hp.accum == BR_ACCUM_ON_REFRESH && (st = accumulate_factors_simt(h, L, G32)) != BR_OK) return st;
     if ((st = refresh_layer(h, L)) != BR_OK) return st;
   }
-  // Alg. 1 lines 8-9
+  // Alg. 1 (rotation of G and M)
   if ((st = rotate_simt(h, L, G32, h->sT, h->sGt)) != BR_OK) return st;
   if ((st = rotate_simt(h, L, L.M, h->sT, h->sMt)) != BR_OK) return st;
-  // lines 10-11, element-wise part: X overwrites sMt
+  // second-moment update and scaling, element-wise part: X overwrites sMt
   BR_CUDA(h, second_moment_scale(L.V2, h->sGt, h->sMt, mn, hp.beta2, hp.eps, s));
   count(h);
-  // line 11: W <- (1 - eta lambda) W - eta U X V^T
+  // weight update: W <- (1 - eta lambda) W - eta U X V^T
   const float decay = 1.0f - hp.lr * hp.weight_decay;
   float* W = L.d.weight;
   if (L.left && L.right) {

@@ -64,7 +64,7 @@ struct LaunchStats {
 // ---------------------------------------------------------------------------------------------
 cudaError_t set_identity(float* Q, int64_t k, cudaStream_t s);
 
-// Alg. 1 line 4: M <- beta1 M + (1-beta1) G.  G is fp32 or bf16 (g_is_bf16).  Optional outputs:
+// Alg. 1 (momentum update): M <- beta1 M + (1-beta1) G.  G is fp32 or bf16 (g_is_bf16).  Optional outputs:
 // Gf32 (G widened to fp32), Mh/Ml (bf16 hi/lo split of the new M).
 // gscale (optional, DEVICE): clipping factor the gradient is multiplied by
 cudaError_t ema_momentum(float* M, const void* G, int g_is_bf16, int64_t numel, float beta1,
@@ -78,7 +78,7 @@ cudaError_t clip_factor(const void* const* grads, const int64_t* numel, const in
 cudaError_t plain_adam(float* W, float* M, float* V, const void* G, int g_is_bf16, int64_t numel,
                        float lr, float beta1, float beta2, float eps, float wd, const float* gscale, cudaStream_t s);
 
-// Alg. 1 lines 10-11 (element-wise part): V~ <- beta2 V~ + (1-beta2) G~^2 ; X = M~/sqrt(V~+eps).
+// Alg. 1 (second-moment update and scaling) (element-wise part): V~ <- beta2 V~ + (1-beta2) G~^2 ; X = M~/sqrt(V~+eps).
 // X overwrites Mt.
 cudaError_t second_moment_scale(float* V2, const float* Gt, float* Mt, int64_t numel, float beta2,
                                 float eps, cudaStream_t s);
@@ -97,11 +97,11 @@ cudaError_t split3_f64(const double* X, int64_t ld, int64_t rows, int64_t cols, 
 cudaError_t split3_f32(const float* X, int64_t numel, __nv_bfloat16* p1, __nv_bfloat16* p2, __nv_bfloat16* p3,
                        cudaStream_t s);
 cudaError_t sub_f32_from_f64(double* A, int64_t ld, int64_t rows, int64_t cols, const float* D, cudaStream_t s);
-// out <- beta1 M + (1-beta1) G (out-of-place form of Alg. 1 line 4)
+// out <- beta1 M + (1-beta1) G (out-of-place form of Alg. 1 (momentum update))
 cudaError_t ema_out(float* out, const float* M, const void* G, int g_is_bf16, int64_t numel, float beta1,
                     const float* gscale, cudaStream_t s);
 
-// One whole update (Alg. 1 lines 4, 8-11 and the factor EMAs of Alg. 2, no refresh) of a matrix with both
+// One whole update (Alg. 1 (momentum, rotation, second moment, weight update) and the factor EMAs of Alg. 2, no refresh) of a matrix with both
 // dimensions <= 128 in a single one-CTA launch (small_step.cu).  accumulate: update L and R as well.
 bool small_step_eligible(int64_t m, int64_t n, bool left, bool right);
 cudaError_t small_step(int64_t m, int64_t n, bool left, bool right, const void* G, int g_is_bf16, const float* gscale,
@@ -176,7 +176,7 @@ enum Epilogue : int32_t {
   EPI_SPLIT_BF16 = 1,   // Dh <- bf16(acc), Dl <- bf16(acc - Dh)   (Dl optional)
   EPI_SECOND_MOMENT = 2,// D(V~) <- beta*D + alpha*acc^2
   EPI_SCALE_BF16 = 3,   // Dh(X) <- bf16(acc / sqrt(D(V~) + eps))
-  // Alg. 1 lines 4, 10, 11 in rotated coordinates, acc = G~:
+  // Alg. 1 (momentum and second-moment updates, scaling) in rotated coordinates, acc = G~:
   //   D2(M~) <- beta1 D2 + (1-beta1) acc ; D(V~) <- beta D + alpha acc^2 ; Dh(X) <- bf16(D2 / sqrt(D + eps))
   EPI_ROTATED_ADAM = 4
 };

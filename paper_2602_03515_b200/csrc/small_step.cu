@@ -1,9 +1,9 @@
 // One rotated-Adam update of a small weight matrix (both dimensions at most 128) in a single launch of
-// a single CTA: Alg. 1 lines 4 and 8-11 and the factor EMAs of Alg. 2, with every operand staged in
+// a single CTA: Alg. 1 (momentum, rotation, second moment, weight update) and the factor EMAs of Alg. 2, with every operand staged in
 // shared memory and fp32 FFMA dot products.  A matrix of this size is bound by launch latency, not by
 // arithmetic: the general fp32 path takes about fifteen launches per update (momentum EMA, two factor
 // products, four rotations, the element-wise second-moment step, two back rotations, copies), this
-// kernel one.  The refresh of the bases (Alg. 1 lines 5-6) is not part of it: a call on which a refresh
+// kernel one.  The refresh of the bases (Alg. 1 (periodic refresh)) is not part of it: a call on which a refresh
 // is due goes through the general path.
 #include "br_internal.h"
 
@@ -41,7 +41,7 @@ __global__ void __launch_bounds__(kThreads) k_small_step(SmallArgs a) {
   float* sV = sU + (a.left ? m * lm : 0);
   const int t = threadIdx.x;
   const float gs = a.gscale ? *a.gscale : 1.0f;
-  // Alg. 1 line 4: M <- beta1 M + (1 - beta1) G
+  // Alg. 1 (momentum update): M <- beta1 M + (1 - beta1) G
   for (int i = t; i < mn; i += kThreads) {
     const float g = gs * load_g(a.G, a.g_is_bf16, i);
     const float mo = a.beta1 * a.M[i] + (1.0f - a.beta1) * g;
@@ -69,7 +69,7 @@ __global__ void __launch_bounds__(kThreads) k_small_step(SmallArgs a) {
         a.R[e] = b * a.R[e] + ob * s;
       }
   }
-  // Alg. 1 lines 8-9, first side: T1 = U^T G, T2 = U^T M (or the matrices themselves)
+  // Alg. 1 (rotation of G and M), first side: T1 = U^T G, T2 = U^T M (or the matrices themselves)
   for (int e = t; e < mn; e += kThreads) {
     const int i = e / n, j = e % n;
     float s1 = sG[i * ln + j], s2 = sM[i * ln + j];
@@ -80,7 +80,7 @@ __global__ void __launch_bounds__(kThreads) k_small_step(SmallArgs a) {
     sT1[i * ln + j] = s1; sT2[i * ln + j] = s2;
   }
   __syncthreads();
-  // second side: G~ = T1 V, M~ = T2 V; lines 10-11: V~ <- beta2 V~ + (1 - beta2) G~^2, X = M~ / sqrt(V~ + eps)
+  // second side: G~ = T1 V, M~ = T2 V; then the second moment and the scaling: V~ <- beta2 V~ + (1 - beta2) G~^2, X = M~ / sqrt(V~ + eps)
   for (int e = t; e < mn; e += kThreads) {
     const int i = e / n, j = e % n;
     float gt = sT1[i * ln + j], mt = sT2[i * ln + j];
@@ -93,7 +93,7 @@ __global__ void __launch_bounds__(kThreads) k_small_step(SmallArgs a) {
     sG[i * ln + j] = mt / sqrtf(v2 + a.eps);        // X (G is not needed any more)
   }
   __syncthreads();
-  // line 11: W <- decay W - eta U X V^T
+  // weight update: W <- decay W - eta U X V^T
   for (int e = t; e < mn; e += kThreads) {
     const int i = e / n, j = e % n;
     float y = sG[i * ln + j];

@@ -2,7 +2,7 @@
 //
 // Between two refreshes the bases U, V are constant, so the rotated momentum obeys
 //   M~_t = U^T M_t V = beta1 M~_{t-1} + (1 - beta1) U^T G_t V
-// exactly (Alg. 1 line 4 is linear).  The tensor-core path therefore keeps M~ as its state instead
+// exactly (Alg. 1 (momentum update) is linear).  The tensor-core path therefore keeps M~ as its state instead
 // of M: the momentum is never rotated, which removes one of the four two-sided products of Alg. 1,
 // and its EMA joins the second-moment update and the Adam scaling in one fused epilogue.  Only a
 // refresh needs M itself: the due layers are re-expressed, M = U M~ V^T with the old basis before
@@ -12,12 +12,12 @@
 // every phase is ONE grouped launch over all layers of the chunk:
 //
 //   factors   L <- b L + (1-b) G G^T , R <- b R + (1-b) G^T G            (Alg. 2)
-//   [refresh of the layers that are due, bracketed by the re-expression]  (Alg. 1 lines 5-6)
-//   fwd1      T = U^T G  (or T = G V when n > m: the larger side first) -> bf16 hi/lo   (Alg. 1 line 8, first side)
+//   [refresh of the layers that are due, bracketed by the re-expression]  (Alg. 1 (periodic refresh))
+//   fwd1      T = U^T G  (or T = G V when n > m: the larger side first) -> bf16 hi/lo   (Alg. 1 (rotation of G), first side)
 //   adam      G~ = T V, fused epilogue: M~ <- b1 M~ + (1-b1) G~ ; V~ <- b2 V~ + (1-b2) G~^2 ;
-//             X = M~ / sqrt(V~ + eps)                                      (lines 4, 8-11)
+//             X = M~ / sqrt(V~ + eps)                                      (momentum, rotation, second moment, weight update)
 //   back1     Y = U X
-//   wwrite    W <- (1 - eta lambda) W - eta Y V^T     fused epilogue      (line 11)
+//   wwrite    W <- (1 - eta lambda) W - eta Y V^T     fused epilogue      (weight update)
 //
 // fp32 operands of the forward rotations (U, V, T, and M / M~ in the re-expression) enter as a
 // bf16 hi/lo pair and the products hi*hi + lo*hi + hi*lo are accumulated in tensor memory: a single

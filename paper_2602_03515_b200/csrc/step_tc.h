@@ -12,7 +12,7 @@ struct Layer {
   bool left = false, right = false;   // which sides carry a rotation
   bool use_tc = false;                // contractions run on the tcgen05 tile kernel
   int freq = 1;
-  // M holds the momentum of Alg. 1 line 4: in the original space on the fp32 path, in ROTATED
+  // M holds the momentum of Alg. 1 (momentum update): in the original space on the fp32 path, in ROTATED
   // coordinates (M~ = U^T M V) on the tensor-core path (see step_tc.cu)
   float *M = nullptr, *V2 = nullptr, *U = nullptr, *V = nullptr, *L = nullptr, *R = nullptr;
   float* Morig = nullptr;             // tensor-core layers with S = 1st: M_t in the original space for a refresh
